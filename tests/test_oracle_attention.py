@@ -1,0 +1,172 @@
+"""Pins for the oracle's attention, split partials and Eq. 5 reduction (CPU only)."""
+import numpy as np
+import pytest
+
+from paper_2604_16957_b200 import inputs as I
+
+
+def _cache(oracle, shape, S, seed, S_cap=None, lens=None):
+    k, v = I.make_kv(shape, S, seed)
+    cache = oracle.Cache(shape.B, shape.H_kv, S_cap or S, shape.d)
+    cache.append(k, v)
+    if lens is not None:
+        cache.lens[:] = lens
+    return cache
+
+
+def _dequant(oracle, cache):
+    return (oracle.dequant_rows(cache.k_packed, cache.k_scale, cache.k_zero),
+            oracle.dequant_rows(cache.v_packed, cache.v_scale, cache.v_zero))
+
+
+def test_softmax_weights_sum_to_one(oracle):
+    cache = _cache(oracle, I.TINY, 256, 1)
+    q = I.make_q(I.TINY, 1)
+    for h in range(4):
+        w = oracle.attention_weights(cache, q, I.TINY.alpha, 0, h)
+        assert w.shape == (256,) and w.min() >= 0
+        assert abs(w.sum() - 1.0) < 1e-12
+
+
+def test_matches_library_attention_on_dequantised_values(oracle):
+    """The definition, evaluated by a library routine (torch fp64 SDPA) on the dequantised K, V."""
+    import torch
+    sh = I.Shape("t", 2, 8, 2, 64, 0.37, k_outlier_channels=2)
+    cache = _cache(oracle, sh, 100, 21)
+    q = I.make_q(sh, 21)
+    got = oracle.attention(cache, q, sh.alpha)
+    kd, vd = _dequant(oracle, cache)
+    G = sh.H_q // sh.H_kv
+    kt = torch.from_numpy(kd).repeat_interleave(G, dim=1)  # consecutive query heads share a KV head
+    vt = torch.from_numpy(vd).repeat_interleave(G, dim=1)
+    qt = torch.from_numpy(q.astype(np.float64))[:, :, None, :]
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, scale=sh.alpha)[:, :, 0, :].numpy()
+    assert np.abs(got - ref).max() < 1e-12
+
+
+def test_brute_force_tiny_python_loops(oracle):
+    """Pure-Python evaluation from the unpacked codes: softmax(alpha q.k^) weighted sum of v^."""
+    import math
+    sh = I.Shape("t", 1, 2, 1, 32, 0.5)
+    cache = _cache(oracle, sh, 5, 33)
+    q = I.make_q(sh, 33).astype(np.float64)
+    kc, vc = oracle.unpack_nibbles(cache.k_packed), oracle.unpack_nibbles(cache.v_packed)
+    got = oracle.attention(cache, q.astype(np.float16), sh.alpha)
+    for h in range(2):
+        scores, vrows = [], []
+        for i in range(5):
+            sk, zk = float(cache.k_scale[0, 0, i, 0]), float(cache.k_zero[0, 0, i, 0])
+            sv, zv = float(cache.v_scale[0, 0, i, 0]), float(cache.v_zero[0, 0, i, 0])
+            scores.append(sh.alpha * sum(float(q[0, h, c]) * (int(kc[0, 0, i, c]) - zk) * sk for c in range(32)))
+            vrows.append([(int(vc[0, 0, i, c]) - zv) * sv for c in range(32)])
+        mx = max(scores)
+        p = [math.exp(a - mx) for a in scores]
+        out = [sum(p[i] * vrows[i][c] for i in range(5)) / sum(p) for c in range(32)]
+        assert np.abs(got[0, h] - np.array(out)).max() < 1e-13
+
+
+def test_algorithm1_one_pass_equals_two_pass_definition(oracle):
+    sh = I.Shape("t", 2, 4, 2, 64, 0.125)
+    cache = _cache(oracle, sh, 300, 8, lens=[300, 17])
+    q = I.make_q(sh, 8)
+    full = oracle.attention(cache, q, sh.alpha)
+    for b in range(2):
+        for h in range(4):
+            assert np.abs(oracle.algorithm1(cache, q, sh.alpha, b, h) - full[b, h]).max() < 1e-12
+
+
+def test_constant_v_returns_v(oracle):
+    sh = I.Shape("t", 1, 4, 2, 64, 0.125)
+    k, _ = I.make_kv(sh, 64, 12)
+    # (a) every token has the same V row: output is that row's dequantised value
+    row = I.make_kv(sh, 1, 13)[1]
+    v = np.repeat(row, 64, axis=2)
+    cache = oracle.Cache(1, 2, 64, 64)
+    cache.append(k, v)
+    out = oracle.attention(cache, I.make_q(sh, 12), sh.alpha)
+    vd = oracle.dequant_rows(cache.v_packed, cache.v_scale, cache.v_zero)
+    for h in range(4):
+        assert np.abs(out[0, h] - vd[0, h // 2, 0]).max() < 1e-12
+    # (b) all elements equal (degenerate groups): output equals the constant exactly
+    v2 = np.full_like(v, np.float16(-2.75))
+    cache2 = oracle.Cache(1, 2, 64, 64)
+    cache2.append(k, v2)
+    out2 = oracle.attention(cache2, I.make_q(sh, 12), sh.alpha)
+    assert np.abs(out2 - (-2.75)).max() < 1e-12
+
+
+def test_single_token_zero_query_and_permutation(oracle):
+    sh = I.Shape("t", 1, 4, 2, 64, 0.125)
+    cache = _cache(oracle, sh, 50, 14)
+    kd, vd = _dequant(oracle, cache)
+    q = I.make_q(sh, 14)
+    # S = 1: the output is v^_0
+    c1 = _cache(oracle, sh, 50, 14, lens=[1])
+    o1 = oracle.attention(c1, q, sh.alpha)
+    for h in range(4):
+        assert np.array_equal(o1[0, h], vd[0, h // 2, 0])
+    # q = 0: uniform weights -> mean of v^
+    o0 = oracle.attention(cache, np.zeros_like(q), sh.alpha)
+    for h in range(4):
+        assert np.abs(o0[0, h] - vd[0, h // 2].mean(0)).max() < 1e-12
+    # permuting the tokens of the cache leaves the output unchanged
+    perm = np.random.default_rng(1).permutation(50)
+    pc = oracle.Cache(1, 2, 50, 64)
+    for dst, src in zip(pc.arrays(), cache.arrays()):
+        dst[:] = src[:, :, perm]
+    pc.lens[:] = 50
+    assert np.abs(oracle.attention(pc, q, sh.alpha) - oracle.attention(cache, q, sh.alpha)).max() < 1e-12
+
+
+def test_gqa_head_mapping(oracle):
+    sh = I.Shape("t", 1, 8, 2, 64, 0.125)
+    cache = _cache(oracle, sh, 40, 15)
+    q = I.make_q(sh, 15)
+    q[0, :] = q[0, 0]  # identical queries: heads 0..3 share KV head 0, heads 4..7 share KV head 1
+    out = oracle.attention(cache, q, sh.alpha)
+    for h in range(1, 4):
+        assert np.array_equal(out[0, h], out[0, 0])
+    for h in range(5, 8):
+        assert np.array_equal(out[0, h], out[0, 4])
+    assert np.abs(out[0, 0] - out[0, 4]).max() > 1e-3
+    # heads restriction computes the same rows
+    part = oracle.attention(cache, q, sh.alpha, heads=(4, 6))
+    assert np.array_equal(part[0, 4:6], out[0, 4:6]) and np.all(part[0, :4] == 0) and np.all(part[0, 6:] == 0)
+
+
+def test_attn_scale_is_a_plain_multiplier(oracle):
+    sh = I.Shape("t", 1, 4, 2, 64, 0.25)
+    cache = _cache(oracle, sh, 40, 16)
+    q = I.make_q(sh, 16)
+    a = oracle.attention(cache, q, 0.25)
+    b = oracle.attention(cache, (q.astype(np.float32) * 0.25).astype(np.float16), 1.0)  # exact: power of two
+    assert np.abs(a - b).max() < 1e-12
+    assert np.abs(a - oracle.attention(cache, q, 1.0)).max() > 1e-3
+
+
+@pytest.mark.parametrize("bounds", [[0, 300], [0, 1, 300], [0, 0, 150, 150, 299, 300], [0, 64, 128, 192, 256, 300],
+                                    [0, 300, 300]])
+def test_split_partials_recombine_by_eq5(oracle, bounds):
+    sh = I.Shape("t", 2, 4, 2, 64, 0.125)
+    cache = _cache(oracle, sh, 300, 17, lens=[300, 200])
+    q = I.make_q(sh, 17)
+    b2 = np.array([bounds, [min(x, 200) for x in bounds]], np.int32)
+    o, m, l = oracle.attention_partials(cache, q, sh.alpha, b2)
+    full = oracle.attention(cache, q, sh.alpha)
+    assert np.abs(oracle.combine(o, m, l) - full).max() < 1e-12
+    # empty splits report (0, -inf, 0)
+    empty = np.diff(b2, axis=1) == 0
+    for b in range(2):
+        for c in np.nonzero(empty[b])[0]:
+            assert np.all(l[b, :, c] == 0) and np.all(np.isneginf(m[b, :, c])) and np.all(o[b, :, c] == 0)
+    # partial outputs are normalised: a one-token split returns that token's v^
+    if bounds[:2] == [0, 1]:
+        vd = oracle.dequant_rows(cache.v_packed, cache.v_scale, cache.v_zero)
+        assert np.array_equal(o[0, 0, 0], vd[0, 0, 0]) and l[0, 0, 0] == 1.0
+
+
+def test_zero_length_sequence_gives_zero(oracle):
+    sh = I.Shape("t", 2, 4, 2, 64, 0.125)
+    cache = _cache(oracle, sh, 10, 18, lens=[0, 10])
+    out = oracle.attention(cache, I.make_q(sh, 18), sh.alpha)
+    assert np.all(out[0] == 0) and np.abs(out[1]).max() > 0
