@@ -1,0 +1,164 @@
+/*
+ * tq.h -- C ABI of libtq: fused int4 compressed-domain decode attention for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the decode-time hot path of "Open-TQ-Metal": the KV cache is kept in
+ * per-group asymmetric int4 (Sec. 2.1, Eq. 2-3), new tokens are quantised and appended in
+ * place, and single-query attention is computed directly on the packed cache (Sec. 3.1,
+ * Algorithm 1) with split-K over the sequence (Sec. 3.2) followed by the reduction of Eq. 5.
+ *
+ * General rules
+ *   - Every pointer named below is a DEVICE pointer unless it says "host".  The caller owns all
+ *     memory; the library allocates nothing, keeps no state between calls and never
+ *     synchronises.  Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream) and is ordered by it.
+ *   - All device pointers must be 16-byte aligned.
+ *   - Every entry point returns a tq_result.  Errors that the host can see (null pointer, bad
+ *     shape, bad alignment, workspace too small) are returned before anything is launched.
+ *   - Conditions only the device can see (a full cache, an empty sequence) OR bits into the
+ *     caller's `status` word (int32 in device memory, may be NULL) and the offending piece of
+ *     work is skipped; kernels never trap and contain no unbounded wait.
+ *   - fp16 means IEEE binary16; such buffers are declared `void*` / `uint16_t*` (bit patterns).
+ *
+ * Data format (Sec. 2.1).  A K or V vector of `d` elements (one token, one KV head) is cut into
+ * d/32 groups of 32 consecutive elements.  Each group stores
+ *     scale s = fp16((max - min) / 15),   zero z = fp16(-min / s)   (z is real-valued, not an integer)
+ *     code  q = clamp(round_half_even(x / s + z), 0, 15)            (s the stored fp16 value)
+ * and reconstructs x^ = (q - z) * s.  Codes are packed two per byte, element 2b in the low nibble
+ * of byte b and element 2b+1 in the high nibble (the order implied by the masks of Eq. 4).  That
+ * is 20 bytes per 32 elements, 3.2x smaller than fp16.  The quantiser is evaluated in IEEE
+ * binary32 with one rounding per operation (true division, no fused multiply-add); a group whose
+ * scale rounds to zero in fp16 stores s = 1, z = -min and all codes 0; z is clamped to +-65504.
+ */
+#ifndef TQ_H_
+#define TQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum tq_result {
+  TQ_OK = 0,
+  TQ_ERR_NULL = 1,      /* a required pointer is NULL */
+  TQ_ERR_SHAPE = 2,     /* unsupported or inconsistent sizes (see each function) */
+  TQ_ERR_ALIGN = 3,     /* a device pointer is not 16-byte aligned */
+  TQ_ERR_WORKSPACE = 4, /* workspace_bytes smaller than tq_dequant_workspace_bytes() */
+  TQ_ERR_CUDA = 5       /* a CUDA call failed; tq_last_cuda_error() has the code */
+} tq_result;
+
+/* bits OR-ed into the device status word */
+#define TQ_STATUS_CACHE_FULL 1 /* quantize_append: seq_lens[b] + T > S_cap; that sequence was skipped */
+#define TQ_STATUS_EMPTY_SEQ 2  /* attention over a sequence with seq_lens[b] <= 0; its output is zero */
+#define TQ_STATUS_BAD_LEN 4    /* seq_lens[b] outside [0, S_cap]; treated as clamped to that range */
+
+#define TQ_GROUP 32         /* quantisation group size g (fixed) */
+#define TQ_SPLIT_QUANTUM 16 /* split boundaries fall on multiples of this many tokens */
+
+/*
+ * The int4 KV cache of ONE layer.  Token-major arrays; sequence b, KV head h, token i is row
+ * (b * H_kv + h) * S_cap + i of each array.  Rows at or beyond seq_lens[b] are unspecified.
+ * Requirements: d in {64, 128, 256}; S_cap a positive multiple of 16; B, H_kv >= 1.
+ */
+typedef struct tq_kv_cache {
+  uint8_t* k_packed;  /* [B][H_kv][S_cap][d/2]  packed codes of K */
+  uint8_t* v_packed;  /* [B][H_kv][S_cap][d/2]  packed codes of V */
+  uint16_t* k_scale;  /* [B][H_kv][S_cap][d/32] fp16 scales of K */
+  uint16_t* k_zero;   /* [B][H_kv][S_cap][d/32] fp16 zero-points of K */
+  uint16_t* v_scale;  /* [B][H_kv][S_cap][d/32] */
+  uint16_t* v_zero;   /* [B][H_kv][S_cap][d/32] */
+  int32_t* seq_lens;  /* [B] number of valid tokens per sequence (device memory, updated by append) */
+  int32_t B, H_kv, S_cap, d;
+} tq_kv_cache;
+
+/*
+ * Quantise T new tokens per sequence and append them in place (Sec. 2.1, Eq. 2-3; "quantizes the
+ * KV cache to int4 on the fly").  The paper's implementation appends by concatenation and names
+ * that as its main end-to-end overhead; here the cache is pre-allocated and rows are written at
+ * seq_lens[b] .. seq_lens[b] + T - 1.
+ *   k_new, v_new : [B][H_kv][T][d] fp16, read only.
+ *   T >= 1.  On return (in stream order) seq_lens[b] has grown by T for every sequence that had
+ *   room; a sequence with seq_lens[b] + T > S_cap is left untouched and TQ_STATUS_CACHE_FULL is
+ *   set.  T = S with seq_lens = 0 is the bulk quantisation of a prefilled cache.
+ * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE (cache requirements, T < 1), TQ_ERR_ALIGN, TQ_ERR_CUDA.
+ */
+int tq_kv_quantize_append(const tq_kv_cache* cache /* host */, const void* k_new, const void* v_new, int32_t T,
+                          int32_t* status, void* stream);
+
+/*
+ * Number of sequence splits C the library would pick for a decode step over sequences of up to
+ * `max_seq_len` tokens (host function, no CUDA call).  Chosen from the SM count so that
+ * B * H_kv * ceil(G / 8) * C thread blocks fill the GPU in whole waves while every split keeps
+ * enough tokens to stream efficiently.  Always in [1, TQ_MAX_SPLITS].
+ */
+#define TQ_MAX_SPLITS 256
+int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len);
+
+/*
+ * Token range of split c of a sequence of `len` tokens cut into C splits (host function): with
+ * nb = ceil(len / 16), split c covers tokens [16 * floor(c * nb / C), min(len, 16 * floor((c + 1) * nb / C))).
+ * This is the partition tq_sdpa_int4_decode uses; exposed so that partials can be checked.
+ */
+void tq_split_range(int32_t len, int32_t C, int32_t c, int32_t* t0 /* host */, int32_t* t1 /* host */);
+
+/*
+ * Phase 1 of the fused int4 attention (Sec. 3.1 Algorithm 1 run per split, Sec. 3.2): for every
+ * sequence b, query head h and split c, attend over the split's tokens reading packed codes,
+ * scales and zeros straight from the cache, dequantising in registers, and write the partial
+ * triple of Sec. 3.2:
+ *   o_part [B][H_q][C][d] fp32   partial output, already divided by l_part (as Eq. 5 expects)
+ *   m_part [B][H_q][C]    fp32   maximum of attn_scale * q.k^ over the split (natural-log units)
+ *   l_part [B][H_q][C]    fp32   sum over the split of exp(score - m_part)
+ * An empty split writes o = 0, m = -inf, l = 0.
+ *   q          : [B][H_q][d] fp16.  Query head h reads KV head h / (H_q / H_kv) (Sec. 3.1, GQA).
+ *   attn_scale : the factor alpha in alpha * q.k (1/sqrt(d) for Llama, 1.0 for Gemma-style models).
+ *   num_splits : C >= 1, or 0 for tq_auto_splits(B, H_kv, H_q, d, S_cap).
+ * All seq_lens[b] cached tokens are attended (no mask).  Requirements: H_q a multiple of H_kv,
+ * H_q / H_kv <= 64, C <= TQ_MAX_SPLITS.
+ * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_CUDA.  Status: TQ_STATUS_EMPTY_SEQ, TQ_STATUS_BAD_LEN.
+ */
+int tq_sdpa_int4_decode(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
+                        int32_t num_splits, float* o_part, float* m_part, float* l_part, int32_t* status,
+                        void* stream);
+
+/*
+ * Phase 2, the reduction of Eq. 5:
+ *   out[b][h][:] = sum_c w_c * o_part[b][h][c][:] / sum_c w_c,   w_c = l_c * exp(m_c - max_c m_c),
+ * skipping splits with l_c = 0; if all are empty the output row is zero.
+ *   out : [B][H_q][d], fp16 (out_is_fp32 = 0) or fp32 (out_is_fp32 = 1).
+ * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE (B, H_q, num_splits < 1, d not a multiple of 32 or > 256), TQ_ERR_ALIGN,
+ * TQ_ERR_CUDA.
+ */
+int tq_sdpa_int4_combine(const float* o_part, const float* m_part, const float* l_part, int32_t B, int32_t H_q,
+                         int32_t d, int32_t num_splits, void* out, int32_t out_is_fp32, void* stream);
+
+/* Bytes needed for o_part + m_part + l_part when laid out back to back (host function). */
+size_t tq_partials_bytes(int32_t B, int32_t H_q, int32_t d, int32_t num_splits);
+
+/*
+ * Comparison path: the "dequantize-then-attend" baseline the paper measures against (Sec. 3.1 first
+ * paragraph, Table 2).  Dequantises all valid rows of K and V into a materialised
+ * [B][H_kv][S_cap][d] matrix in `workspace` (fp32 as in the paper when ws_is_fp32 = 1, fp16
+ * otherwise), then runs split attention and the Eq. 5 reduction on the materialised matrices.
+ * Same result as decode + combine up to rounding.
+ *   workspace_bytes >= tq_dequant_workspace_bytes(...), 16-byte aligned, contents destroyed.
+ */
+int tq_sdpa_dequant_then_attend(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
+                                void* workspace, size_t workspace_bytes, int32_t ws_is_fp32, void* out,
+                                int32_t out_is_fp32, int32_t* status, void* stream);
+
+size_t tq_dequant_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t S_cap, int32_t d,
+                                  int32_t ws_is_fp32);
+
+/* Bytes of one layer's cache arrays (packed + scales + zeros, K and V), i.e. Eq. 1 with the int4 format. */
+size_t tq_cache_bytes(int32_t B, int32_t H_kv, int32_t S_cap, int32_t d);
+
+const char* tq_result_string(int result);
+int tq_last_cuda_error(void); /* cudaError_t of the most recent failing CUDA call of this thread, 0 if none */
+const char* tq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TQ_H_ */

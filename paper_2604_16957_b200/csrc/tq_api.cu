@@ -1,0 +1,191 @@
+// extern "C" entry points of libtq: argument validation and dispatch.  See include/tq.h.
+#include <cstdlib>
+#include <cstring>
+
+#include "tq_internal.cuh"
+
+namespace tq {
+
+static thread_local int g_last_cuda_error = 0;
+
+int device_sm_count() {
+  static const int sms = [] {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        n <= 0) {
+      (void)cudaGetLastError();
+      n = 148;  // B200
+    }
+    return n;
+  }();
+  return sms;
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_cache(const tq_kv_cache* c) {
+  if (!c) return TQ_ERR_NULL;
+  if (!c->k_packed || !c->v_packed || !c->k_scale || !c->k_zero || !c->v_scale || !c->v_zero || !c->seq_lens)
+    return TQ_ERR_NULL;
+  if (!(c->d == 64 || c->d == 128 || c->d == 256)) return TQ_ERR_SHAPE;
+  if (c->B < 1 || c->B > 65535 || c->H_kv < 1 || c->H_kv > 4096 || c->S_cap < 16 || (c->S_cap % 16) != 0)
+    return TQ_ERR_SHAPE;
+  if (!aligned16(c->k_packed) || !aligned16(c->v_packed) || !aligned16(c->k_scale) || !aligned16(c->k_zero) ||
+      !aligned16(c->v_scale) || !aligned16(c->v_zero) || (reinterpret_cast<uintptr_t>(c->seq_lens) & 3u))
+    return TQ_ERR_ALIGN;
+  return TQ_OK;
+}
+
+int check_heads(const tq_kv_cache* c, int H_q) {
+  if (H_q < 1 || (H_q % c->H_kv) != 0 || H_q / c->H_kv > 64) return TQ_ERR_SHAPE;
+  return TQ_OK;
+}
+
+int finish(cudaError_t e) {
+  if (e == cudaSuccess) return TQ_OK;
+  g_last_cuda_error = static_cast<int>(e);
+  return TQ_ERR_CUDA;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+bool use_simple_decode() {
+  const char* e = std::getenv("TQ_DECODE_IMPL");
+  return e && std::strcmp(e, "simple") == 0;
+}
+
+}  // namespace
+}  // namespace tq
+
+using namespace tq;
+
+extern "C" {
+
+int tq_kv_quantize_append(const tq_kv_cache* cache, const void* k_new, const void* v_new, int32_t T, int32_t* status,
+                          void* stream) {
+  if (int r = check_cache(cache)) return r;
+  if (!k_new || !v_new) return TQ_ERR_NULL;
+  if (T < 1 || T > cache->S_cap) return TQ_ERR_SHAPE;
+  if (!aligned16(k_new) || !aligned16(v_new) || (reinterpret_cast<uintptr_t>(status) & 3u)) return TQ_ERR_ALIGN;
+  return finish(launch_quantize_append(*cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new), T,
+                                       status, static_cast<cudaStream_t>(stream)));
+}
+
+int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len) {
+  (void)d;
+  if (B < 1 || H_kv < 1 || H_q < H_kv || max_seq_len < 1) return 1;
+  const long long G = H_q / H_kv;
+  const long long base = static_cast<long long>(B) * H_kv * ((G + 7) / 8);
+  const long long slots = 2LL * device_sm_count();  // two resident thread blocks per SM
+  long long C = base < slots ? slots / base : (4 * slots + base - 1) / base;
+  const long long by_len = max_seq_len / 512;  // keep at least 512 tokens per split
+  if (C > by_len) C = by_len;
+  if (C > TQ_MAX_SPLITS) C = TQ_MAX_SPLITS;
+  if (C < 1) C = 1;
+  return static_cast<int32_t>(C);
+}
+
+void tq_split_range(int32_t len, int32_t C, int32_t c, int32_t* t0, int32_t* t1) {
+  int a = 0, b = 0;
+  if (C >= 1 && c >= 0 && c < C) split_range(len, C, c, a, b);
+  if (t0) *t0 = a;
+  if (t1) *t1 = b;
+}
+
+int tq_sdpa_int4_decode(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale, int32_t num_splits,
+                        float* o_part, float* m_part, float* l_part, int32_t* status, void* stream) {
+  if (int r = check_cache(cache)) return r;
+  if (!q || !o_part || !m_part || !l_part) return TQ_ERR_NULL;
+  if (int r = check_heads(cache, H_q)) return r;
+  if (num_splits < 0 || num_splits > TQ_MAX_SPLITS) return TQ_ERR_SHAPE;
+  if (!aligned16(q) || !aligned16(o_part) || (reinterpret_cast<uintptr_t>(m_part) & 3u) ||
+      (reinterpret_cast<uintptr_t>(l_part) & 3u) || (reinterpret_cast<uintptr_t>(status) & 3u))
+    return TQ_ERR_ALIGN;
+  const int C = num_splits ? num_splits : tq_auto_splits(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
+  auto st = static_cast<cudaStream_t>(stream);
+  auto qh = static_cast<const __half*>(q);
+  if (use_simple_decode())
+    return finish(launch_decode_simple(*cache, qh, H_q, attn_scale, C, o_part, m_part, l_part, status, st));
+  return finish(launch_decode_mma(*cache, qh, H_q, attn_scale, C, o_part, m_part, l_part, status, st));
+}
+
+int tq_sdpa_int4_combine(const float* o_part, const float* m_part, const float* l_part, int32_t B, int32_t H_q,
+                         int32_t d, int32_t num_splits, void* out, int32_t out_is_fp32, void* stream) {
+  if (!o_part || !m_part || !l_part || !out) return TQ_ERR_NULL;
+  if (B < 1 || H_q < 1 || num_splits < 1 || num_splits > TQ_MAX_SPLITS || d < 32 || d > 256 || (d % 32) != 0 ||
+      static_cast<long long>(B) * H_q > 0x7fffffffLL)
+    return TQ_ERR_SHAPE;
+  if (!aligned16(o_part) || !aligned16(out) || (reinterpret_cast<uintptr_t>(m_part) & 3u) ||
+      (reinterpret_cast<uintptr_t>(l_part) & 3u))
+    return TQ_ERR_ALIGN;
+  return finish(launch_combine(o_part, m_part, l_part, B, H_q, d, num_splits, out, out_is_fp32 != 0,
+                               static_cast<cudaStream_t>(stream)));
+}
+
+size_t tq_partials_bytes(int32_t B, int32_t H_q, int32_t d, int32_t num_splits) {
+  if (B < 1 || H_q < 1 || d < 1 || num_splits < 1) return 0;
+  const size_t n = static_cast<size_t>(B) * H_q * num_splits;
+  return align256(n * d * sizeof(float)) + 2 * align256(n * sizeof(float));
+}
+
+size_t tq_dequant_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t S_cap, int32_t d, int32_t ws_is_fp32) {
+  if (B < 1 || H_kv < 1 || H_q < 1 || S_cap < 1 || d < 1) return 0;
+  const size_t mat = align256(static_cast<size_t>(B) * H_kv * S_cap * d * (ws_is_fp32 ? 4 : 2));
+  const int C = tq_auto_splits(B, H_kv, H_q, d, S_cap);
+  return 2 * mat + tq_partials_bytes(B, H_q, d, C);
+}
+
+int tq_sdpa_dequant_then_attend(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale, void* workspace,
+                                size_t workspace_bytes, int32_t ws_is_fp32, void* out, int32_t out_is_fp32,
+                                int32_t* status, void* stream) {
+  if (int r = check_cache(cache)) return r;
+  if (!q || !workspace || !out) return TQ_ERR_NULL;
+  if (int r = check_heads(cache, H_q)) return r;
+  if (!aligned16(q) || !aligned16(workspace) || !aligned16(out) || (reinterpret_cast<uintptr_t>(status) & 3u))
+    return TQ_ERR_ALIGN;
+  if (workspace_bytes < tq_dequant_workspace_bytes(cache->B, cache->H_kv, H_q, cache->S_cap, cache->d, ws_is_fp32))
+    return TQ_ERR_WORKSPACE;
+  const bool f32 = ws_is_fp32 != 0;
+  const int d = cache->d;
+  const int C = tq_auto_splits(cache->B, cache->H_kv, H_q, d, cache->S_cap);
+  const size_t mat = align256(static_cast<size_t>(cache->B) * cache->H_kv * cache->S_cap * d * (f32 ? 4 : 2));
+  const size_t n = static_cast<size_t>(cache->B) * H_q * C;
+  char* ws = static_cast<char*>(workspace);
+  void* k_mat = ws;
+  void* v_mat = ws + mat;
+  float* o_part = reinterpret_cast<float*>(ws + 2 * mat);
+  float* m_part = reinterpret_cast<float*>(ws + 2 * mat + align256(n * d * sizeof(float)));
+  float* l_part = reinterpret_cast<float*>(reinterpret_cast<char*>(m_part) + align256(n * sizeof(float)));
+  auto st = static_cast<cudaStream_t>(stream);
+  if (int r = finish(launch_dequant(*cache, k_mat, v_mat, f32, st))) return r;
+  if (int r = finish(launch_attend_materialized(*cache, k_mat, v_mat, f32, static_cast<const __half*>(q), H_q,
+                                                attn_scale, C, o_part, m_part, l_part, status, st)))
+    return r;
+  return finish(launch_combine(o_part, m_part, l_part, cache->B, H_q, d, C, out, out_is_fp32 != 0, st));
+}
+
+size_t tq_cache_bytes(int32_t B, int32_t H_kv, int32_t S_cap, int32_t d) {
+  if (B < 1 || H_kv < 1 || S_cap < 1 || d < 1) return 0;
+  const size_t per_vec = static_cast<size_t>(d) / 2 + 2 * (static_cast<size_t>(d) / TQ_GROUP) * 2;
+  return 2 * static_cast<size_t>(B) * H_kv * S_cap * per_vec;
+}
+
+const char* tq_result_string(int r) {
+  switch (r) {
+    case TQ_OK: return "ok";
+    case TQ_ERR_NULL: return "null pointer";
+    case TQ_ERR_SHAPE: return "unsupported or inconsistent shape";
+    case TQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case TQ_ERR_WORKSPACE: return "workspace too small";
+    case TQ_ERR_CUDA: return "CUDA error";
+    default: return "unknown";
+  }
+}
+
+int tq_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* tq_version(void) { return "libtq 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,235 @@
+// Scalar split attention kernels and the dequantise-to-matrix kernel.
+//
+//  * attend_simple_kernel<D, Src>: Algorithm 1 run per split on CUDA cores, one warp per token
+//    stream, one lane per D/32 consecutive channels, warp-shuffle dot products, fp32 online
+//    softmax.  Src selects where a K/V row comes from:
+//      SrcInt4  -- the packed cache, dequantised in registers (a plain reference variant of the
+//                  fused kernel, selected with TQ_DECODE_IMPL=simple; the tensor-core kernel in
+//                  tq_decode_mma.cu is the production path)
+//      SrcF32 / SrcF16 -- a materialised [B][H_kv][S_cap][D] matrix: the attention half of the
+//                  dequantize-then-attend comparison path (Sec. 3.1 first paragraph, Table 2).
+//  * dequant_kernel: the other half of that comparison path, x^ = (q - z) * s for every valid
+//    row (Eq. 3), written to the materialised matrix.
+#include "tq_internal.cuh"
+
+namespace tq {
+namespace {
+
+constexpr int kWarps = 4;
+constexpr int kHeadTile = 8;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+template <int D>
+struct SrcInt4 {
+  static constexpr int EPL = D / 32;  // elements per lane
+  const uint8_t *kp, *vp;
+  const __half *ks, *kz, *vs, *vz;
+  __device__ void load(bool is_v, long long row, int lane, float (&x)[EPL]) const {
+    const uint8_t* p = (is_v ? vp : kp) + row * (D / 2) + lane * (EPL / 2);
+    const int g = (lane * EPL) / 32;
+    const float s = __half2float((is_v ? vs : ks)[row * (D / 32) + g]);
+    const float z = __half2float((is_v ? vz : kz)[row * (D / 32) + g]);
+#pragma unroll
+    for (int i = 0; i < EPL / 2; ++i) {
+      const uint32_t byte = p[i];
+      x[2 * i] = (static_cast<float>(byte & 0xF) - z) * s;
+      x[2 * i + 1] = (static_cast<float>(byte >> 4) - z) * s;
+    }
+  }
+};
+
+template <int D, typename T>
+struct SrcMat {
+  static constexpr int EPL = D / 32;
+  const T *k, *v;
+  __device__ void load(bool is_v, long long row, int lane, float (&x)[EPL]) const {
+    const T* p = (is_v ? v : k) + row * D + lane * EPL;
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) {
+      if constexpr (sizeof(T) == 4) x[i] = p[i];
+      else x[i] = __half2float(p[i]);
+    }
+  }
+};
+
+// grid: (C, H_kv * head_tiles, B); block: kWarps warps.
+template <int D, typename Src>
+__global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, const int32_t* seq_lens, int H_kv,
+                                                                    int S_cap, const __half* q, int H_q,
+                                                                    float attn_scale, int C, float* o_part,
+                                                                    float* m_part, float* l_part, int32_t* status) {
+  constexpr int EPL = D / 32;
+  const int G = H_q / H_kv;
+  const int tiles = (G + kHeadTile - 1) / kHeadTile;
+  const int c = blockIdx.x, kvh = blockIdx.y / tiles, tile = blockIdx.y % tiles, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int len = checked_len(seq_lens, b, S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
+  int t0, t1;
+  split_range(len, C, c, t0, t1);
+  const int h0 = kvh * G + tile * kHeadTile;
+  const int nh = min(kHeadTile, G - tile * kHeadTile);
+
+  float qr[kHeadTile][EPL], o[kHeadTile][EPL], m[kHeadTile], l[kHeadTile];
+#pragma unroll
+  for (int h = 0; h < kHeadTile; ++h) {
+    m[h] = -INFINITY;
+    l[h] = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      o[h][e] = 0.f;
+      qr[h][e] = h < nh ? __half2float(q[(static_cast<long long>(b) * H_q + h0 + h) * D + lane * EPL + e]) : 0.f;
+    }
+  }
+  const long long row0 = (static_cast<long long>(b) * H_kv + kvh) * S_cap;
+  const float sc = attn_scale * kLog2e;
+  for (int i = t0 + warp; i < t1; i += kWarps) {
+    float kx[EPL], vx[EPL];
+    src.load(false, row0 + i, lane, kx);
+    src.load(true, row0 + i, lane, vx);
+#pragma unroll
+    for (int h = 0; h < kHeadTile; ++h) {
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) dot = fmaf(qr[h][e], kx[e], dot);
+#pragma unroll
+      for (int off = 16; off; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+      const float a = dot * sc;  // log2 units
+      const float mn = fmaxf(m[h], a);
+      const float corr = exp2f(m[h] - mn);  // exp2(-inf) = 0 on the first token
+      const float p = exp2f(a - mn);
+      l[h] = l[h] * corr + p;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) o[h][e] = o[h][e] * corr + p * vx[e];
+      m[h] = mn;
+    }
+  }
+  // merge the warps' (m, l, o) through shared memory, then write the normalised partial
+  __shared__ float sm_m[kWarps][kHeadTile], sm_l[kWarps][kHeadTile];
+  __shared__ float sm_o[kWarps][kHeadTile][D];
+#pragma unroll
+  for (int h = 0; h < kHeadTile; ++h) {
+    if (lane == 0) {
+      sm_m[warp][h] = m[h];
+      sm_l[warp][h] = l[h];
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) sm_o[warp][h][lane * EPL + e] = o[h][e];
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < nh * D; idx += blockDim.x) {
+    const int h = idx / D, x = idx % D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_m[w][h]);
+    float num = 0.f, den = 0.f;
+    if (M > -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const float f = exp2f(sm_m[w][h] - M);
+        num += f * sm_o[w][h][x];
+        den += f * sm_l[w][h];
+      }
+    }
+    const long long pidx = (static_cast<long long>(b) * H_q + h0 + h) * C + c;
+    o_part[pidx * D + x] = den > 0.f ? num / den : 0.f;
+    if (x == 0) {
+      m_part[pidx] = M * kLn2;  // back to natural-log units of attn_scale * q.k
+      l_part[pidx] = den;
+    }
+  }
+}
+
+template <int D, typename Src>
+cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C,
+                          float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+  const int G = H_q / c.H_kv;
+  const int tiles = (G + kHeadTile - 1) / kHeadTile;
+  dim3 grid(C, c.H_kv * tiles, c.B);
+  attend_simple_kernel<D, Src><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, attn_scale, C,
+                                                             o_part, m_part, l_part, status);
+  return cudaGetLastError();
+}
+
+// x^ = (q - z) * s for every valid row; one thread per 8 consecutive elements.
+template <typename T>
+__global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T* v_mat) {
+  const int d = c.d, cpr = d >> 3;
+  const int b = blockIdx.y;
+  int len = c.seq_lens[b];
+  len = len < 0 ? 0 : (len > c.S_cap ? c.S_cap : len);
+  const bool is_v = blockIdx.z != 0;
+  const long long per_seq = static_cast<long long>(c.H_kv) * len * cpr;
+  const long long local = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (local >= per_seq) return;
+  const long long r = local / cpr;  // h * len + t
+  const int cc = static_cast<int>(local - r * cpr);
+  const long long h = r / len;
+  const int t = static_cast<int>(r - h * len);
+  const long long row = (static_cast<long long>(b) * c.H_kv + h) * c.S_cap + t;
+  const uint32_t w = reinterpret_cast<const uint32_t*>((is_v ? c.v_packed : c.k_packed) + row * (d >> 1))[cc];
+  const float s = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_scale : c.k_scale)[row * (d >> 5) + (cc >> 2)]);
+  const float z = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_zero : c.k_zero)[row * (d >> 5) + (cc >> 2)]);
+  float x[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(__fsub_rn(static_cast<float>((w >> (4 * i)) & 0xF), z), s);
+  T* dst = (is_v ? v_mat : k_mat) + row * d + cc * 8;
+  if constexpr (sizeof(T) == 4) {
+    reinterpret_cast<float4*>(dst)[0] = make_float4(x[0], x[1], x[2], x[3]);
+    reinterpret_cast<float4*>(dst)[1] = make_float4(x[4], x[5], x[6], x[7]);
+  } else {
+    __half2 h2[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h2[i] = __floats2half2_rn(x[2 * i], x[2 * i + 1]);
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<uint4*>(h2);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C,
+                                 float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+  auto run = [&](auto dtag) {
+    constexpr int D = decltype(dtag)::value;
+    SrcInt4<D> src{c.k_packed, c.v_packed, reinterpret_cast<const __half*>(c.k_scale),
+                   reinterpret_cast<const __half*>(c.k_zero), reinterpret_cast<const __half*>(c.v_scale),
+                   reinterpret_cast<const __half*>(c.v_zero)};
+    return launch_simple<D>(src, c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
+  };
+  switch (c.d) {
+    case 64: return run(std::integral_constant<int, 64>{});
+    case 128: return run(std::integral_constant<int, 128>{});
+    default: return run(std::integral_constant<int, 256>{});
+  }
+}
+
+cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, const void* v_mat, bool fp32,
+                                       const __half* q, int H_q, float attn_scale, int C, float* o_part, float* m_part,
+                                       float* l_part, int32_t* status, cudaStream_t st) {
+  auto run = [&](auto dtag, auto ttag) {
+    constexpr int D = decltype(dtag)::value;
+    using T = decltype(ttag);
+    SrcMat<D, T> src{static_cast<const T*>(k_mat), static_cast<const T*>(v_mat)};
+    return launch_simple<D>(src, c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
+  };
+  auto by_d = [&](auto ttag) {
+    switch (c.d) {
+      case 64: return run(std::integral_constant<int, 64>{}, ttag);
+      case 128: return run(std::integral_constant<int, 128>{}, ttag);
+      default: return run(std::integral_constant<int, 256>{}, ttag);
+    }
+  };
+  return fp32 ? by_d(float{}) : by_d(__half{});
+}
+
+cudaError_t launch_dequant(const tq_kv_cache& c, void* k_mat, void* v_mat, bool fp32, cudaStream_t st) {
+  const long long per_seq = static_cast<long long>(c.H_kv) * c.S_cap * (c.d >> 3);
+  dim3 grid(static_cast<unsigned>((per_seq + 255) / 256), c.B, 2);
+  if (fp32)
+    dequant_kernel<float><<<grid, 256, 0, st>>>(c, static_cast<float*>(k_mat), static_cast<float*>(v_mat));
+  else
+    dequant_kernel<__half><<<grid, 256, 0, st>>>(c, static_cast<__half*>(k_mat), static_cast<__half*>(v_mat));
+  return cudaGetLastError();
+}
+
+}  // namespace tq

@@ -1,0 +1,51 @@
+// Internal declarations shared by the translation units of libtq (not part of the ABI).
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tq.h"
+
+namespace tq {
+
+constexpr int kGroup = TQ_GROUP;
+constexpr int kQuantum = TQ_SPLIT_QUANTUM;
+
+// Split partition shared by host and device: split c of C over a sequence of len tokens.
+__host__ __device__ inline void split_range(int len, int C, int c, int& t0, int& t1) {
+  if (len < 0) len = 0;
+  long long nb = (len + kQuantum - 1) / kQuantum;
+  long long b0 = (nb * c) / C, b1 = (nb * (c + 1)) / C;
+  t0 = (int)(b0 * kQuantum);
+  long long e = b1 * kQuantum;
+  t1 = (int)(e < len ? e : len);
+  if (t1 < t0) t1 = t0;
+}
+
+// Clamp a device-side sequence length into [0, S_cap], flagging bad or empty values.
+__device__ inline int checked_len(const int32_t* seq_lens, int b, int S_cap, int32_t* status) {
+  int len = seq_lens[b];
+  if (len < 0 || len > S_cap) {
+    if (status && threadIdx.x == 0) atomicOr(status, TQ_STATUS_BAD_LEN);
+    len = len < 0 ? 0 : S_cap;
+  }
+  if (len == 0 && status && threadIdx.x == 0) atomicOr(status, TQ_STATUS_EMPTY_SEQ);
+  return len;
+}
+
+// host-side launchers (each returns cudaGetLastError() after its launches)
+cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, const __half* v_new, int T,
+                                   int32_t* status, cudaStream_t st);
+cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C, float* o_part,
+                              float* m_part, float* l_part, int32_t* status, cudaStream_t st);
+cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C,
+                                 float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
+cudaError_t launch_combine(const float* o_part, const float* m_part, const float* l_part, int B, int H_q, int d, int C,
+                           void* out, bool out_fp32, cudaStream_t st);
+cudaError_t launch_dequant(const tq_kv_cache& c, void* k_mat, void* v_mat, bool fp32, cudaStream_t st);
+cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, const void* v_mat, bool fp32,
+                                       const __half* q, int H_q, float attn_scale, int C, float* o_part, float* m_part,
+                                       float* l_part, int32_t* status, cudaStream_t st);
+int device_sm_count();
+
+}  // namespace tq

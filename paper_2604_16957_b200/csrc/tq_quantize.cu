@@ -1,0 +1,172 @@
+// int4 quantise-and-append of new K/V tokens (Sec. 2.1, Eq. 2-3), written in place into a
+// pre-allocated cache.
+//
+// Mapping: one thread owns 8 consecutive elements (one 16-byte load, one packed 32-bit store);
+// the 4 threads of a lane quad own one quantisation group of 32, so min/max need two shuffles.
+// A warp covers 256 consecutive elements: its packed stores are 128 contiguous bytes and its
+// scale / zero stores 16 contiguous bytes each.
+//
+// All arithmetic is IEEE binary32 with explicit round-to-nearest intrinsics so that the result
+// is bit-identical on any machine that follows the same operation order:
+//   s = fp16((max - min) / 15);  z = fp16((0 - min) / s);  q = clamp(rint(x / s + z), 0, 15).
+#include "tq_internal.cuh"
+
+namespace tq {
+namespace {
+
+struct QuantDst {
+  uint8_t* packed;
+  __half* scale;
+  __half* zero;
+};
+
+// Quantise the 8 elements held by this thread (quad = one group).  All 32 lanes must call.
+__device__ __forceinline__ void quantize_chunk(const uint4 raw, bool active, uint32_t& word, __half& s_out,
+                                               __half& z_out) {
+  const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+  float x[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 f = __half22float2(h2[i]);
+    x[2 * i] = f.x;
+    x[2 * i + 1] = f.y;
+  }
+  float mn = x[0], mx = x[0];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) {
+    mn = fminf(mn, x[i]);
+    mx = fmaxf(mx, x[i]);
+  }
+#pragma unroll
+  for (int off = 1; off <= 2; off <<= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  }
+  (void)active;
+  const float range = __fsub_rn(mx, mn);
+  const float s32 = __fdiv_rn(range, 15.0f);
+  __half s16 = __float2half_rn(s32);
+  word = 0u;
+  if ((__half_as_ushort(s16) & 0x7FFFu) == 0) {  // scale rounds to zero: constant (or nearly constant) group
+    s_out = __ushort_as_half(0x3C00u);            // 1.0
+    z_out = __float2half_rn(__fsub_rn(0.0f, mn));
+    return;
+  }
+  const float sf = __half2float(s16);
+  float z32 = __fdiv_rn(__fsub_rn(0.0f, mn), sf);
+  z32 = fminf(fmaxf(z32, -65504.0f), 65504.0f);
+  const __half z16 = __float2half_rn(z32);
+  const float zf = __half2float(z16);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float t = __fdiv_rn(x[i], sf);
+    const float u = __fadd_rn(t, zf);
+    float r = rintf(u);
+    if (!(r >= 0.0f)) r = 0.0f;
+    if (r > 15.0f) r = 15.0f;
+    word |= static_cast<uint32_t>(static_cast<int>(r)) << (4 * i);
+  }
+  s_out = s16;
+  z_out = z16;
+}
+
+// chunk index -> (b, h, t, c) of a [B][H_kv][T][d] tensor and the destination row in the cache
+__device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half* src, const QuantDst& dst, int T,
+                                              long long chunk, bool in_range, int b, int len) {
+  const int d = c.d;
+  const int cpr = d >> 3;  // chunks per row
+  uint4 raw = make_uint4(0, 0, 0, 0);
+  long long row_in = 0;
+  int cc = 0;
+  if (in_range) {
+    row_in = chunk / cpr;  // (b * H_kv + h) * T + t
+    cc = static_cast<int>(chunk - row_in * cpr);
+    raw = *reinterpret_cast<const uint4*>(src + row_in * d + cc * 8);
+  }
+  uint32_t word;
+  __half s, z;
+  quantize_chunk(raw, in_range, word, s, z);
+  if (in_range) {
+    const long long bh = row_in / T;
+    const int t = static_cast<int>(row_in - bh * T);
+    const long long row_out = bh * c.S_cap + len + t;
+    (void)b;
+    reinterpret_cast<uint32_t*>(dst.packed + row_out * (d >> 1))[cc] = word;
+    if ((cc & 3) == 0) {
+      dst.scale[row_out * (d >> 5) + (cc >> 2)] = s;
+      dst.zero[row_out * (d >> 5) + (cc >> 2)] = z;
+    }
+  }
+}
+
+// Bulk variant: grid.x over chunks of one sequence, grid.y = sequence, grid.z = {K, V}.
+// seq_lens is read only here and bumped by bump_lens_kernel afterwards, so that no block can
+// observe a length that another block of the same launch has already advanced.
+__global__ void __launch_bounds__(256) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
+                                                            int T) {
+  const int b = blockIdx.y;
+  const int len = c.seq_lens[b];
+  if (len < 0 || len + T > c.S_cap) return;  // flagged by bump_lens_kernel
+  const bool is_v = blockIdx.z != 0;
+  const __half* src = is_v ? v_new : k_new;
+  QuantDst dst = is_v ? QuantDst{c.v_packed, reinterpret_cast<__half*>(c.v_scale), reinterpret_cast<__half*>(c.v_zero)}
+                      : QuantDst{c.k_packed, reinterpret_cast<__half*>(c.k_scale), reinterpret_cast<__half*>(c.k_zero)};
+  const long long per_seq = static_cast<long long>(c.H_kv) * T * (c.d >> 3);
+  const long long local = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const bool in_range = local < per_seq;
+  process_chunk(c, src, dst, T, static_cast<long long>(b) * per_seq + local, in_range, b, len);
+}
+
+__global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= c.B) return;
+  const int len = c.seq_lens[b];
+  if (len < 0 || len + T > c.S_cap) {
+    if (status) atomicOr(status, TQ_STATUS_CACHE_FULL);
+    return;
+  }
+  c.seq_lens[b] = len + T;
+}
+
+// Decode-step variant (small T): one block per sequence quantises K and V of all its KV heads,
+// then advances the length itself -- a single launch, and no block reads another's length.
+__global__ void __launch_bounds__(256) quantize_step_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
+                                                            int T, int32_t* status) {
+  const int b = blockIdx.x;
+  const int len = c.seq_lens[b];
+  if (len < 0 || len + T > c.S_cap) {
+    if (status && threadIdx.x == 0) atomicOr(status, TQ_STATUS_CACHE_FULL);
+    return;
+  }
+  const long long per_seq = static_cast<long long>(c.H_kv) * T * (c.d >> 3);
+  const QuantDst dk{c.k_packed, reinterpret_cast<__half*>(c.k_scale), reinterpret_cast<__half*>(c.k_zero)};
+  const QuantDst dv{c.v_packed, reinterpret_cast<__half*>(c.v_scale), reinterpret_cast<__half*>(c.v_zero)};
+  for (long long base = 0; base < 2 * per_seq; base += blockDim.x) {  // per_seq is a multiple of 4: quads stay whole
+    const long long i = base + threadIdx.x;
+    const bool is_v = i >= per_seq;
+    const long long local = is_v ? i - per_seq : i;
+    const bool in_range = i < 2 * per_seq;
+    process_chunk(c, is_v ? v_new : k_new, is_v ? dv : dk, T, static_cast<long long>(b) * per_seq + local, in_range, b,
+                  len);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) c.seq_lens[b] = len + T;
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, const __half* v_new, int T,
+                                   int32_t* status, cudaStream_t st) {
+  const long long per_seq = static_cast<long long>(c.H_kv) * T * (c.d >> 3);
+  if (2 * per_seq <= 8192) {
+    quantize_step_kernel<<<c.B, 256, 0, st>>>(c, k_new, v_new, T, status);
+  } else {
+    const long long blocks = (per_seq + 255) / 256;
+    dim3 grid(static_cast<unsigned>(blocks), c.B, 2);
+    quantize_bulk_kernel<<<grid, 256, 0, st>>>(c, k_new, v_new, T);
+    bump_lens_kernel<<<(c.B + 127) / 128, 128, 0, st>>>(c, T, status);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace tq

@@ -1,0 +1,178 @@
+"""ctypes binding of libtq.so -- same names as include/tq.h, argument marshalling only.
+
+Tensors are torch CUDA tensors (torch supplies device memory and streams, nothing else); every
+function forwards data pointers and sizes to the C entry point and raises TqError on a non-zero
+result.  There is no CPU fallback: importing this module fails if the library has not been
+built (python -m paper_2604_16957_b200.build), and calls fail without a CUDA device.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtq.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2604_16957_b200.build`")
+
+_lib = C.CDLL(LIB_PATH)
+
+TQ_OK, TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_WORKSPACE, TQ_ERR_CUDA = range(6)
+TQ_STATUS_CACHE_FULL, TQ_STATUS_EMPTY_SEQ, TQ_STATUS_BAD_LEN = 1, 2, 4
+TQ_GROUP, TQ_SPLIT_QUANTUM, TQ_MAX_SPLITS = 32, 16, 256
+
+# every symbol include/tq.h declares
+SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa_int4_decode", "tq_sdpa_int4_combine",
+           "tq_partials_bytes", "tq_sdpa_dequant_then_attend", "tq_dequant_workspace_bytes", "tq_cache_bytes",
+           "tq_result_string", "tq_last_cuda_error", "tq_version")
+
+
+class tq_kv_cache(C.Structure):
+    _fields_ = [("k_packed", C.c_void_p), ("v_packed", C.c_void_p), ("k_scale", C.c_void_p), ("k_zero", C.c_void_p),
+                ("v_scale", C.c_void_p), ("v_zero", C.c_void_p), ("seq_lens", C.c_void_p), ("B", C.c_int32),
+                ("H_kv", C.c_int32), ("S_cap", C.c_int32), ("d", C.c_int32)]
+
+
+_vp, _i32, _f32, _sz = C.c_void_p, C.c_int32, C.c_float, C.c_size_t
+_cache_p = C.POINTER(tq_kv_cache)
+_lib.tq_kv_quantize_append.argtypes = [_cache_p, _vp, _vp, _i32, _vp, _vp]
+_lib.tq_kv_quantize_append.restype = C.c_int
+_lib.tq_auto_splits.argtypes = [_i32] * 5
+_lib.tq_auto_splits.restype = _i32
+_lib.tq_split_range.argtypes = [_i32, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32)]
+_lib.tq_split_range.restype = None
+_lib.tq_sdpa_int4_decode.argtypes = [_cache_p, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp]
+_lib.tq_sdpa_int4_decode.restype = C.c_int
+_lib.tq_sdpa_int4_combine.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32, _vp]
+_lib.tq_sdpa_int4_combine.restype = C.c_int
+_lib.tq_partials_bytes.argtypes = [_i32] * 4
+_lib.tq_partials_bytes.restype = _sz
+_lib.tq_sdpa_dequant_then_attend.argtypes = [_cache_p, _vp, _i32, _f32, _vp, _sz, _i32, _vp, _i32, _vp, _vp]
+_lib.tq_sdpa_dequant_then_attend.restype = C.c_int
+_lib.tq_dequant_workspace_bytes.argtypes = [_i32] * 6
+_lib.tq_dequant_workspace_bytes.restype = _sz
+_lib.tq_cache_bytes.argtypes = [_i32] * 4
+_lib.tq_cache_bytes.restype = _sz
+_lib.tq_result_string.argtypes = [C.c_int]
+_lib.tq_result_string.restype = C.c_char_p
+_lib.tq_last_cuda_error.restype = C.c_int
+_lib.tq_version.restype = C.c_char_p
+
+
+class TqError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        msg = _lib.tq_result_string(code).decode()
+        if code == TQ_ERR_CUDA:
+            msg += f" (cudaError {_lib.tq_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{code}]")
+
+
+def _check(code, where):
+    if code != TQ_OK:
+        raise TqError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+class KVCache:
+    """Device buffers of one layer's int4 KV cache plus the C struct that describes them."""
+
+    def __init__(self, B, H_kv, S_cap, d, device="cuda"):
+        self.B, self.H_kv, self.S_cap, self.d = B, H_kv, S_cap, d
+        g = d // TQ_GROUP
+        u8 = dict(dtype=torch.uint8, device=device)
+        f16 = dict(dtype=torch.float16, device=device)
+        self.k_packed = torch.zeros((B, H_kv, S_cap, d // 2), **u8)
+        self.v_packed = torch.zeros((B, H_kv, S_cap, d // 2), **u8)
+        self.k_scale = torch.zeros((B, H_kv, S_cap, g), **f16)
+        self.k_zero = torch.zeros((B, H_kv, S_cap, g), **f16)
+        self.v_scale = torch.zeros((B, H_kv, S_cap, g), **f16)
+        self.v_zero = torch.zeros((B, H_kv, S_cap, g), **f16)
+        self.seq_lens = torch.zeros((B,), dtype=torch.int32, device=device)
+
+    def arrays(self):
+        return (self.k_packed, self.k_scale, self.k_zero, self.v_packed, self.v_scale, self.v_zero)
+
+    def struct(self):
+        return tq_kv_cache(self.k_packed.data_ptr(), self.v_packed.data_ptr(), self.k_scale.data_ptr(),
+                           self.k_zero.data_ptr(), self.v_scale.data_ptr(), self.v_zero.data_ptr(),
+                           self.seq_lens.data_ptr(), self.B, self.H_kv, self.S_cap, self.d)
+
+
+def _cs(cache):
+    return cache if isinstance(cache, tq_kv_cache) else cache.struct()
+
+
+def tq_kv_quantize_append(cache, k_new, v_new, status=None, stream=None):
+    """k_new, v_new: [B][H_kv][T][d] float16 CUDA tensors (contiguous)."""
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.dtype == torch.float16 == v_new.dtype
+    assert k_new.shape == v_new.shape and k_new.dim() == 4
+    cs = _cs(cache)
+    _check(_lib.tq_kv_quantize_append(C.byref(cs), _ptr(k_new), _ptr(v_new), k_new.shape[2], _ptr(status),
+                                      _stream(stream)), "tq_kv_quantize_append")
+
+
+def tq_auto_splits(B, H_kv, H_q, d, max_seq_len):
+    return int(_lib.tq_auto_splits(B, H_kv, H_q, d, max_seq_len))
+
+
+def tq_split_range(length, C_, c):
+    t0, t1 = _i32(), _i32()
+    _lib.tq_split_range(length, C_, c, C.byref(t0), C.byref(t1))
+    return t0.value, t1.value
+
+
+def tq_partials_bytes(B, H_q, d, num_splits):
+    return int(_lib.tq_partials_bytes(B, H_q, d, num_splits))
+
+
+def tq_dequant_workspace_bytes(B, H_kv, H_q, S_cap, d, ws_is_fp32):
+    return int(_lib.tq_dequant_workspace_bytes(B, H_kv, H_q, S_cap, d, int(ws_is_fp32)))
+
+
+def tq_cache_bytes(B, H_kv, S_cap, d):
+    return int(_lib.tq_cache_bytes(B, H_kv, S_cap, d))
+
+
+def tq_version():
+    return _lib.tq_version().decode()
+
+
+def tq_sdpa_int4_decode(cache, q, attn_scale, num_splits, o_part, m_part, l_part, status=None, stream=None):
+    """q: [B][H_q][d] float16; o_part [B][H_q][C][d], m_part / l_part [B][H_q][C] float32."""
+    assert q.is_contiguous() and q.dtype == torch.float16 and q.dim() == 3
+    cs = _cs(cache)
+    _check(_lib.tq_sdpa_int4_decode(C.byref(cs), _ptr(q), q.shape[1], float(attn_scale), int(num_splits), _ptr(o_part),
+                                    _ptr(m_part), _ptr(l_part), _ptr(status), _stream(stream)), "tq_sdpa_int4_decode")
+
+
+def tq_sdpa_int4_combine(o_part, m_part, l_part, out, stream=None):
+    B, H_q, Cn, d = o_part.shape
+    assert out.shape == (B, H_q, d) and out.dtype in (torch.float16, torch.float32) and out.is_contiguous()
+    _check(_lib.tq_sdpa_int4_combine(_ptr(o_part), _ptr(m_part), _ptr(l_part), B, H_q, d, Cn, _ptr(out),
+                                     int(out.dtype == torch.float32), _stream(stream)), "tq_sdpa_int4_combine")
+
+
+def tq_sdpa_dequant_then_attend(cache, q, attn_scale, workspace, ws_is_fp32, out, status=None, stream=None):
+    assert q.is_contiguous() and q.dtype == torch.float16 and workspace.dtype == torch.uint8
+    cs = _cs(cache)
+    _check(_lib.tq_sdpa_dequant_then_attend(C.byref(cs), _ptr(q), q.shape[1], float(attn_scale), _ptr(workspace),
+                                            workspace.numel(), int(ws_is_fp32), _ptr(out),
+                                            int(out.dtype == torch.float32), _ptr(status), _stream(stream)),
+           "tq_sdpa_dequant_then_attend")
+
+
+def alloc_partials(B, H_q, d, num_splits, device="cuda"):
+    o = torch.empty((B, H_q, num_splits, d), dtype=torch.float32, device=device)
+    m = torch.empty((B, H_q, num_splits), dtype=torch.float32, device=device)
+    l = torch.empty((B, H_q, num_splits), dtype=torch.float32, device=device)
+    return o, m, l

@@ -1,0 +1,73 @@
+"""The C-ABI library loads, exports every symbol the header declares, and rejects bad arguments
+on the host before touching a GPU (CPU only: no kernel is launched here)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_16957_b200 import build
+    return C.CDLL(build.build())
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "tq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(tq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert {"tq_kv_quantize_append", "tq_sdpa_int4_decode", "tq_sdpa_int4_combine",
+            "tq_sdpa_dequant_then_attend"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    from paper_2604_16957_b200 import tq
+    assert sorted(tq.SYMBOLS) == names
+
+
+def test_host_side_helpers(lib):
+    from paper_2604_16957_b200 import tq
+    assert tq.tq_cache_bytes(1, 8, 131072, 128) * 80 == int(12.5 * 2 ** 30)       # Table 4, 128K row
+    assert tq.tq_partials_bytes(1, 64, 128, 37) >= 64 * 37 * 130 * 4
+    # split ranges tile [0, len) in order, on multiples of 16 except the end
+    for length, Cn in ((0, 3), (1, 4), (257, 5), (131072, 37), (4097, 256)):
+        prev = 0
+        for c in range(Cn):
+            t0, t1 = tq.tq_split_range(length, Cn, c)
+            assert t0 == prev and t1 >= t0 and (t0 % 16 == 0)
+            prev = t1
+        assert prev == length
+    c = tq.tq_auto_splits(1, 8, 64, 128, 131072)
+    assert 1 <= c <= 256
+    assert tq.tq_auto_splits(1, 8, 64, 128, 100) == 1
+
+
+def test_argument_validation_without_gpu(lib):
+    from paper_2604_16957_b200 import tq
+    lib.tq_result_string.restype = C.c_char_p
+    assert lib.tq_result_string(0) == b"ok"
+    assert tq._lib.tq_kv_quantize_append(None, None, None, 1, None, None) == tq.TQ_ERR_NULL
+    fake = 0x1000  # never dereferenced: validation fails first
+    cs = tq.tq_kv_cache(fake, fake, fake, fake, fake, fake, fake, 1, 1, 64, 100)   # d = 100
+    assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 1, None, None) == tq.TQ_ERR_SHAPE
+    cs = tq.tq_kv_cache(fake, fake, fake, fake, fake, fake, fake, 1, 1, 60, 128)   # S_cap % 16 != 0
+    assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 8, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
+    cs = tq.tq_kv_cache(fake + 8, fake, fake, fake, fake, fake, fake, 1, 1, 64, 128)
+    assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 1, None, None) == tq.TQ_ERR_ALIGN
+    cs = tq.tq_kv_cache(fake, fake, fake, fake, fake, fake, fake, 1, 2, 64, 128)
+    assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 7, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 8, 1.0, 300, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), None, 8, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_NULL
+    assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 0, None, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_int4_combine(fake, fake, fake, 1, 8, 100, 4, fake, 1, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_int4_combine(fake, fake, fake, 1, 8, 128, 0, fake, 1, None) == tq.TQ_ERR_SHAPE
+    need = tq.tq_dequant_workspace_bytes(1, 2, 8, 64, 128, 1)
+    assert need >= 2 * 2 * 64 * 128 * 4
+    assert tq._lib.tq_sdpa_dequant_then_attend(C.byref(cs), fake, 8, 1.0, fake, need - 1, 1, fake, 1, None,
+                                               None) == tq.TQ_ERR_WORKSPACE
