@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the int4 compressed-domain decode-attention hot path on B200.
+
+Workload (N = 1): the Llama-3.1-70B-shaped long-context configuration -- 64 query heads, 8 KV
+heads, d = 128, 131072 cached tokens, all 80 layers' int4 KV caches resident (13.4 GB).  One
+step is one decode step run layer by layer: for each of the 80 layers, quantize-append of the
+new token's K/V, fused int4 attention (split-K partials) and the split reduction.  The metric
+is microseconds per layer-step; the roofline object reports the fused kernel's algorithmic
+HBM bytes per second against the measured copy bandwidth of this GPU pool.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--context S] [--layers L]
+
+Prints ONE JSON line on stdout (rank 0).  All inputs are seeded and synthetic.
+"""
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+H_Q, H_KV, D, LAYERS, CONTEXT = 64, 8, 128, 80, 131072
+ALPHA = D ** -0.5
+BYTES_PER_TOKEN_HEAD = 2 * (D // 2 + 2 * (D // 32) * 2)  # K + V: codes + fp16 scale + fp16 zero = 160 B
+HBM_NOMINAL_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+PAPER_CONTEXT = {"hardware": "Apple M1 Max 64 GB (Metal)", "fused_ms_at_128K": 9.9,
+                 "dequant_then_attend_ms_at_128K": 480.6, "speedup_at_128K": 48,
+                 "note": "paper Table 2; another machine and API, context only"}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--context", type=int, default=CONTEXT)
+    ap.add_argument("--layers", type=int, default=LAYERS)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-compare", action="store_true", help="skip the dequantize-then-attend timing")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, device copy)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------ clocks (read-only NVML sampling)
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+               0x80: "hw_power_brake", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting"}
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ CPU oracle leg
+def oracle_sample_us_per_layer(context, repeats=1):
+    """Time the CPU oracle as it stands on a bounded sample of the workload: ONE of the 8 KV
+    heads (its 8 query heads) of one `context`-token layer, quantised by the oracle itself;
+    the time is scaled by 8 to a full layer.  Returns (us_per_layer, seconds list, threads)."""
+    import numpy as np
+    from oracle import tq_oracle as O
+    from paper_2604_16957_b200 import inputs as I
+    sh = I.Shape("llama-1kvhead", 1, H_Q // H_KV, 1, D, ALPHA, k_outlier_channels=4)
+    k, v = I.make_kv(sh, context, seed=1000)
+    q = I.make_q(sh, seed=1000)
+    cache = O.Cache(1, 1, context, D)
+    cache.append(k, v)
+    del k, v
+    secs = []
+    for _ in range(repeats):
+        t = time.perf_counter()
+        out = O.attention(cache, q, ALPHA)
+        secs.append(time.perf_counter() - t)
+    assert np.all(np.isfinite(out))
+    return [s * H_KV * 1e6 for s in secs], secs, O.num_threads()
+
+
+def run_reference(args, rank):
+    """--impl reference: the oracle, timed on the host cores, same metric and config."""
+    if rank != 0:
+        return
+    # one cache build, then warmup + steps timed repetitions on it
+    per, secs, threads = oracle_sample_us_per_layer(args.context, repeats=args.warmup + args.steps)
+    timed = per[args.warmup:]
+    value = sum(timed) / len(timed)
+    sample = (f"1 of {H_KV} KV heads ({H_Q // H_KV} of {H_Q} query heads) of one {args.context}-token layer per step, "
+              f"fp64 oracle, time scaled x{H_KV} to a full layer")
+    line = {"impl": "reference", "metric": "int4 decode-attn us/layer @128K (Llama-70B shape)", "value": value,
+            "unit": "us/layer", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": value * args.layers / 1e3, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(args),
+            "cpu_baseline": {"value": value, "unit": "us/layer", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "us/layer", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def config_dict(args):
+    return {"workload": f"llama70b-shape long context: B=1, H_q={H_Q}, H_kv={H_KV}, d={D}, context={args.context}, "
+                        f"{args.layers} layers resident, int4 KV group 32, attn_scale=1/sqrt(d), one decode step "
+                        f"layer by layer (quantize-append + fused int4 attention + split combine)",
+            "context": args.context, "layers": args.layers, "H_q": H_Q, "H_kv": H_KV, "d": D,
+            "l2": "inputs larger than L2: every layer's cache (168 MB at 128K) is a distinct buffer, 13.4 GB in all"}
+
+
+# ------------------------------------------------------------------ GPU arm
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    from paper_2604_16957_b200 import tq  # fails loudly if libtq.so is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    L, S = args.layers, args.context
+    total_appends = 2 * (args.warmup + args.steps) + 8
+    S_cap = (S + total_appends + 15) // 16 * 16
+    C = tq.tq_auto_splits(1, H_KV, H_Q, D, S)
+
+    # ---- resident state: L quantised layer caches, filled from seeded device-side normals.
+    # K gets 4 seeded outlier channels x10 per KV head, like the parity-test generator.
+    caches = []
+    gen = torch.Generator(device=dev)
+    ch_rng = torch.Generator().manual_seed(4242)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    for layer in range(L):
+        gen.manual_seed(7000 + layer + 1000 * rank)
+        k = torch.randn((1, H_KV, S, D), generator=gen, device=dev, dtype=torch.float32)
+        for h in range(H_KV):
+            ch = torch.randperm(D, generator=ch_rng)[:4].to(dev)
+            k[0, h, :, ch] *= 10.0
+        k = k.to(torch.float16)
+        v = torch.randn((1, H_KV, S, D), generator=gen, device=dev, dtype=torch.float32).to(torch.float16)
+        cache = tq.KVCache(1, H_KV, S_cap, D, device=dev)
+        tq.tq_kv_quantize_append(cache, k, v, status)
+        caches.append(cache)
+        del k, v
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+    # per-layer step inputs (q, k_new, v_new) in one buffer, outputs in another
+    per_layer_in = H_Q * D + 2 * H_KV * D
+    gen.manual_seed(99 + rank)
+    inp = torch.randn((L, per_layer_in), generator=gen, device=dev, dtype=torch.float32).to(torch.float16)
+    out = torch.zeros((L, H_Q, D), dtype=torch.float16, device=dev)
+    o_part, m_part, l_part = tq.alloc_partials(1, H_Q, D, C, device=dev)
+    q_l = [inp[i, :H_Q * D].view(1, H_Q, D) for i in range(L)]
+    kn_l = [inp[i, H_Q * D:H_Q * D + H_KV * D].view(1, H_KV, 1, D) for i in range(L)]
+    vn_l = [inp[i, H_Q * D + H_KV * D:].view(1, H_KV, 1, D) for i in range(L)]
+    out_l = [out[i].view(1, H_Q, D) for i in range(L)]
+
+    def reset_lens():
+        for cch in caches:
+            cch.seq_lens.fill_(S)
+
+    def enqueue(append=True, decode=True, combine=True):
+        for i in range(L):
+            if append:
+                tq.tq_kv_quantize_append(caches[i], kn_l[i], vn_l[i], status)
+            if decode:
+                tq.tq_sdpa_int4_decode(caches[i], q_l[i], ALPHA, C, o_part, m_part, l_part, status)
+            if combine:
+                tq.tq_sdpa_int4_combine(o_part, m_part, l_part, out_l[i])
+
+    def make_graph(**kw):
+        enqueue(**kw)  # eager once (also sets function attributes outside capture)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            enqueue(**kw)
+        return g
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def time_graph(g, warmup, steps, pre=None, post=None):
+        """K replays bracketed by events on the current stream; returns seconds for the K steps."""
+        reset_lens()
+        for _ in range(warmup):
+            if pre: pre()
+            g.replay()
+            if post: post()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            if pre: pre()
+            g.replay()
+            if post: post()
+        e1.record()
+        barrier()
+        t = e0.elapsed_time(e1) / 1e3
+        if world > 1:
+            tt = torch.tensor([t], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            t = float(tt.item())
+        return t
+
+    g_step = make_graph()
+    g_decode = make_graph(append=False, combine=False)
+    g_attn = make_graph(append=False)
+    g_append = make_graph(decode=False, combine=False)
+
+    W, K = args.warmup, args.steps
+    with ClockSampler(local_rank) as clocks:
+        t_step = time_graph(g_step, W, K)
+    us_per_layer = t_step / K / L * 1e6
+
+    # per-kernel figures (same graph-replay timing, decode launches back to back over the L distinct layers)
+    t_decode = time_graph(g_decode, W, K)
+    t_attn = time_graph(g_attn, W, K)
+    t_append = time_graph(g_append, W, K)
+    decode_us = t_decode / K / L * 1e6
+
+    # ---- end to end through host buffers: pinned host inputs -> device, the step, outputs -> pinned host
+    h_in = torch.empty_like(inp, device="cpu").pin_memory()
+    h_in.copy_(inp)
+    h_out = torch.empty_like(out, device="cpu").pin_memory()
+    t_e2e = time_graph(g_step, W, K, pre=lambda: inp.copy_(h_in, non_blocking=True),
+                       post=lambda: (h_out.copy_(out, non_blocking=True), torch.cuda.current_stream().synchronize()))
+    e2e_us = t_e2e / K / L * 1e6
+    assert int(status.item()) == 0, "device status word set during the benchmark"
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (fused decode)
+    peak, peak_src = measured_peak()
+    alg_bytes = H_KV * S * BYTES_PER_TOKEN_HEAD
+    achieved = alg_bytes / (decode_us * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_mma_kernel<128>", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_src, "traffic": ncu_traffic_bytes(),
+                "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": decode_us,
+                "frac_of_nominal_8TBs": achieved / HBM_NOMINAL_GBS}
+
+    line = {"metric": "int4 decode-attn us/layer @128K (Llama-70B shape)", "value": us_per_layer / world,
+            "unit": "us/layer", "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": t_step / K * 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f16 codes->f32 accum",
+            "data": "synthetic", "config": config_dict(args), "clocks": clocks.summary(),
+            "e2e": {"value": e2e_us / world, "unit": "us/layer", "h2d_bytes_per_step": inp.numel() * 2,
+                    "d2h_bytes_per_step": out.numel() * 2},
+            "gpu_launches": 3 * L * K, "roofline": roofline,
+            "breakdown_us_per_layer": {"append+decode+combine": us_per_layer, "decode+combine": t_attn / K / L * 1e6,
+                                       "decode": decode_us, "append": t_append / K / L * 1e6},
+            "hbm_gbs_whole_step": alg_bytes / (us_per_layer * 1e-6) / 1e9, "num_splits": C,
+            "paper_context": PAPER_CONTEXT}
+    if world > 1:
+        line["config"]["replicas"] = "independent replicas, no collective (the path does not shard in this build)"
+
+    if not args.no_compare:
+        line["dequant_then_attend_us_per_layer"] = time_dequant_then_attend(tq, torch, caches, q_l, out, S, S_cap, dev)
+    if not args.no_cpu_baseline:
+        per, secs, threads = oracle_sample_us_per_layer(S, repeats=2)
+        line["cpu_baseline"] = {"value": min(per), "unit": "us/layer", "cores": threads, "kind": "oracle",
+                                "sample": f"1 of {H_KV} KV heads ({H_Q // H_KV} of {H_Q} query heads) of one {S}-token "
+                                          f"layer, best of 2 runs ({min(secs):.2f} s), scaled x{H_KV} to a full layer"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def ncu_traffic_bytes():
+    """DRAM bytes (read + write) of one fused-decode launch from the committed ncu summary, if any."""
+    path = os.path.join(ROOT, "profiles", "decode_mma_llama128k_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f)["dram_bytes_per_launch"]
+    except Exception:
+        return None
+
+
+def time_dequant_then_attend(tq, torch, caches, q_l, out, S, S_cap, dev):
+    """The comparison path on the same GPU and inputs, one layer at a time (its matrix workspace is
+    1 GB in fp32), rotating over distinct layers."""
+    res = {}
+    for name, f32 in (("fp32_workspace", True), ("fp16_workspace", False)):
+        nbytes = tq.tq_dequant_workspace_bytes(1, H_KV, H_Q, S_cap, D, f32)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        o = out[0].view(1, H_Q, D)
+        n = min(len(caches), 8)
+        for i in range(2):
+            tq.tq_sdpa_dequant_then_attend(caches[i % n], q_l[i % n], ALPHA, ws, f32, o)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(n):
+            tq.tq_sdpa_dequant_then_attend(caches[i], q_l[i], ALPHA, ws, f32, o)
+        e1.record()
+        torch.cuda.synchronize()
+        res[name] = e0.elapsed_time(e1) / n * 1e3
+        del ws
+    return res
+
+
+if __name__ == "__main__":
+    main()
