@@ -27,8 +27,8 @@
 //
 // Shared-memory layout of one stage (16 tokens of one KV head):
 //   K codes [16][D/2] | V codes [16][D/2] | K scale [16][D/32] | K zero | V scale | V zero
-// The 16-byte chunks of a code row are XOR-swizzled with the token index so that both access
-// patterns below are bank-conflict free:
+// Code rows are padded by 16 bytes (pitch D/2 + 16) so that both access patterns below are
+// bank-conflict free while every address is one per-lane base plus a compile-time offset:
 //   K: lane (gid, tid4) reads word tid4 of group g of token gid      (8 tokens x 16 B per load)
 //   V: lane (gid, tid4) reads word gid%4 of group g of token 2*tid4  (4 tokens x 16 B per load)
 #include "tq_internal.cuh"
@@ -48,16 +48,21 @@ constexpr uint32_t kMaskHi = 0x00F000F0u;  // nibbles 1 / 5: n * 2^-20 as fp16
 template <int D>
 struct Cfg {
   static constexpr int NG = D / 32;                 // groups per row == 16-byte chunks per code row
-  static constexpr int ROWB = D / 2;                // bytes per code row
-  static constexpr int PK = kBlk * ROWB;            // code bytes per stage, K or V
+  static constexpr int ROWB = D / 2;                // bytes per code row in global memory
+  static constexpr int PITCH = ROWB + 16;           // bytes per code row in shared memory
+  static constexpr int PK = kBlk * PITCH;           // code bytes per stage, K or V
   static constexpr int SZ = kBlk * NG * 2;          // bytes of one scale or zero array per stage
-  static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1280 / 2560 / 5120 bytes
-  static constexpr int SWZ_SHIFT = NG == 2 ? 2 : (NG == 4 ? 1 : 0);
-  static constexpr int NST = D == 64 ? 8 : 4;       // stages in the per-warp ring
+  static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1792 / 3072 / 5632 bytes
+  static constexpr int NST = D == 64 ? 6 : 4;       // stages in the per-warp ring
   static constexpr int MINB = D == 256 ? 1 : 2;     // resident blocks per SM
-  static constexpr int PIPE = kWarps * NST * STAGE; // 80 KB (D = 64, 128), 160 KB (D = 256)
+  static constexpr int PIPE = kWarps * NST * STAGE; // 84 KB (D = 64), 96 KB (128), 176 KB (256)
   static constexpr int MERGE = kWarps * (8 * D + 16) * 4;
   static constexpr int SMEM = (PIPE > MERGE ? PIPE : MERGE) + 8 * NG * 4;
+  // loader geometry
+  static constexpr int TOK_PER_PASS = 32 / NG;      // tokens covered by one warp-wide pass of 16-byte chunks
+  static constexpr int CODE_PASSES = kBlk / TOK_PER_PASS;
+  static constexpr int LPA = NG == 2 ? 4 : 8;       // lanes per scale/zero array
+  static constexpr int SZ_PASSES = (SZ / 16) / LPA;
 };
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -92,33 +97,42 @@ __device__ __forceinline__ void cp_async_wait() {
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
 
-// Global pointers of one (sequence, KV head): row 0 of each array.
-struct HeadPtrs {
-  const uint8_t *kp, *vp;
-  const uint8_t *ks, *kz, *vs, *vz;  // byte pointers to the fp16 arrays
-};
-
-// Issue the cp.async copies of token block `gb` (tokens 16*gb .. 16*gb+15) into the stage at
-// shared address `sdst`.  The whole block lies inside the allocation (S_cap % 16 == 0).
+// Per-lane source pointers of the next token block to fetch, and the per-lane destination
+// offsets inside a stage.  Advancing to the warp's next block is three pointer additions.
 template <int D>
-__device__ __forceinline__ void issue_stage(const HeadPtrs& hp, int gb, uint32_t sdst, int lane) {
+struct Loader {
   using C = Cfg<D>;
-  const long long tok0 = static_cast<long long>(gb) * kBlk;
-#pragma unroll
-  for (int i = lane; i < kBlk * C::NG; i += 32) {
-    const int tok = i / C::NG, g = i % C::NG;
-    const uint32_t off = tok * C::ROWB + ((g ^ ((tok >> C::SWZ_SHIFT) & (C::NG - 1))) << 4);
-    cp_async16(sdst + off, hp.kp + tok0 * C::ROWB + i * 16);
-    cp_async16(sdst + C::PK + off, hp.vp + tok0 * C::ROWB + i * 16);
+  const uint8_t *pk, *pv, *psz;  // psz points into one of the four scale / zero arrays, chosen by lane
+  uint32_t dst_code, dst_sz;
+  bool sz_lane;                  // this lane copies scale / zero chunks (all lanes unless D = 64)
+
+  __device__ __forceinline__ void init(const tq_kv_cache& cache, long long row0, int first_blk, int lane) {
+    const long long tok0 = static_cast<long long>(first_blk) * kBlk;
+    pk = cache.k_packed + (row0 + tok0) * C::ROWB + lane * 16;
+    pv = cache.v_packed + (row0 + tok0) * C::ROWB + lane * 16;
+    dst_code = (lane / C::NG) * C::PITCH + (lane % C::NG) * 16;
+    const int arr = lane / C::LPA, ch = lane % C::LPA;
+    const uint16_t* base = arr == 0 ? cache.k_scale : (arr == 1 ? cache.k_zero : (arr == 2 ? cache.v_scale : cache.v_zero));
+    sz_lane = arr < 4;
+    psz = reinterpret_cast<const uint8_t*>(base) + (row0 + tok0) * (C::NG * 2) + ch * 16;
+    dst_sz = 2 * C::PK + arr * C::SZ + ch * 16;
   }
-  constexpr int kSzChunks = C::SZ / 16;  // per array
+  // copy one 16-token block into the stage at shared address `stage`, then step to the block kWarps further on
+  __device__ __forceinline__ void issue(uint32_t stage) {
 #pragma unroll
-  for (int j = lane; j < 4 * kSzChunks; j += 32) {
-    const int arr = j / kSzChunks, ch = j % kSzChunks;
-    const uint8_t* base = arr == 0 ? hp.ks : (arr == 1 ? hp.kz : (arr == 2 ? hp.vs : hp.vz));
-    cp_async16(sdst + 2 * C::PK + arr * C::SZ + ch * 16, base + tok0 * (C::NG * 2) + ch * 16);
+    for (int j = 0; j < C::CODE_PASSES; ++j) {
+      cp_async16(stage + dst_code + j * C::TOK_PER_PASS * C::PITCH, pk + j * 512);
+      cp_async16(stage + C::PK + dst_code + j * C::TOK_PER_PASS * C::PITCH, pv + j * 512);
+    }
+    if (C::LPA * 4 == 32 || sz_lane) {
+#pragma unroll
+      for (int j = 0; j < C::SZ_PASSES; ++j) cp_async16(stage + dst_sz + j * C::LPA * 16, psz + j * C::LPA * 16);
+    }
+    pk += kWarps * kBlk * C::ROWB;
+    pv += kWarps * kBlk * C::ROWB;
+    psz += kWarps * kBlk * C::NG * 2;
   }
-}
+};
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
@@ -171,27 +185,22 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     if (gid < nh)
       raw = *reinterpret_cast<const uint4*>(q + (static_cast<long long>(b) * H_q + h0 + gid) * D + g * 32 + tid4 * 8);
     const __half2 sixteenth = __float2half2_rn(0.0625f);
-    qf[g][0] = __byte_perm(raw.x, raw.z, 0x5410);                                        // (c0, c4)
+    qf[g][0] = __byte_perm(raw.x, raw.z, 0x5410);                                            // (c0, c4)
     qf[g][1] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(raw.x, raw.z, 0x7632)), sixteenth));  // (c1, c5) / 16
-    qf[g][2] = __byte_perm(raw.y, raw.w, 0x5410);                                        // (c2, c6)
+    qf[g][2] = __byte_perm(raw.y, raw.w, 0x5410);                                            // (c2, c6)
     qf[g][3] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(raw.y, raw.w, 0x7632)), sixteenth));  // (c3, c7) / 16
     qs[g][0] = sm_qs[(2 * tid4) * NG + g];
     qs[g][1] = sm_qs[(2 * tid4 + 1) * NG + g];
   }
 
-  // ---- this warp's token blocks: gb = blk0 + warp, blk0 + warp + kWarps, ...
+  // ---- this warp's token blocks: blk0 + warp, blk0 + warp + kWarps, ...
   const int blk0 = t0 / kBlk, blk1 = (t1 + kBlk - 1) / kBlk;
   const int nblk = blk1 - blk0 > warp ? (blk1 - blk0 - warp + kWarps - 1) / kWarps : 0;
   const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
-  HeadPtrs hp;
-  hp.kp = cache.k_packed + row0 * Cf::ROWB;
-  hp.vp = cache.v_packed + row0 * Cf::ROWB;
-  hp.ks = reinterpret_cast<const uint8_t*>(cache.k_scale) + row0 * (NG * 2);
-  hp.kz = reinterpret_cast<const uint8_t*>(cache.k_zero) + row0 * (NG * 2);
-  hp.vs = reinterpret_cast<const uint8_t*>(cache.v_scale) + row0 * (NG * 2);
-  hp.vz = reinterpret_cast<const uint8_t*>(cache.v_zero) + row0 * (NG * 2);
+  Loader<D> ld;
+  ld.init(cache, row0, blk0 + warp, lane);
 
-  uint8_t* ring = smem + warp * (Cf::NST * Cf::STAGE);
+  uint8_t* const ring = smem + warp * (Cf::NST * Cf::STAGE);
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
 
   float oacc[D / 16][4];  // [M tile][c0..c3]: rows = channels, cols = heads 2*tid4, 2*tid4+1
@@ -203,34 +212,36 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
   const float cs = attn_scale * kLog2e * 16777216.0f;  // scores carry 2^-24 from the code operands
 
-  // per-lane constants of the V side
-  const int swzA = ((2 * tid4) >> Cf::SWZ_SHIFT) & (NG - 1);
-  const int swzB = ((2 * tid4 + 1) >> Cf::SWZ_SHIFT) & (NG - 1);
-  const int swzK = (gid >> Cf::SWZ_SHIFT) & (NG - 1);
+  // per-lane byte offsets inside a stage (everything else is a compile-time offset from these)
+  const uint32_t k_lane = gid * Cf::PITCH + tid4 * 4;                          // K codes: token gid, word tid4
+  const uint32_t v_lane = Cf::PK + (2 * tid4) * Cf::PITCH + (gid & 3) * 4;     // V codes: token 2*tid4, word gid%4
+  const uint32_t ksz_lane = 2 * Cf::PK + gid * (NG * 2);                       // K scale row of token gid
+  const uint32_t vsz_lane = 2 * Cf::PK + 2 * Cf::SZ + (2 * tid4) * (NG * 2);   // V scale rows of tokens 2*tid4, +1
   const uint32_t bsel0 = gid >> 2, bsel1 = 2 + (gid >> 2);  // byte of the word used for M-tile half 0 / 1
   const uint32_t sel0 = bsel0 | (bsel0 << 4) | ((4 + bsel0) << 8) | ((4 + bsel0) << 12);
   const uint32_t sel1 = bsel1 | (bsel1 << 4) | ((4 + bsel1) << 8) | ((4 + bsel1) << 12);
 
 #pragma unroll
   for (int s = 0; s < Cf::NST - 1; ++s) {
-    if (s < nblk) issue_stage<D>(hp, blk0 + warp + s * kWarps, ring_s + s * Cf::STAGE, lane);
+    if (s < nblk) ld.issue(ring_s + s * Cf::STAGE);
     cp_async_commit();
   }
 
+  int stage = 0;                    // stage consumed in this iteration
+  int fill = Cf::NST - 1;           // stage filled in this iteration
   for (int k = 0; k < nblk; ++k) {
     cp_async_wait<Cf::NST - 2>();
     __syncwarp();
-    {
-      const int kn = k + Cf::NST - 1;
-      if (kn < nblk) issue_stage<D>(hp, blk0 + warp + kn * kWarps, ring_s + (kn % Cf::NST) * Cf::STAGE, lane);
-      cp_async_commit();
-    }
-    uint8_t* st = ring + (k % Cf::NST) * Cf::STAGE;
-    const int gb = blk0 + warp + k * kWarps;
-    const int valid = t1 - gb * kBlk;  // >= 16 except in the block that holds the end of the sequence
-    if (valid < kBlk) {
+    if (k + Cf::NST - 1 < nblk) ld.issue(ring_s + fill * Cf::STAGE);
+    cp_async_commit();
+    fill = fill + 1 == Cf::NST ? 0 : fill + 1;
+    const uint8_t* st = ring + stage * Cf::STAGE;
+    stage = stage + 1 == Cf::NST ? 0 : stage + 1;
+    const int valid = t1 - (blk0 + warp + k * kWarps) * kBlk;  // >= 16 except in the block holding the sequence end
+    const bool tail = valid < kBlk;
+    if (tail) {
       // rows past the end hold unspecified bytes: give them scale = zero = 0 so they dequantise to 0
-      __half* sz = reinterpret_cast<__half*>(st + 2 * Cf::PK);
+      __half* sz = reinterpret_cast<__half*>(const_cast<uint8_t*>(st) + 2 * Cf::PK);
       for (int i = lane; i < 4 * kBlk * NG; i += 32) {
         const int tok = (i / NG) % kBlk;
         if (tok >= valid) sz[i] = __ushort_as_half(0);
@@ -241,20 +252,31 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     // ---------------- scores: S[token][head] over this block's 16 tokens
     float sc[4] = {0.f, 0.f, 0.f, 0.f};
     {
-      const __half* ks = reinterpret_cast<const __half*>(st + 2 * Cf::PK);
-      const __half* kz = reinterpret_cast<const __half*>(st + 2 * Cf::PK + Cf::SZ);
-      const uint8_t* kp = st;
+      const uint8_t* kp = st + k_lane;
+      // scales and zeros of tokens gid and gid + 8, all groups
+      __half2 ks_lo[NG / 2], kz_lo[NG / 2], ks_hi[NG / 2], kz_hi[NG / 2];
+      {
+        const uint32_t* r = reinterpret_cast<const uint32_t*>(st + ksz_lane);
+#pragma unroll
+        for (int i = 0; i < NG / 2; ++i) {
+          ks_lo[i] = u32_as_h2(r[i]);
+          kz_lo[i] = u32_as_h2(r[Cf::SZ / 4 + i]);
+          ks_hi[i] = u32_as_h2(r[8 * NG / 2 + i]);
+          kz_hi[i] = u32_as_h2(r[Cf::SZ / 4 + 8 * NG / 2 + i]);
+        }
+      }
 #pragma unroll
       for (int g = 0; g < NG; ++g) {
-        const uint32_t off = ((g ^ swzK) << 4) + tid4 * 4;
-        const uint32_t w0 = *reinterpret_cast<const uint32_t*>(kp + gid * Cf::ROWB + off);
-        const uint32_t w8 = *reinterpret_cast<const uint32_t*>(kp + (gid + 8) * Cf::ROWB + off);
+        const uint32_t w0 = *reinterpret_cast<const uint32_t*>(kp + g * 16);
+        const uint32_t w8 = *reinterpret_cast<const uint32_t*>(kp + 8 * Cf::PITCH + g * 16);
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         mma16816(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1]);
         const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
         mma16816(acc, y0 & kMaskLo, y8 & kMaskLo, y0 & kMaskHi, y8 & kMaskHi, qf[g][2], qf[g][3]);
-        const float s_lo = __half2float(ks[gid * NG + g]), z_lo = __half2float(kz[gid * NG + g]);
-        const float s_hi = __half2float(ks[(gid + 8) * NG + g]), z_hi = __half2float(kz[(gid + 8) * NG + g]);
+        const float s_lo = (g & 1) ? __high2float(ks_lo[g >> 1]) : __low2float(ks_lo[g >> 1]);
+        const float z_lo = (g & 1) ? __high2float(kz_lo[g >> 1]) : __low2float(kz_lo[g >> 1]);
+        const float s_hi = (g & 1) ? __high2float(ks_hi[g >> 1]) : __low2float(ks_hi[g >> 1]);
+        const float z_hi = (g & 1) ? __high2float(kz_hi[g >> 1]) : __low2float(kz_hi[g >> 1]);
         sc[0] = fmaf(s_lo, fmaf(-z_lo, qs[g][0], acc[0]), sc[0]);
         sc[1] = fmaf(s_lo, fmaf(-z_lo, qs[g][1], acc[1]), sc[1]);
         sc[2] = fmaf(s_hi, fmaf(-z_hi, qs[g][0], acc[2]), sc[2]);
@@ -263,7 +285,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     }
     // ---------------- online softmax (log2 domain)
     float a0 = sc[0] * cs, a1 = sc[1] * cs, a2 = sc[2] * cs, a3 = sc[3] * cs;
-    if (valid < kBlk) {
+    if (tail) {
       if (gid >= valid) a0 = a1 = -INFINITY;
       if (gid + 8 >= valid) a2 = a3 = -INFINITY;
     }
@@ -275,9 +297,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, off));
         bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, off));
       }
-      const float n0 = fmaxf(m0, bm0), n1 = fmaxf(m1, bm1);
-      const float f0 = n0 == -INFINITY ? 1.f : ex2(m0 - n0);
-      const float f1 = n1 == -INFINITY ? 1.f : ex2(m1 - n1);
+      const float n0 = fmaxf(m0, bm0), n1 = fmaxf(m1, bm1);  // finite: every block has a valid token
+      const float f0 = ex2(m0 - n0), f1 = ex2(m1 - n1);      // ex2(-inf) = 0 on the first block
       m0 = n0;
       m1 = n1;
       l0 *= f0;
@@ -291,10 +312,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         zacc[g][0] *= f0; zacc[g][1] *= f1; zacc[g][2] *= f0; zacc[g][3] *= f1;
       }
     }
-    const float p0 = a0 == -INFINITY ? 0.f : ex2(a0 - m0);
-    const float p1 = a1 == -INFINITY ? 0.f : ex2(a1 - m1);
-    const float p2 = a2 == -INFINITY ? 0.f : ex2(a2 - m0);
-    const float p3 = a3 == -INFINITY ? 0.f : ex2(a3 - m1);
+    const float p0 = ex2(a0 - m0), p1 = ex2(a1 - m1), p2 = ex2(a2 - m0), p3 = ex2(a3 - m1);  // ex2(-inf) = 0
     l0 += p0 + p2;
     l1 += p1 + p3;
     // P^T as B fragments: (tokens 2*tid4, 2*tid4+1 | head gid) and (tokens 8+2*tid4, 9+2*tid4 | head gid)
@@ -303,33 +321,31 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
     // ---------------- P.V: O^T[channel][head] += V^T[channel][token] * (P * s)[token][head]
     {
-      const uint8_t* vp = st + Cf::PK;
-      const uint32_t* vs32 = reinterpret_cast<const uint32_t*>(st + 2 * Cf::PK + 2 * Cf::SZ);
-      const uint32_t* vz32 = reinterpret_cast<const uint32_t*>(st + 2 * Cf::PK + 3 * Cf::SZ);
-      const int tA = 2 * tid4;  // tokens tA, tA+1 (k slots 2*tid4, +1) and tA+8, tA+9 (k slots 2*tid4+8, +9)
-      // scales / zeros of the four tokens, NG halves each = NG/2 words each
-      uint32_t sA[NG / 2], sB[NG / 2], sC[NG / 2], sD[NG / 2], zA[NG / 2], zB[NG / 2], zC[NG / 2], zD[NG / 2];
+      const uint8_t* vp = st + v_lane;
+      // scales / zeros of tokens (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9): NG halves per token
+      uint32_t sAB[NG], sCD[NG], zAB[NG], zCD[NG];  // [0, NG/2) first token, [NG/2, NG) second token
+      {
+        const uint32_t* r = reinterpret_cast<const uint32_t*>(st + vsz_lane);
 #pragma unroll
-      for (int i = 0; i < NG / 2; ++i) {
-        sA[i] = vs32[tA * (NG / 2) + i];       sB[i] = vs32[(tA + 1) * (NG / 2) + i];
-        sC[i] = vs32[(tA + 8) * (NG / 2) + i]; sD[i] = vs32[(tA + 9) * (NG / 2) + i];
-        zA[i] = vz32[tA * (NG / 2) + i];       zB[i] = vz32[(tA + 1) * (NG / 2) + i];
-        zC[i] = vz32[(tA + 8) * (NG / 2) + i]; zD[i] = vz32[(tA + 9) * (NG / 2) + i];
+        for (int i = 0; i < NG; ++i) {
+          sAB[i] = r[i];
+          sCD[i] = r[8 * NG / 2 + i];
+          zAB[i] = r[Cf::SZ / 4 + i];
+          zCD[i] = r[Cf::SZ / 4 + 8 * NG / 2 + i];
+        }
       }
-      const uint32_t wofs = (gid & 3) * 4;
 #pragma unroll
       for (int g = 0; g < NG; ++g) {
         const uint32_t psel = (g & 1) ? 0x7632u : 0x5410u;
-        const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(__byte_perm(sA[g >> 1], sB[g >> 1], psel))));
-        const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(__byte_perm(sC[g >> 1], sD[g >> 1], psel))));
-        const uint32_t zab = __byte_perm(zA[g >> 1], zB[g >> 1], psel);
-        const uint32_t zcd = __byte_perm(zC[g >> 1], zD[g >> 1], psel);
+        const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(__byte_perm(sAB[g >> 1], sAB[NG / 2 + (g >> 1)], psel))));
+        const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(__byte_perm(sCD[g >> 1], sCD[NG / 2 + (g >> 1)], psel))));
+        const uint32_t zab = __byte_perm(zAB[g >> 1], zAB[NG / 2 + (g >> 1)], psel);
+        const uint32_t zcd = __byte_perm(zCD[g >> 1], zCD[NG / 2 + (g >> 1)], psel);
         mma16816(zacc[g], zab, zab, zcd, zcd, b0, b1);
-        const uint32_t offA = ((g ^ swzA) << 4) + wofs, offB = ((g ^ swzB) << 4) + wofs;
-        const uint32_t wA = *reinterpret_cast<const uint32_t*>(vp + tA * Cf::ROWB + offA);
-        const uint32_t wB = *reinterpret_cast<const uint32_t*>(vp + (tA + 1) * Cf::ROWB + offB);
-        const uint32_t wC = *reinterpret_cast<const uint32_t*>(vp + (tA + 8) * Cf::ROWB + offA);
-        const uint32_t wD = *reinterpret_cast<const uint32_t*>(vp + (tA + 9) * Cf::ROWB + offB);
+        const uint32_t wA = *reinterpret_cast<const uint32_t*>(vp + g * 16);
+        const uint32_t wB = *reinterpret_cast<const uint32_t*>(vp + Cf::PITCH + g * 16);
+        const uint32_t wC = *reinterpret_cast<const uint32_t*>(vp + 8 * Cf::PITCH + g * 16);
+        const uint32_t wD = *reinterpret_cast<const uint32_t*>(vp + 9 * Cf::PITCH + g * 16);
         uint32_t u = __byte_perm(wA, wB, sel0), u2 = __byte_perm(wC, wD, sel0);
         mma16816(oacc[2 * g], u & kMaskLo, u & kMaskHi, u2 & kMaskLo, u2 & kMaskHi, b0, b1);
         u = __byte_perm(wA, wB, sel1);
@@ -347,16 +363,16 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     l1 += __shfl_xor_sync(0xffffffffu, l1, off);
   }
   __syncthreads();  // every warp is done with its ring; the memory is reused below
-  float* mo = reinterpret_cast<float*>(smem) + warp * (8 * D + 16);  // [8 heads][D] then m[8], l[8]
+  float* mo = reinterpret_cast<float*>(smem) + warp * (8 * D + 16);  // [D channels][8 heads] then m[8], l[8]
 #pragma unroll
   for (int mt = 0; mt < D / 16; ++mt) {
     const int g = mt >> 1;
     const int ch = 32 * g + 8 * (gid & 3) + 2 * (2 * (mt & 1) + (gid >> 2));
     // even channel: codes carried 2^-24; odd channel (high nibble): 2^-20
-    mo[(2 * tid4) * D + ch] = oacc[mt][0] * 16777216.0f - zacc[g][0];
-    mo[(2 * tid4 + 1) * D + ch] = oacc[mt][1] * 16777216.0f - zacc[g][1];
-    mo[(2 * tid4) * D + ch + 1] = oacc[mt][2] * 1048576.0f - zacc[g][0];
-    mo[(2 * tid4 + 1) * D + ch + 1] = oacc[mt][3] * 1048576.0f - zacc[g][1];
+    *reinterpret_cast<float2*>(mo + ch * 8 + 2 * tid4) =
+        make_float2(oacc[mt][0] * 16777216.0f - zacc[g][0], oacc[mt][1] * 16777216.0f - zacc[g][1]);
+    *reinterpret_cast<float2*>(mo + (ch + 1) * 8 + 2 * tid4) =
+        make_float2(oacc[mt][2] * 1048576.0f - zacc[g][0], oacc[mt][3] * 1048576.0f - zacc[g][1]);
   }
   if (gid == 0) {
     mo[8 * D + 2 * tid4] = m0;
@@ -366,8 +382,9 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   __syncthreads();
   const float* all = reinterpret_cast<const float*>(smem);
-  for (int idx = threadIdx.x; idx < nh * D; idx += kThreads) {
-    const int h = idx / D, x = idx - h * D;
+  for (int idx = threadIdx.x; idx < 8 * D; idx += kThreads) {
+    const int x = idx >> 3, h = idx & 7;  // consecutive threads take consecutive heads of one channel
+    if (h >= nh) continue;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) M = fmaxf(M, all[w * (8 * D + 16) + 8 * D + h]);
@@ -376,9 +393,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) {
         const float* wb = all + w * (8 * D + 16);
-        const float mw = wb[8 * D + h];
-        const float f = mw == -INFINITY ? 0.f : ex2(mw - M);
-        num = fmaf(f, wb[h * D + x], num);
+        const float f = ex2(wb[8 * D + h] - M);  // ex2(-inf) = 0 for a warp that saw no token
+        num = fmaf(f, wb[idx], num);
         den = fmaf(f, wb[8 * D + 8 + h], den);
       }
     }
@@ -394,8 +410,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 template <int D>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C, float* o_part,
                    float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  static const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                       Cfg<D>::SMEM);
+  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                Cfg<D>::SMEM);
   if (attr != cudaSuccess) return attr;
   const int G = H_q / c.H_kv;
   dim3 grid(C, c.H_kv * ((G + 7) / 8), c.B);
