@@ -57,17 +57,22 @@ typedef enum tq_result {
 #define TQ_SPLIT_QUANTUM 16 /* split boundaries fall on multiples of this many tokens */
 
 /*
- * The int4 KV cache of ONE layer.  Token-major arrays; sequence b, KV head h, token i is row
- * (b * H_kv + h) * S_cap + i of each array.  Rows at or beyond seq_lens[b] are unspecified.
+ * The int4 KV cache of ONE layer.  The paper fixes the values (codes, fp16 scale, fp16 zero per
+ * group of 32) but not the array order; this is the order the kernels are built for.
+ *   codes : token-major.  Sequence b, KV head h, token i is row (b * H_kv + h) * S_cap + i, d/2 bytes.
+ *   scales, zeros : blocked by 16 tokens so that the 16 values of one group are contiguous:
+ *       element (b, h, token i, group g) is at index
+ *       (((b * H_kv + h) * (S_cap / 16) + i / 16) * (d / 32) + g) * 16 + i % 16.
+ * Rows at or beyond seq_lens[b] are unspecified.
  * Requirements: d in {64, 128, 256}; S_cap a positive multiple of 16; B, H_kv >= 1.
  */
 typedef struct tq_kv_cache {
-  uint8_t* k_packed;  /* [B][H_kv][S_cap][d/2]  packed codes of K */
-  uint8_t* v_packed;  /* [B][H_kv][S_cap][d/2]  packed codes of V */
-  uint16_t* k_scale;  /* [B][H_kv][S_cap][d/32] fp16 scales of K */
-  uint16_t* k_zero;   /* [B][H_kv][S_cap][d/32] fp16 zero-points of K */
-  uint16_t* v_scale;  /* [B][H_kv][S_cap][d/32] */
-  uint16_t* v_zero;   /* [B][H_kv][S_cap][d/32] */
+  uint8_t* k_packed;  /* [B][H_kv][S_cap][d/2]        packed codes of K */
+  uint8_t* v_packed;  /* [B][H_kv][S_cap][d/2]        packed codes of V */
+  uint16_t* k_scale;  /* [B][H_kv][S_cap/16][d/32][16] fp16 scales of K */
+  uint16_t* k_zero;   /* [B][H_kv][S_cap/16][d/32][16] fp16 zero-points of K */
+  uint16_t* v_scale;  /* [B][H_kv][S_cap/16][d/32][16] */
+  uint16_t* v_zero;   /* [B][H_kv][S_cap/16][d/32][16] */
   int32_t* seq_lens;  /* [B] number of valid tokens per sequence (device memory, updated by append) */
   int32_t B, H_kv, S_cap, d;
 } tq_kv_cache;

@@ -25,11 +25,14 @@ struct SrcInt4 {
   static constexpr int EPL = D / 32;  // elements per lane
   const uint8_t *kp, *vp;
   const __half *ks, *kz, *vs, *vz;
+  int S_cap;
   __device__ void load(bool is_v, long long row, int lane, float (&x)[EPL]) const {
     const uint8_t* p = (is_v ? vp : kp) + row * (D / 2) + lane * (EPL / 2);
     const int g = (lane * EPL) / 32;
-    const float s = __half2float((is_v ? vs : ks)[row * (D / 32) + g]);
-    const float z = __half2float((is_v ? vz : kz)[row * (D / 32) + g]);
+    const long long bh = row / S_cap;
+    const long long si = scale_index(bh, S_cap, D / 32, static_cast<int>(row - bh * S_cap), g);
+    const float s = __half2float((is_v ? vs : ks)[si]);
+    const float z = __half2float((is_v ? vz : kz)[si]);
 #pragma unroll
     for (int i = 0; i < EPL / 2; ++i) {
       const uint32_t byte = p[i];
@@ -168,8 +171,9 @@ __global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T
   const int t = static_cast<int>(r - h * len);
   const long long row = (static_cast<long long>(b) * c.H_kv + h) * c.S_cap + t;
   const uint32_t w = reinterpret_cast<const uint32_t*>((is_v ? c.v_packed : c.k_packed) + row * (d >> 1))[cc];
-  const float s = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_scale : c.k_scale)[row * (d >> 5) + (cc >> 2)]);
-  const float z = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_zero : c.k_zero)[row * (d >> 5) + (cc >> 2)]);
+  const long long si = scale_index(static_cast<long long>(b) * c.H_kv + h, c.S_cap, d >> 5, t, cc >> 2);
+  const float s = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_scale : c.k_scale)[si]);
+  const float z = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_zero : c.k_zero)[si]);
   float x[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(__fsub_rn(static_cast<float>((w >> (4 * i)) & 0xF), z), s);
@@ -193,7 +197,7 @@ cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q,
     constexpr int D = decltype(dtag)::value;
     SrcInt4<D> src{c.k_packed, c.v_packed, reinterpret_cast<const __half*>(c.k_scale),
                    reinterpret_cast<const __half*>(c.k_zero), reinterpret_cast<const __half*>(c.v_scale),
-                   reinterpret_cast<const __half*>(c.v_zero)};
+                   reinterpret_cast<const __half*>(c.v_zero), c.S_cap};
     return launch_simple<D>(src, c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
   };
   switch (c.d) {

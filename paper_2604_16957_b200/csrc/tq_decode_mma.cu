@@ -26,11 +26,17 @@
 // the rescale of the accumulators rare).
 //
 // Shared-memory layout of one stage (16 tokens of one KV head):
-//   K codes [16][D/2] | V codes [16][D/2] | K scale [16][D/32] | K zero | V scale | V zero
-// Code rows are padded by 16 bytes (pitch D/2 + 16) so that both access patterns below are
-// bank-conflict free while every address is one per-lane base plus a compile-time offset:
-//   K: lane (gid, tid4) reads word tid4 of group g of token gid      (8 tokens x 16 B per load)
-//   V: lane (gid, tid4) reads word gid%4 of group g of token 2*tid4  (4 tokens x 16 B per load)
+//   K codes [16][D/2] | V codes [16][D/2] | K scale [D/32][16] | K zero | V scale | V zero
+// The 16-byte chunks of the code rows are XOR-swizzled with the token index.  That keeps every
+// quarter-warp of a cp.async writing one aligned 128-byte line (one shared-memory wavefront; a
+// padded layout costs 3-4x the wavefronts on the copy) and makes the fragment loads conflict
+// free.  Fragments come from ldmatrix, whose 8x8 b16 "matrix" is here 8 tokens x one 16-byte
+// chunk (32 codes of one group):
+//   K: plain ldmatrix  -> lane (gid, tid4) holds word tid4 of token gid: 8 codes of one token,
+//      the A operand rows of the score MMA;
+//   V: ldmatrix.trans  -> lane (gid, tid4) holds 16-bit lane gid of tokens 2*tid4 and 2*tid4+1
+//      side by side: the token-pair interleave the P.V MMA needs (k = tokens), done by the
+//      load itself, so V needs no byte permutes.
 #include "tq_internal.cuh"
 
 namespace tq {
@@ -42,6 +48,7 @@ constexpr int kBlk = 16;              // tokens per stage = MMA M (scores) = MMA
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 4.0f;  // log2 units
+constexpr float kNoMax = -1.0e30f;         // running reference before any token was seen
 constexpr uint32_t kMaskLo = 0x000F000Fu;  // nibbles 0 / 4 of a 32-bit word: n * 2^-24 as fp16
 constexpr uint32_t kMaskHi = 0x00F000F0u;  // nibbles 1 / 5: n * 2^-20 as fp16
 
@@ -49,18 +56,19 @@ template <int D>
 struct Cfg {
   static constexpr int NG = D / 32;                 // groups per row == 16-byte chunks per code row
   static constexpr int ROWB = D / 2;                // bytes per code row in global memory
-  static constexpr int PITCH = ROWB + 16;           // bytes per code row in shared memory
-  static constexpr int PK = kBlk * PITCH;           // code bytes per stage, K or V
+  static constexpr int PK = kBlk * ROWB;            // code bytes per stage, K or V
+  static constexpr int SWZ_SHIFT = NG == 2 ? 2 : (NG == 4 ? 1 : 0);  // chunk' = chunk ^ ((tok >> SHIFT) & (NG - 1))
   static constexpr int SZ = kBlk * NG * 2;          // bytes of one scale or zero array per stage
-  static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1792 / 3072 / 5632 bytes
-  static constexpr int NST = D == 64 ? 6 : 4;       // stages in the per-warp ring
+  static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1280 / 2560 / 5120 bytes
+  static constexpr int NST = 4;                     // stages in the per-warp ring (power of two)
   static constexpr int MINB = D == 256 ? 1 : 2;     // resident blocks per SM
-  static constexpr int PIPE = kWarps * NST * STAGE; // 84 KB (D = 64), 96 KB (128), 176 KB (256)
+  static constexpr int PIPE = kWarps * NST * STAGE; // 40 KB (D = 64), 80 KB (128), 160 KB (256)
   static constexpr int MERGE = kWarps * (8 * D + 16) * 4;
   static constexpr int SMEM = (PIPE > MERGE ? PIPE : MERGE) + 8 * NG * 4;
   // loader geometry
-  static constexpr int TOK_PER_PASS = 32 / NG;      // tokens covered by one warp-wide pass of 16-byte chunks
-  static constexpr int CODE_PASSES = kBlk / TOK_PER_PASS;
+  static constexpr int PASS_TOK = 32 / NG;          // token rows covered by one warp-wide pass of 16-byte chunks
+  static constexpr int CODE_PASSES = kBlk / PASS_TOK;
+  __host__ __device__ static constexpr int swz(int tok) { return (tok >> SWZ_SHIFT) & (NG - 1); }
   static constexpr int LPA = NG == 2 ? 4 : 8;       // lanes per scale/zero array
   static constexpr int SZ_PASSES = (SZ / 16) / LPA;
 };
@@ -73,10 +81,31 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// d = a * b + z where z is a quad of registers that hold zero (kept apart from d so that no
+// accumulator has to be cleared)
+__device__ __forceinline__ void mma16816_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1, const float (&z)[4]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};\n"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(z[0]), "f"(z[1]), "f"(z[2]), "f"(z[3]));
+}
+
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   uint32_t d;
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
   return d;
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -108,9 +137,12 @@ struct Loader {
 
   __device__ __forceinline__ void init(const tq_kv_cache& cache, long long row0, int first_blk, int lane) {
     const long long tok0 = static_cast<long long>(first_blk) * kBlk;
+    // lane i of a pass copies global chunk i (token i / NG, chunk i % NG): a quarter-warp reads 128
+    // contiguous bytes and writes one aligned 128-byte line.
+    const int tok = lane / C::NG, chunk = lane % C::NG;
     pk = cache.k_packed + (row0 + tok0) * C::ROWB + lane * 16;
     pv = cache.v_packed + (row0 + tok0) * C::ROWB + lane * 16;
-    dst_code = (lane / C::NG) * C::PITCH + (lane % C::NG) * 16;
+    dst_code = tok * C::ROWB + ((chunk ^ C::swz(tok)) << 4);
     const int arr = lane / C::LPA, ch = lane % C::LPA;
     const uint16_t* base = arr == 0 ? cache.k_scale : (arr == 1 ? cache.k_zero : (arr == 2 ? cache.v_scale : cache.v_zero));
     sz_lane = arr < 4;
@@ -121,8 +153,10 @@ struct Loader {
   __device__ __forceinline__ void issue(uint32_t stage) {
 #pragma unroll
     for (int j = 0; j < C::CODE_PASSES; ++j) {
-      cp_async16(stage + dst_code + j * C::TOK_PER_PASS * C::PITCH, pk + j * 512);
-      cp_async16(stage + C::PK + dst_code + j * C::TOK_PER_PASS * C::PITCH, pv + j * 512);
+      // D = 256: a pass covers 4 rows, so odd passes land on rows whose swizzle term differs in bit 2
+      const uint32_t d = stage + ((C::NG == 8 && (j & 1)) ? (dst_code ^ 64u) : dst_code) + j * 512;
+      cp_async16(d, pk + j * 512);
+      cp_async16(d + C::PK, pv + j * 512);
     }
     if (C::LPA * 4 == 32 || sz_lane) {
 #pragma unroll
@@ -133,6 +167,142 @@ struct Loader {
     psz += kWarps * kBlk * C::NG * 2;
   }
 };
+
+template <int D>
+struct WarpCtx {
+  uint8_t* ring;
+  uint32_t kaddr[D / 64];  // ldmatrix row address (offset in a stage) this lane supplies, per K load
+  uint32_t vaddr[D / 64];  // same for the V loads
+  uint32_t ksz_lane, vsz_lane;
+  float cs;
+  int gid;
+};
+
+// One 16-token block: scores -> online softmax -> P.V, all in registers.  TAIL = the block
+// holding the end of the sequence: only its first `valid` tokens count.
+template <int D, bool TAIL>
+__device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, int valid,
+                                           const uint32_t (&qf)[D / 32][4], const float (&qs)[D / 32][2],
+                                           float (&oacc)[D / 16][4], float (&zacc)[D / 32][4], const float (&zero4)[4], float& m0, float& m1,
+                                           float& l0, float& l1) {
+  using Cf = Cfg<D>;
+  constexpr int NG = Cf::NG;
+  if (TAIL) {
+    // rows past the end hold unspecified bytes: give them scale = zero = 0 so they dequantise to 0
+    __half* sz = reinterpret_cast<__half*>(const_cast<uint8_t*>(st) + 2 * Cf::PK);
+    const int lane = threadIdx.x & 31;
+    for (int i = lane; i < 4 * kBlk * NG; i += 32) {
+      if ((i % kBlk) >= valid) sz[i] = __ushort_as_half(0);  // arrays are [group][16 tokens]
+    }
+    __syncwarp();
+  }
+
+  // ---------------- scores: S[token][head] over this block's 16 tokens (carry a factor 2^-24)
+  float sc[4];
+  {
+    // matrix j = 4 * i + m of load i is (tokens 8 * (j / NG) .., group j % NG)
+    uint32_t kw[NG / 2][4], ksz[4];
+#pragma unroll
+    for (int i = 0; i < NG / 2; ++i) ldmatrix_x4(kw[i], st_s + cx.kaddr[i]);
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {
+      const uint32_t w0 = kw[g / 4][g % 4];                      // token gid
+      const uint32_t w8 = kw[(NG + g) / 4][(NG + g) % 4];        // token gid + 8
+      float acc[4];
+      mma16816_first(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1], zero4);
+      const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
+      mma16816(acc, y0 & kMaskLo, y8 & kMaskLo, y0 & kMaskHi, y8 & kMaskHi, qf[g][2], qf[g][3]);
+      // Scales and zeros of tokens gid and gid + 8 for groups g, g+1 by one transposing ldmatrix: its
+      // matrices are (scale | tokens 0-7), (scale | 8-15), (zero | 0-7), (zero | 8-15), each with rows
+      // alternating between the 16-byte chunks of groups g and g+1, so every lane receives element gid
+      // of both chunks: half2 (x[g][token], x[g+1][token]).
+      if ((g & 1) == 0) ldmatrix_x4_trans(ksz, st_s + cx.ksz_lane + 32 * g);
+      const float s_lo = (g & 1) ? __high2float(u32_as_h2(ksz[0])) : __low2float(u32_as_h2(ksz[0]));
+      const float s_hi = (g & 1) ? __high2float(u32_as_h2(ksz[1])) : __low2float(u32_as_h2(ksz[1]));
+      const float z_lo = (g & 1) ? __high2float(u32_as_h2(ksz[2])) : __low2float(u32_as_h2(ksz[2]));
+      const float z_hi = (g & 1) ? __high2float(u32_as_h2(ksz[3])) : __low2float(u32_as_h2(ksz[3]));
+      const float t0 = fmaf(-z_lo, qs[g][0], acc[0]), t1 = fmaf(-z_lo, qs[g][1], acc[1]);
+      const float t2 = fmaf(-z_hi, qs[g][0], acc[2]), t3 = fmaf(-z_hi, qs[g][1], acc[3]);
+      if (g == 0) {
+        sc[0] = s_lo * t0; sc[1] = s_lo * t1; sc[2] = s_hi * t2; sc[3] = s_hi * t3;
+      } else {
+        sc[0] = fmaf(s_lo, t0, sc[0]); sc[1] = fmaf(s_lo, t1, sc[1]);
+        sc[2] = fmaf(s_hi, t2, sc[2]); sc[3] = fmaf(s_hi, t3, sc[3]);
+      }
+    }
+  }
+  // ---------------- online softmax in the log2 domain.  d = score - running reference m; the
+  // reference is raised only when some d exceeds the threshold, so the common path is 4 FMAs.
+  float d0 = fmaf(sc[0], cx.cs, -m0), d1 = fmaf(sc[1], cx.cs, -m1);
+  float d2 = fmaf(sc[2], cx.cs, -m0), d3 = fmaf(sc[3], cx.cs, -m1);
+  if (TAIL) {
+    if (cx.gid >= valid) d0 = d1 = -INFINITY;
+    if (cx.gid + 8 >= valid) d2 = d3 = -INFINITY;
+  }
+  const bool need = fmaxf(fmaxf(d0, d2), fmaxf(d1, d3)) > kRescaleThreshold;
+  if (__any_sync(0xffffffffu, need)) {
+    float a0 = sc[0] * cx.cs, a1 = sc[1] * cx.cs, a2 = sc[2] * cx.cs, a3 = sc[3] * cx.cs;
+    if (TAIL) {
+      if (cx.gid >= valid) a0 = a1 = -INFINITY;
+      if (cx.gid + 8 >= valid) a2 = a3 = -INFINITY;
+    }
+    float bm0 = fmaxf(a0, a2), bm1 = fmaxf(a1, a3);
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {
+      bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, off));
+      bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, off));
+    }
+    const float n0 = fmaxf(m0, bm0), n1 = fmaxf(m1, bm1);
+    const float f0 = ex2(m0 - n0), f1 = ex2(m1 - n1);  // m starts at -1e30: the first factor underflows to 0
+    m0 = n0;
+    m1 = n1;
+    l0 *= f0;
+    l1 *= f1;
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) {
+      oacc[i][0] *= f0; oacc[i][1] *= f1; oacc[i][2] *= f0; oacc[i][3] *= f1;
+    }
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {
+      zacc[g][0] *= f0; zacc[g][1] *= f1;
+    }
+    d0 = a0 - m0; d1 = a1 - m1; d2 = a2 - m0; d3 = a3 - m1;
+  }
+  const float p0 = ex2(d0), p1 = ex2(d1), p2 = ex2(d2), p3 = ex2(d3);  // ex2(-inf) = 0 for masked tokens
+  l0 += p0 + p2;
+  l1 += p1 + p3;
+  // P^T as B fragments: (tokens 2*tid4, 2*tid4+1 | head gid) and (tokens 8+2*tid4, 9+2*tid4 | head gid)
+  const uint32_t pt0 = movmatrix_trans(h2_as_u32(__floats2half2_rn(p0, p1)));
+  const uint32_t pt1 = movmatrix_trans(h2_as_u32(__floats2half2_rn(p2, p3)));
+
+  // ---------------- P.V: O^T[channel][head] += V^T[channel][token] * (P * s)[token][head]
+  {
+    // matrix j = 4 * i + m of load i is (group j / 2, tokens 8 * (j % 2) ..)
+    uint32_t vw[4];
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {
+      // Scales / zeros of token pairs (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9) of group g: an ldmatrix
+      // whose eight row addresses are equal hands every lane word tid4 of that 16-byte chunk; the four
+      // matrices are (scale | tokens 0-7), (scale | 8-15), (zero | 0-7), (zero | 8-15).
+      uint32_t vsz[4];
+      ldmatrix_x4(vsz, st_s + cx.vsz_lane + 32 * g);
+      const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vsz[0])));
+      const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vsz[1])));
+      const uint32_t zab = vsz[2], zcd = vsz[3];
+      // r1 = (tokens 2*tid4, 2*tid4+1), r2 = (tokens 2*tid4+8, +9): 16-bit lane gid of chunk g, i.e. codes of
+      // channels 32g + 4*gid .. +3 of two tokens side by side
+      if ((g & 1) == 0) ldmatrix_x4_trans(vw, st_s + cx.vaddr[g / 2]);
+      const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
+      mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
+      const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
+      const uint32_t uh = y1 & kMaskHi, u2h = y2 & kMaskHi;
+      mma16816(oacc[2 * g + 1], y1 & kMaskLo, uh, y2 & kMaskLo, u2h, b0, b1);
+      // zero-point term: rows 0-7 of A hold z_g (so c0, c1 accumulate sum_tok z_g * B_g); rows 8-15 reuse
+      // the operand registers of the MMA above and produce values that are never read
+      mma16816(zacc[g], zab, uh, zcd, u2h, b0, b1);
+    }
+  }
+}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
@@ -204,22 +374,21 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
 
   float oacc[D / 16][4];  // [M tile][c0..c3]: rows = channels, cols = heads 2*tid4, 2*tid4+1
-  float zacc[NG][4];      // sum_tok B_g * z_g  (rows identical; [0], [1] are used)
+  float zacc[NG][4];      // sum_tok B_g * z_g: [0], [1] are heads 2*tid4, 2*tid4+1; [2], [3] are not used
+  float zero4[4];         // four registers holding 0, opaque to the compiler: the C operand of accumulator-less MMAs
+#pragma unroll
+  for (int i = 0; i < 4; ++i) asm volatile("mov.f32 %0, 0f00000000;\n" : "=f"(zero4[i]));
 #pragma unroll
   for (int i = 0; i < D / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
 #pragma unroll
   for (int g = 0; g < NG; ++g) zacc[g][0] = zacc[g][1] = zacc[g][2] = zacc[g][3] = 0.f;
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  float m0 = kNoMax, m1 = kNoMax, l0 = 0.f, l1 = 0.f;
   const float cs = attn_scale * kLog2e * 16777216.0f;  // scores carry 2^-24 from the code operands
 
   // per-lane byte offsets inside a stage (everything else is a compile-time offset from these)
-  const uint32_t k_lane = gid * Cf::PITCH + tid4 * 4;                          // K codes: token gid, word tid4
-  const uint32_t v_lane = Cf::PK + (2 * tid4) * Cf::PITCH + (gid & 3) * 4;     // V codes: token 2*tid4, word gid%4
-  const uint32_t ksz_lane = 2 * Cf::PK + gid * (NG * 2);                       // K scale row of token gid
-  const uint32_t vsz_lane = 2 * Cf::PK + 2 * Cf::SZ + (2 * tid4) * (NG * 2);   // V scale rows of tokens 2*tid4, +1
-  const uint32_t bsel0 = gid >> 2, bsel1 = 2 + (gid >> 2);  // byte of the word used for M-tile half 0 / 1
-  const uint32_t sel0 = bsel0 | (bsel0 << 4) | ((4 + bsel0) << 8) | ((4 + bsel0) << 12);
-  const uint32_t sel1 = bsel1 | (bsel1 << 4) | ((4 + bsel1) << 8) | ((4 + bsel1) << 12);
+  // ldmatrix row addresses (offsets in a stage) for the scale / zero fragments, see block_step
+  const uint32_t ksz_lane = 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32;
+  const uint32_t vsz_lane = 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16;
 
 #pragma unroll
   for (int s = 0; s < Cf::NST - 1; ++s) {
@@ -227,132 +396,30 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     cp_async_commit();
   }
 
-  int stage = 0;                    // stage consumed in this iteration
-  int fill = Cf::NST - 1;           // stage filled in this iteration
+  // The block that holds the end of the sequence (if this warp owns it) is partial and goes
+  // through the masking variant of the step; every other block through the plain one.
+  const int rem_last = t1 - (blk0 + warp + (nblk - 1) * kWarps) * kBlk;  // tokens in this warp's last block
+  const int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;
+  WarpCtx<D> cx;
+  cx.ring = ring; cx.ksz_lane = ksz_lane; cx.vsz_lane = vsz_lane; cx.cs = cs; cx.gid = gid;
+#pragma unroll
+  for (int i = 0; i < NG / 2; ++i) {
+    const int j = 4 * i + (lane >> 3);
+    const int ktok = (lane & 7) + 8 * (j / NG), kgrp = j % NG;
+    cx.kaddr[i] = ktok * Cf::ROWB + ((kgrp ^ Cf::swz(ktok)) << 4);
+    const int vtok = (lane & 7) + 8 * (j % 2), vgrp = j / 2;
+    cx.vaddr[i] = Cf::PK + vtok * Cf::ROWB + ((vgrp ^ Cf::swz(vtok)) << 4);
+  }
   for (int k = 0; k < nblk; ++k) {
     cp_async_wait<Cf::NST - 2>();
     __syncwarp();
-    if (k + Cf::NST - 1 < nblk) ld.issue(ring_s + fill * Cf::STAGE);
+    if (k + Cf::NST - 1 < nblk) ld.issue(ring_s + ((k + Cf::NST - 1) & (Cf::NST - 1)) * Cf::STAGE);
     cp_async_commit();
-    fill = fill + 1 == Cf::NST ? 0 : fill + 1;
-    const uint8_t* st = ring + stage * Cf::STAGE;
-    stage = stage + 1 == Cf::NST ? 0 : stage + 1;
-    const int valid = t1 - (blk0 + warp + k * kWarps) * kBlk;  // >= 16 except in the block holding the sequence end
-    const bool tail = valid < kBlk;
-    if (tail) {
-      // rows past the end hold unspecified bytes: give them scale = zero = 0 so they dequantise to 0
-      __half* sz = reinterpret_cast<__half*>(const_cast<uint8_t*>(st) + 2 * Cf::PK);
-      for (int i = lane; i < 4 * kBlk * NG; i += 32) {
-        const int tok = (i / NG) % kBlk;
-        if (tok >= valid) sz[i] = __ushort_as_half(0);
-      }
-      __syncwarp();
-    }
-
-    // ---------------- scores: S[token][head] over this block's 16 tokens
-    float sc[4] = {0.f, 0.f, 0.f, 0.f};
-    {
-      const uint8_t* kp = st + k_lane;
-      // scales and zeros of tokens gid and gid + 8, all groups
-      __half2 ks_lo[NG / 2], kz_lo[NG / 2], ks_hi[NG / 2], kz_hi[NG / 2];
-      {
-        const uint32_t* r = reinterpret_cast<const uint32_t*>(st + ksz_lane);
-#pragma unroll
-        for (int i = 0; i < NG / 2; ++i) {
-          ks_lo[i] = u32_as_h2(r[i]);
-          kz_lo[i] = u32_as_h2(r[Cf::SZ / 4 + i]);
-          ks_hi[i] = u32_as_h2(r[8 * NG / 2 + i]);
-          kz_hi[i] = u32_as_h2(r[Cf::SZ / 4 + 8 * NG / 2 + i]);
-        }
-      }
-#pragma unroll
-      for (int g = 0; g < NG; ++g) {
-        const uint32_t w0 = *reinterpret_cast<const uint32_t*>(kp + g * 16);
-        const uint32_t w8 = *reinterpret_cast<const uint32_t*>(kp + 8 * Cf::PITCH + g * 16);
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        mma16816(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1]);
-        const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
-        mma16816(acc, y0 & kMaskLo, y8 & kMaskLo, y0 & kMaskHi, y8 & kMaskHi, qf[g][2], qf[g][3]);
-        const float s_lo = (g & 1) ? __high2float(ks_lo[g >> 1]) : __low2float(ks_lo[g >> 1]);
-        const float z_lo = (g & 1) ? __high2float(kz_lo[g >> 1]) : __low2float(kz_lo[g >> 1]);
-        const float s_hi = (g & 1) ? __high2float(ks_hi[g >> 1]) : __low2float(ks_hi[g >> 1]);
-        const float z_hi = (g & 1) ? __high2float(kz_hi[g >> 1]) : __low2float(kz_hi[g >> 1]);
-        sc[0] = fmaf(s_lo, fmaf(-z_lo, qs[g][0], acc[0]), sc[0]);
-        sc[1] = fmaf(s_lo, fmaf(-z_lo, qs[g][1], acc[1]), sc[1]);
-        sc[2] = fmaf(s_hi, fmaf(-z_hi, qs[g][0], acc[2]), sc[2]);
-        sc[3] = fmaf(s_hi, fmaf(-z_hi, qs[g][1], acc[3]), sc[3]);
-      }
-    }
-    // ---------------- online softmax (log2 domain)
-    float a0 = sc[0] * cs, a1 = sc[1] * cs, a2 = sc[2] * cs, a3 = sc[3] * cs;
-    if (tail) {
-      if (gid >= valid) a0 = a1 = -INFINITY;
-      if (gid + 8 >= valid) a2 = a3 = -INFINITY;
-    }
-    float bm0 = fmaxf(a0, a2), bm1 = fmaxf(a1, a3);
-    const bool need = (bm0 > m0 + kRescaleThreshold) || (bm1 > m1 + kRescaleThreshold);
-    if (__any_sync(0xffffffffu, need)) {
-#pragma unroll
-      for (int off = 4; off <= 16; off <<= 1) {
-        bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, off));
-        bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, off));
-      }
-      const float n0 = fmaxf(m0, bm0), n1 = fmaxf(m1, bm1);  // finite: every block has a valid token
-      const float f0 = ex2(m0 - n0), f1 = ex2(m1 - n1);      // ex2(-inf) = 0 on the first block
-      m0 = n0;
-      m1 = n1;
-      l0 *= f0;
-      l1 *= f1;
-#pragma unroll
-      for (int i = 0; i < D / 16; ++i) {
-        oacc[i][0] *= f0; oacc[i][1] *= f1; oacc[i][2] *= f0; oacc[i][3] *= f1;
-      }
-#pragma unroll
-      for (int g = 0; g < NG; ++g) {
-        zacc[g][0] *= f0; zacc[g][1] *= f1; zacc[g][2] *= f0; zacc[g][3] *= f1;
-      }
-    }
-    const float p0 = ex2(a0 - m0), p1 = ex2(a1 - m1), p2 = ex2(a2 - m0), p3 = ex2(a3 - m1);  // ex2(-inf) = 0
-    l0 += p0 + p2;
-    l1 += p1 + p3;
-    // P^T as B fragments: (tokens 2*tid4, 2*tid4+1 | head gid) and (tokens 8+2*tid4, 9+2*tid4 | head gid)
-    const uint32_t pt0 = movmatrix_trans(h2_as_u32(__floats2half2_rn(p0, p1)));
-    const uint32_t pt1 = movmatrix_trans(h2_as_u32(__floats2half2_rn(p2, p3)));
-
-    // ---------------- P.V: O^T[channel][head] += V^T[channel][token] * (P * s)[token][head]
-    {
-      const uint8_t* vp = st + v_lane;
-      // scales / zeros of tokens (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9): NG halves per token
-      uint32_t sAB[NG], sCD[NG], zAB[NG], zCD[NG];  // [0, NG/2) first token, [NG/2, NG) second token
-      {
-        const uint32_t* r = reinterpret_cast<const uint32_t*>(st + vsz_lane);
-#pragma unroll
-        for (int i = 0; i < NG; ++i) {
-          sAB[i] = r[i];
-          sCD[i] = r[8 * NG / 2 + i];
-          zAB[i] = r[Cf::SZ / 4 + i];
-          zCD[i] = r[Cf::SZ / 4 + 8 * NG / 2 + i];
-        }
-      }
-#pragma unroll
-      for (int g = 0; g < NG; ++g) {
-        const uint32_t psel = (g & 1) ? 0x7632u : 0x5410u;
-        const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(__byte_perm(sAB[g >> 1], sAB[NG / 2 + (g >> 1)], psel))));
-        const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(__byte_perm(sCD[g >> 1], sCD[NG / 2 + (g >> 1)], psel))));
-        const uint32_t zab = __byte_perm(zAB[g >> 1], zAB[NG / 2 + (g >> 1)], psel);
-        const uint32_t zcd = __byte_perm(zCD[g >> 1], zCD[NG / 2 + (g >> 1)], psel);
-        mma16816(zacc[g], zab, zab, zcd, zcd, b0, b1);
-        const uint32_t wA = *reinterpret_cast<const uint32_t*>(vp + g * 16);
-        const uint32_t wB = *reinterpret_cast<const uint32_t*>(vp + Cf::PITCH + g * 16);
-        const uint32_t wC = *reinterpret_cast<const uint32_t*>(vp + 8 * Cf::PITCH + g * 16);
-        const uint32_t wD = *reinterpret_cast<const uint32_t*>(vp + 9 * Cf::PITCH + g * 16);
-        uint32_t u = __byte_perm(wA, wB, sel0), u2 = __byte_perm(wC, wD, sel0);
-        mma16816(oacc[2 * g], u & kMaskLo, u & kMaskHi, u2 & kMaskLo, u2 & kMaskHi, b0, b1);
-        u = __byte_perm(wA, wB, sel1);
-        u2 = __byte_perm(wC, wD, sel1);
-        mma16816(oacc[2 * g + 1], u & kMaskLo, u & kMaskHi, u2 & kMaskLo, u2 & kMaskHi, b0, b1);
-      }
-    }
+    const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
+    if (k < nfull)
+      block_step<D, false>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, kBlk, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
+    else
+      block_step<D, true>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, rem_last, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
   }
   cp_async_wait<0>();
 
@@ -367,7 +434,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #pragma unroll
   for (int mt = 0; mt < D / 16; ++mt) {
     const int g = mt >> 1;
-    const int ch = 32 * g + 8 * (gid & 3) + 2 * (2 * (mt & 1) + (gid >> 2));
+    const int ch = 32 * g + 4 * gid + 2 * (mt & 1);
     // even channel: codes carried 2^-24; odd channel (high nibble): 2^-20
     *reinterpret_cast<float2*>(mo + ch * 8 + 2 * tid4) =
         make_float2(oacc[mt][0] * 16777216.0f - zacc[g][0], oacc[mt][1] * 16777216.0f - zacc[g][1]);
@@ -389,19 +456,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) M = fmaxf(M, all[w * (8 * D + 16) + 8 * D + h]);
     float num = 0.f, den = 0.f;
-    if (M > -INFINITY) {
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        const float* wb = all + w * (8 * D + 16);
-        const float f = ex2(wb[8 * D + h] - M);  // ex2(-inf) = 0 for a warp that saw no token
-        num = fmaf(f, wb[idx], num);
-        den = fmaf(f, wb[8 * D + 8 + h], den);
-      }
+    for (int w = 0; w < kWarps; ++w) {
+      const float* wb = all + w * (8 * D + 16);
+      const float f = ex2(wb[8 * D + h] - M);  // underflows to 0 for a warp that saw no token (m = -1e30)
+      num = fmaf(f, wb[idx], num);
+      den = fmaf(f, wb[8 * D + 8 + h], den);     // l = 0 there as well
     }
     const long long pidx = (static_cast<long long>(b) * H_q + h0 + h) * C + c;
     o_part[pidx * D + x] = den > 0.f ? num / den : 0.f;
     if (x == 0) {
-      m_part[pidx] = M * kLn2;  // natural-log units of attn_scale * q.k^
+      m_part[pidx] = den > 0.f ? M * kLn2 : -INFINITY;  // natural-log units of attn_scale * q.k^
       l_part[pidx] = den;
     }
   }

@@ -22,6 +22,13 @@ __host__ __device__ inline void split_range(int len, int C, int c, int& t0, int&
   if (t1 < t0) t1 = t0;
 }
 
+// Element index of (sequence*head bh, token tok, group g) in a scale or zero array.  Those arrays
+// are blocked by 16 tokens: [B * H_kv][S_cap / 16][d / 32][16], so that the 16 tokens of one
+// group are contiguous (what the decode kernel's fragment loads want).
+__host__ __device__ inline long long scale_index(long long bh, int S_cap, int NG, int tok, int g) {
+  return ((bh * (S_cap >> 4) + (tok >> 4)) * NG + g) * 16 + (tok & 15);
+}
+
 // Clamp a device-side sequence length into [0, S_cap], flagging bad or empty values.
 __device__ inline int checked_len(const int32_t* seq_lens, int b, int S_cap, int32_t* status) {
   int len = seq_lens[b];

@@ -89,12 +89,14 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
   if (in_range) {
     const long long bh = row_in / T;
     const int t = static_cast<int>(row_in - bh * T);
-    const long long row_out = bh * c.S_cap + len + t;
+    const int tok = len + t;
+    const long long row_out = bh * c.S_cap + tok;
     (void)b;
     reinterpret_cast<uint32_t*>(dst.packed + row_out * (d >> 1))[cc] = word;
     if ((cc & 3) == 0) {
-      dst.scale[row_out * (d >> 5) + (cc >> 2)] = s;
-      dst.zero[row_out * (d >> 5) + (cc >> 2)] = z;
+      const long long si = scale_index(bh, c.S_cap, d >> 5, tok, cc >> 2);
+      dst.scale[si] = s;
+      dst.zero[si] = z;
     }
   }
 }

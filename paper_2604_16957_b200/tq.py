@@ -93,14 +93,25 @@ class KVCache:
         f16 = dict(dtype=torch.float16, device=device)
         self.k_packed = torch.zeros((B, H_kv, S_cap, d // 2), **u8)
         self.v_packed = torch.zeros((B, H_kv, S_cap, d // 2), **u8)
-        self.k_scale = torch.zeros((B, H_kv, S_cap, g), **f16)
-        self.k_zero = torch.zeros((B, H_kv, S_cap, g), **f16)
-        self.v_scale = torch.zeros((B, H_kv, S_cap, g), **f16)
-        self.v_zero = torch.zeros((B, H_kv, S_cap, g), **f16)
+        assert S_cap % 16 == 0
+        # scale / zero arrays are blocked by 16 tokens: [B][H_kv][S_cap/16][d/32][16]
+        self.k_scale = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
+        self.k_zero = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
+        self.v_scale = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
+        self.v_zero = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
         self.seq_lens = torch.zeros((B,), dtype=torch.int32, device=device)
 
     def arrays(self):
         return (self.k_packed, self.k_scale, self.k_zero, self.v_packed, self.v_scale, self.v_zero)
+
+    def token_major(self, a):
+        """View of a scale / zero array in token-major order [B][H_kv][S_cap][d/32] (a copy)."""
+        return a.permute(0, 1, 2, 4, 3).reshape(self.B, self.H_kv, self.S_cap, self.d // TQ_GROUP)
+
+    def arrays_token_major(self):
+        """All six arrays with scales and zeros re-ordered to [B][H_kv][S_cap][d/32]."""
+        return (self.k_packed, self.token_major(self.k_scale), self.token_major(self.k_zero), self.v_packed,
+                self.token_major(self.v_scale), self.token_major(self.v_zero))
 
     def struct(self):
         return tq_kv_cache(self.k_packed.data_ptr(), self.v_packed.data_ptr(), self.k_scale.data_ptr(),

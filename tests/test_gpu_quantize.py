@@ -70,7 +70,7 @@ def test_decode_step_appends_and_overflow(gpu, oracle):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     for step, T in enumerate([1, 3, 1, 1]):
         k, v = I.make_kv(shape, T, 7, stream=step + 1)
-        before = [a.clone() for a in dev.arrays()]
+        before = [a.clone() for a in dev.arrays_token_major()]
         lens_before = dev.seq_lens.cpu().numpy().copy()
         skipped = host.append(k, v)
         tq.tq_kv_quantize_append(dev, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
@@ -79,7 +79,7 @@ def test_decode_step_appends_and_overflow(gpu, oracle):
         assert_cache_bits_equal(dev, host)
         assert (int(status.item()) & tq.TQ_STATUS_CACHE_FULL != 0) == (skipped > 0 or step > 1)
         # rows outside [len, len + T) of every sequence are untouched
-        for a, a0 in zip(dev.arrays(), before):
+        for a, a0 in zip(dev.arrays_token_major(), before):
             an, a0n = a.cpu().numpy(), a0.cpu().numpy()
             for b in range(shape.B):
                 lo = int(lens_before[b])
@@ -106,5 +106,5 @@ def test_bulk_path_with_ragged_lengths_and_overflow(gpu, oracle):
     assert dev.seq_lens.cpu().tolist() == [1500, 2500, 3000]
     # compare only rows that were ever written on both sides
     assert_cache_bits_equal(dev, host, lens=[1500, 0, 0])
-    for name, d_arr, h_arr in zip("abcdef", dev.arrays(), host.arrays()):
+    for name, d_arr, h_arr in zip("abcdef", dev.arrays_token_major(), host.arrays()):
         assert np.array_equal(d_arr.cpu().numpy()[1, :, 1000:2500].view(np.uint8), h_arr[1, :, 1000:2500].view(np.uint8))

@@ -50,7 +50,7 @@ def assert_cache_bits_equal(dev_cache, host_cache, lens=None):
     B = host_cache.B
     lens = host_cache.lens if lens is None else lens
     for name, d_arr, h_arr in zip(("k_packed", "k_scale", "k_zero", "v_packed", "v_scale", "v_zero"),
-                                  dev_cache.arrays(), host_cache.arrays()):
+                                  dev_cache.arrays_token_major(), host_cache.arrays()):
         d_np = d_arr.cpu().numpy()
         for b in range(B):
             n = int(lens[b])
