@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=LAYERS)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-compare", action="store_true", help="skip the dequantize-then-attend timing")
+    ap.add_argument("--splits", type=int, default=0, help="sequence splits C of the fused kernel (0 = library default)")
     return ap.parse_args()
 
 
@@ -181,7 +182,7 @@ def main():
     L, S = args.layers, args.context
     total_appends = 2 * (args.warmup + args.steps) + 8
     S_cap = (S + total_appends + 15) // 16 * 16
-    C = tq.tq_auto_splits(1, H_KV, H_Q, D, S)
+    C = args.splits or tq.tq_auto_splits(1, H_KV, H_Q, D, S)
 
     # ---- resident state: L quantised layer caches, filled from seeded device-side normals.
     # K gets 4 seeded outlier channels x10 per KV head, like the parity-test generator.

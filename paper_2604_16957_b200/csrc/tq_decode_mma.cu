@@ -63,8 +63,8 @@ struct Cfg {
   static constexpr int NST = 4;                     // stages in the per-warp ring (power of two)
   static constexpr int MINB = D == 256 ? 1 : 2;     // resident blocks per SM
   static constexpr int PIPE = kWarps * NST * STAGE; // 40 KB (D = 64), 80 KB (128), 160 KB (256)
-  static constexpr int MERGE = kWarps * (8 * D + 16) * 4;
-  static constexpr int SMEM = (PIPE > MERGE ? PIPE : MERGE) + 8 * NG * 4;
+  static constexpr int MERGE = (kWarps * 16 + kWarps * D * 10 + 8 * (D + 4)) * 4;
+  static constexpr int SMEM = PIPE > MERGE ? PIPE : MERGE;
   // loader geometry
   static constexpr int PASS_TOK = 32 / NG;          // token rows covered by one warp-wide pass of 16-byte chunks
   static constexpr int CODE_PASSES = kBlk / PASS_TOK;
@@ -283,23 +283,21 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
     for (int g = 0; g < NG; ++g) {
       // Scales / zeros of token pairs (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9) of group g: an ldmatrix
       // whose eight row addresses are equal hands every lane word tid4 of that 16-byte chunk; the four
-      // matrices are (scale | tokens 0-7), (scale | 8-15), (zero | 0-7), (zero | 8-15).
+      // matrices are (zero | tokens 0-7), (scale | 0-7), (zero | 8-15), (scale | 8-15).  In that order the
+      // four result registers are, as they stand, the A operand of the zero-point MMA: rows 0-7 hold z_g
+      // (c0, c1 accumulate sum_tok z_g * B_g), rows 8-15 hold the scales and produce values never read.
       uint32_t vsz[4];
       ldmatrix_x4(vsz, st_s + cx.vsz_lane + 32 * g);
-      const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vsz[0])));
-      const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vsz[1])));
-      const uint32_t zab = vsz[2], zcd = vsz[3];
+      const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vsz[1])));
+      const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vsz[3])));
+      mma16816(zacc[g], vsz[0], vsz[1], vsz[2], vsz[3], b0, b1);
       // r1 = (tokens 2*tid4, 2*tid4+1), r2 = (tokens 2*tid4+8, +9): 16-bit lane gid of chunk g, i.e. codes of
       // channels 32g + 4*gid .. +3 of two tokens side by side
       if ((g & 1) == 0) ldmatrix_x4_trans(vw, st_s + cx.vaddr[g / 2]);
       const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
       mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
       const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
-      const uint32_t uh = y1 & kMaskHi, u2h = y2 & kMaskHi;
-      mma16816(oacc[2 * g + 1], y1 & kMaskLo, uh, y2 & kMaskLo, u2h, b0, b1);
-      // zero-point term: rows 0-7 of A hold z_g (so c0, c1 accumulate sum_tok z_g * B_g); rows 8-15 reuse
-      // the operand registers of the MMA above and produce values that are never read
-      mma16816(zacc[g], zab, uh, zcd, u2h, b0, b1);
+      mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1 & kMaskHi, y2 & kMaskLo, y2 & kMaskHi, b0, b1);
     }
   }
 }
@@ -312,7 +310,6 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   using Cf = Cfg<D>;
   constexpr int NG = Cf::NG;
   extern __shared__ __align__(128) uint8_t smem[];
-  float* sm_qs = reinterpret_cast<float*>(smem + (Cf::SMEM - 8 * NG * 4));  // [8 heads][NG] group sums of q
 
   const int G = H_q / cache.H_kv;
   const int tiles = (G + 7) >> 3;
@@ -324,43 +321,13 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   int t0, t1;
   split_range(len, C, c, t0, t1);
 
-  // ---- group sums of q (for the zero-point term), scaled by 2^-24 like the code operands
-  {
-    const int pair = threadIdx.x >> 2, part = threadIdx.x & 3;  // pair = head * NG + group
-    float s = 0.f;
-    if (pair < 8 * NG) {
-      const int h = pair / NG, g = pair - h * NG;
-      if (h < nh) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(q + (static_cast<long long>(b) * H_q + h0 + h) * D + g * 32 + part * 8);
-        const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 f = __half22float2(h2[i]);
-          s += f.x + f.y;
-        }
-      }
-    }
-    s += __shfl_xor_sync(0xffffffffu, s, 1);
-    s += __shfl_xor_sync(0xffffffffu, s, 2);
-    if (pair < 8 * NG && part == 0) sm_qs[pair] = s * 5.9604644775390625e-8f;  // 2^-24
-  }
-  __syncthreads();
-
-  // ---- q as MMA B fragments: column n = gid is head h0 + gid; k slots follow the nibble order
-  uint32_t qf[NG][4];
-  float qs[NG][2];
+  // ---- q first (a handful of loads that must not queue behind the cache stream), used further down
+  uint4 qraw[NG];
 #pragma unroll
   for (int g = 0; g < NG; ++g) {
-    uint4 raw = make_uint4(0, 0, 0, 0);
+    qraw[g] = make_uint4(0, 0, 0, 0);
     if (gid < nh)
-      raw = *reinterpret_cast<const uint4*>(q + (static_cast<long long>(b) * H_q + h0 + gid) * D + g * 32 + tid4 * 8);
-    const __half2 sixteenth = __float2half2_rn(0.0625f);
-    qf[g][0] = __byte_perm(raw.x, raw.z, 0x5410);                                            // (c0, c4)
-    qf[g][1] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(raw.x, raw.z, 0x7632)), sixteenth));  // (c1, c5) / 16
-    qf[g][2] = __byte_perm(raw.y, raw.w, 0x5410);                                            // (c2, c6)
-    qf[g][3] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(raw.y, raw.w, 0x7632)), sixteenth));  // (c3, c7) / 16
-    qs[g][0] = sm_qs[(2 * tid4) * NG + g];
-    qs[g][1] = sm_qs[(2 * tid4 + 1) * NG + g];
+      qraw[g] = *reinterpret_cast<const uint4*>(q + (static_cast<long long>(b) * H_q + h0 + gid) * D + g * 32 + tid4 * 8);
   }
 
   // ---- this warp's token blocks: blk0 + warp, blk0 + warp + kWarps, ...
@@ -372,6 +339,40 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
   uint8_t* const ring = smem + warp * (Cf::NST * Cf::STAGE);
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
+
+  // start streaming: the first stages are in flight while q is turned into fragments
+#pragma unroll
+  for (int s = 0; s < Cf::NST - 1; ++s) {
+    if (s < nblk) ld.issue(ring_s + s * Cf::STAGE);
+    cp_async_commit();
+  }
+
+
+  // ---- q as MMA B fragments: column n = gid is head h0 + gid; k slots follow the nibble order.
+  // qs[g][j] = 2^-24 * sum of q over group g for heads 2*tid4 + j (the zero-point term of the scores).
+  uint32_t qf[NG][4];
+  float qs[NG][2];
+#pragma unroll
+  for (int g = 0; g < NG; ++g) {
+    const uint4 raw = qraw[g];
+    const __half2 sixteenth = __float2half2_rn(0.0625f);
+    qf[g][0] = __byte_perm(raw.x, raw.z, 0x5410);                                            // (c0, c4)
+    qf[g][1] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(raw.x, raw.z, 0x7632)), sixteenth));  // (c1, c5) / 16
+    qf[g][2] = __byte_perm(raw.y, raw.w, 0x5410);                                            // (c2, c6)
+    qf[g][3] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(raw.y, raw.w, 0x7632)), sixteenth));  // (c3, c7) / 16
+    const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(h2[i]);
+      sum += f.x + f.y;
+    }
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 2);  // every lane of quad gid: sum over group g of head gid
+    sum *= 5.9604644775390625e-8f;                // 2^-24, like the code operands
+    qs[g][0] = __shfl_sync(0xffffffffu, sum, (2 * tid4) * 4);
+    qs[g][1] = __shfl_sync(0xffffffffu, sum, (2 * tid4 + 1) * 4);
+  }
 
   float oacc[D / 16][4];  // [M tile][c0..c3]: rows = channels, cols = heads 2*tid4, 2*tid4+1
   float zacc[NG][4];      // sum_tok B_g * z_g: [0], [1] are heads 2*tid4, 2*tid4+1; [2], [3] are not used
@@ -388,13 +389,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // per-lane byte offsets inside a stage (everything else is a compile-time offset from these)
   // ldmatrix row addresses (offsets in a stage) for the scale / zero fragments, see block_step
   const uint32_t ksz_lane = 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32;
-  const uint32_t vsz_lane = 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16;
-
-#pragma unroll
-  for (int s = 0; s < Cf::NST - 1; ++s) {
-    if (s < nblk) ld.issue(ring_s + s * Cf::STAGE);
-    cp_async_commit();
-  }
+  const uint32_t vsz_lane = 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16;
 
   // The block that holds the end of the sequence (if this warp owns it) is partial and goes
   // through the masking variant of the step; every other block through the plain one.
@@ -423,51 +418,76 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   cp_async_wait<0>();
 
-  // ---------------- per-warp result -> shared, merge the warps, write the normalised partial
+  // ---------------- merge the warps and write the normalised partial (o_c, m_c, l_c)
 #pragma unroll
   for (int off = 4; off <= 16; off <<= 1) {
     l0 += __shfl_xor_sync(0xffffffffu, l0, off);
     l1 += __shfl_xor_sync(0xffffffffu, l1, off);
   }
   __syncthreads();  // every warp is done with its ring; the memory is reused below
-  float* mo = reinterpret_cast<float*>(smem) + warp * (8 * D + 16);  // [D channels][8 heads] then m[8], l[8]
+  // layout (floats): wml[kWarps][16] = each warp's m[8], l[8] | slab[kWarps][D][kChPitch] | tb[8][kRowPitch]
+  constexpr int kChPitch = 10;       // 8 heads per channel row, padded: the float2 fragment stores are conflict free
+  constexpr int kRowPitch = D + 4;   // transposed [head][channel] tile, conflict free for the writes below
+  float* const wml = reinterpret_cast<float*>(smem);
+  float* const slab = wml + kWarps * 16;
+  float* const tb = slab + kWarps * D * kChPitch;
+  if (gid == 0) {
+    wml[warp * 16 + 2 * tid4] = m0;
+    wml[warp * 16 + 2 * tid4 + 1] = m1;
+    wml[warp * 16 + 8 + 2 * tid4] = l0;
+    wml[warp * 16 + 8 + 2 * tid4 + 1] = l1;
+  }
+  __syncthreads();
+  // every thread: unit-wide reference M, denominator and this warp's weight for its two heads
+  float M0 = kNoMax, M1 = kNoMax;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {
+    M0 = fmaxf(M0, wml[w * 16 + 2 * tid4]);
+    M1 = fmaxf(M1, wml[w * 16 + 2 * tid4 + 1]);
+  }
+  float den0 = 0.f, den1 = 0.f;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {  // a warp that saw no token has m = -1e30 and l = 0
+    den0 = fmaf(ex2(wml[w * 16 + 2 * tid4] - M0), wml[w * 16 + 8 + 2 * tid4], den0);
+    den1 = fmaf(ex2(wml[w * 16 + 2 * tid4 + 1] - M1), wml[w * 16 + 8 + 2 * tid4 + 1], den1);
+  }
+  const float f0 = den0 > 0.f ? ex2(m0 - M0) / den0 : 0.f;
+  const float f1 = den1 > 0.f ? ex2(m1 - M1) / den1 : 0.f;
+  float* const mo = slab + warp * D * kChPitch;
 #pragma unroll
   for (int mt = 0; mt < D / 16; ++mt) {
     const int g = mt >> 1;
     const int ch = 32 * g + 4 * gid + 2 * (mt & 1);
     // even channel: codes carried 2^-24; odd channel (high nibble): 2^-20
-    *reinterpret_cast<float2*>(mo + ch * 8 + 2 * tid4) =
-        make_float2(oacc[mt][0] * 16777216.0f - zacc[g][0], oacc[mt][1] * 16777216.0f - zacc[g][1]);
-    *reinterpret_cast<float2*>(mo + (ch + 1) * 8 + 2 * tid4) =
-        make_float2(oacc[mt][2] * 1048576.0f - zacc[g][0], oacc[mt][3] * 1048576.0f - zacc[g][1]);
-  }
-  if (gid == 0) {
-    mo[8 * D + 2 * tid4] = m0;
-    mo[8 * D + 2 * tid4 + 1] = m1;
-    mo[8 * D + 8 + 2 * tid4] = l0;
-    mo[8 * D + 8 + 2 * tid4 + 1] = l1;
+    *reinterpret_cast<float2*>(mo + ch * kChPitch + 2 * tid4) =
+        make_float2((oacc[mt][0] * 16777216.0f - zacc[g][0]) * f0, (oacc[mt][1] * 16777216.0f - zacc[g][1]) * f1);
+    *reinterpret_cast<float2*>(mo + (ch + 1) * kChPitch + 2 * tid4) =
+        make_float2((oacc[mt][2] * 1048576.0f - zacc[g][0]) * f0, (oacc[mt][3] * 1048576.0f - zacc[g][1]) * f1);
   }
   __syncthreads();
-  const float* all = reinterpret_cast<const float*>(smem);
   for (int idx = threadIdx.x; idx < 8 * D; idx += kThreads) {
     const int x = idx >> 3, h = idx & 7;  // consecutive threads take consecutive heads of one channel
-    if (h >= nh) continue;
-    float M = -INFINITY;
+    float sum = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, all[w * (8 * D + 16) + 8 * D + h]);
-    float num = 0.f, den = 0.f;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-      const float* wb = all + w * (8 * D + 16);
-      const float f = ex2(wb[8 * D + h] - M);  // underflows to 0 for a warp that saw no token (m = -1e30)
-      num = fmaf(f, wb[idx], num);
-      den = fmaf(f, wb[8 * D + 8 + h], den);     // l = 0 there as well
-    }
+    for (int w = 0; w < kWarps; ++w) sum += slab[(w * D + x) * kChPitch + h];
+    tb[h * kRowPitch + x] = sum;
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < nh * D; idx += kThreads) {  // coalesced: one head row after the other
+    const int h = idx / D, x = idx - h * D;
     const long long pidx = (static_cast<long long>(b) * H_q + h0 + h) * C + c;
-    o_part[pidx * D + x] = den > 0.f ? num / den : 0.f;
-    if (x == 0) {
-      m_part[pidx] = den > 0.f ? M * kLn2 : -INFINITY;  // natural-log units of attn_scale * q.k^
-      l_part[pidx] = den;
+    o_part[pidx * D + x] = tb[h * kRowPitch + x];
+  }
+  if (warp == 0 && gid == 0) {  // lanes 0..3 hold heads 2*tid4, 2*tid4+1
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int h = 2 * tid4 + j;
+      if (h < nh) {
+        const float den = j ? den1 : den0, M = j ? M1 : M0;
+        const long long pidx = (static_cast<long long>(b) * H_q + h0 + h) * C + c;
+        m_part[pidx] = den > 0.f ? M * kLn2 : -INFINITY;  // natural-log units of attn_scale * q.k^
+        l_part[pidx] = den;
+      }
     }
   }
 }
