@@ -160,6 +160,22 @@ def config_dict(args):
             "l2": "inputs larger than L2: every layer's cache (168 MB at 128K) is a distinct buffer, 13.4 GB in all"}
 
 
+def max_over_ranks(seconds, world, device):
+    """Replicas only: every rank times its own replica; the job's time is the slowest rank's."""
+    if world <= 1:
+        return seconds
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([seconds], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_us_per_layer(seconds_for_steps, steps, layers, world):
+    """N independent replicas complete N * layers layer-steps per step in the time of the slowest."""
+    return seconds_for_steps / steps / layers / world * 1e6
+
+
 # ------------------------------------------------------------------ GPU arm
 def main():
     args = parse_args()
@@ -258,12 +274,7 @@ def main():
             if post: post()
         e1.record()
         barrier()
-        t = e0.elapsed_time(e1) / 1e3
-        if world > 1:
-            tt = torch.tensor([t], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            t = float(tt.item())
-        return t
+        return max_over_ranks(e0.elapsed_time(e1) / 1e3, world, dev)
 
     g_step = make_graph()
     g_decode = make_graph(append=False, combine=False)
@@ -273,7 +284,7 @@ def main():
     W, K = args.warmup, args.steps
     with ClockSampler(local_rank) as clocks:
         t_step = time_graph(g_step, W, K)
-    us_per_layer = t_step / K / L * 1e6
+    us_per_layer = job_us_per_layer(t_step, K, L, 1)
 
     # per-kernel figures (same graph-replay timing, decode launches back to back over the L distinct layers)
     t_decode = time_graph(g_decode, W, K)
@@ -300,11 +311,11 @@ def main():
     alg_bytes = H_KV * S * BYTES_PER_TOKEN_HEAD
     achieved = alg_bytes / (decode_us * 1e-6) / 1e9
     roofline = {"bound": "hbm", "kernel": "decode_mma_kernel<128>", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_src, "traffic": ncu_traffic_bytes(),
+                "frac": achieved / peak, "peak_source": peak_src, "traffic": ncu_traffic_bytes() if S == CONTEXT else None,
                 "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": decode_us,
                 "frac_of_nominal_8TBs": achieved / HBM_NOMINAL_GBS}
 
-    line = {"metric": "int4 decode-attn us/layer @128K (Llama-70B shape)", "value": us_per_layer / world,
+    line = {"metric": "int4 decode-attn us/layer @128K (Llama-70B shape)", "value": job_us_per_layer(t_step, K, L, world),
             "unit": "us/layer", "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": t_step / K * 1e3,
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f16 codes->f32 accum",
             "data": "synthetic", "config": config_dict(args), "clocks": clocks.summary(),
@@ -331,11 +342,13 @@ def main():
 
 
 def ncu_traffic_bytes():
-    """DRAM bytes (read + write) of one fused-decode launch from the committed ncu summary, if any."""
-    path = os.path.join(ROOT, "profiles", "decode_mma_llama128k_traffic.json")
+    """DRAM bytes (read + write) of one fused-decode launch, from the committed ncu summary."""
+    import re
+    path = os.path.join(ROOT, "profiles", "decode_mma_llama128k.md")
     try:
         with open(path) as f:
-            return json.load(f)["dram_bytes_per_launch"]
+            m = re.search(r"^dram_bytes_per_launch:\s*(\d+)", f.read(), re.M)
+        return int(m.group(1)) if m else None
     except Exception:
         return None
 
