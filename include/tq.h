@@ -156,6 +156,36 @@ int tq_sdpa_dequant_then_attend(const tq_kv_cache* cache /* host */, const void*
 size_t tq_dequant_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t S_cap, int32_t d,
                                   int32_t ws_is_fp32);
 
+/*
+ * Fused attention for callers that cannot allocate (the paper has no counterpart for this entry
+ * point; it exists for integration, not for the method).  Some hosts of this library may not call
+ * cudaMalloc at the point where attention runs: an inference server that hands all device memory
+ * to its own pool at start-up, code running while a stream is being captured into a CUDA graph
+ * (where an allocation is illegal), or a latency-critical decode loop where cudaMalloc / cudaFree
+ * would serialise the whole device.  They have nowhere to put the split partials that
+ * tq_sdpa_int4_decode writes and tq_sdpa_int4_combine reads.  This call runs both phases in one go
+ * and keeps the partials in a fixed TQ_STATIC_SCRATCH_BYTES array that is part of the library image
+ * (every GPU on which the library is used holds those bytes until the process exits).
+ *   Result: out[b][h][:] as tq_sdpa_int4_decode followed by tq_sdpa_int4_combine would give it
+ *   (the split count may differ, so agreement is to rounding, not bit for bit).
+ *   It calls no cudaMalloc / cudaFree nor any routine that allocates.  The caller still provides
+ *   q, the cache and out.
+ *   Limit: the partials of the chosen split count, B * H_q * C * (d + 2) * 4 bytes (plus padding),
+ *   must fit the array.  The split count is lowered as far as 1 to make them fit; if they still
+ *   do not, nothing is launched and TQ_ERR_WORKSPACE is returned.
+ *   First use on a device looks up the array's device address (with that device current; the
+ *   device of `stream` must be the current device).  Make that first call outside any stream
+ *   capture; later calls do no set-up.
+ *   All calls share the one array and it keeps the previous call's contents.  Nothing needs
+ *   clearing (every partial is rewritten by each call), but two calls whose kernels overlap on
+ *   the GPU -- different streams, or graphs launched concurrently -- race on it: serialise them.
+ * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_WORKSPACE (see Limit), TQ_ERR_CUDA.
+ * Status: as tq_sdpa_int4_decode.
+ */
+#define TQ_STATIC_SCRATCH_BYTES (8u << 20)
+int tq_sdpa_int4_attend_static(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
+                               void* out, int32_t out_is_fp32, int32_t* status, void* stream);
+
 /* Bytes of one layer's cache arrays (packed + scales + zeros, K and V), i.e. Eq. 1 with the int4 format. */
 size_t tq_cache_bytes(int32_t B, int32_t H_kv, int32_t S_cap, int32_t d);
 

@@ -21,11 +21,12 @@ _lib = C.CDLL(LIB_PATH)
 TQ_OK, TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_WORKSPACE, TQ_ERR_CUDA = range(6)
 TQ_STATUS_CACHE_FULL, TQ_STATUS_EMPTY_SEQ, TQ_STATUS_BAD_LEN = 1, 2, 4
 TQ_GROUP, TQ_SPLIT_QUANTUM, TQ_MAX_SPLITS = 32, 16, 256
+TQ_STATIC_SCRATCH_BYTES = 8 << 20
 
 # every symbol include/tq.h declares
 SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa_int4_decode", "tq_sdpa_int4_combine",
            "tq_partials_bytes", "tq_sdpa_dequant_then_attend", "tq_dequant_workspace_bytes", "tq_cache_bytes",
-           "tq_result_string", "tq_last_cuda_error", "tq_version")
+           "tq_result_string", "tq_last_cuda_error", "tq_version", "tq_sdpa_int4_attend_static")
 
 
 class tq_kv_cache(C.Structure):
@@ -52,6 +53,8 @@ _lib.tq_sdpa_dequant_then_attend.argtypes = [_cache_p, _vp, _i32, _f32, _vp, _sz
 _lib.tq_sdpa_dequant_then_attend.restype = C.c_int
 _lib.tq_dequant_workspace_bytes.argtypes = [_i32] * 6
 _lib.tq_dequant_workspace_bytes.restype = _sz
+_lib.tq_sdpa_int4_attend_static.argtypes = [_cache_p, _vp, _i32, _f32, _vp, _i32, _vp, _vp]
+_lib.tq_sdpa_int4_attend_static.restype = C.c_int
 _lib.tq_cache_bytes.argtypes = [_i32] * 4
 _lib.tq_cache_bytes.restype = _sz
 _lib.tq_result_string.argtypes = [C.c_int]
@@ -180,6 +183,18 @@ def tq_sdpa_dequant_then_attend(cache, q, attn_scale, workspace, ws_is_fp32, out
                                             workspace.numel(), int(ws_is_fp32), _ptr(out),
                                             int(out.dtype == torch.float32), _ptr(status), _stream(stream)),
            "tq_sdpa_dequant_then_attend")
+
+
+def tq_sdpa_int4_attend_static(cache, q, attn_scale, out, status=None, stream=None):
+    """Decode + combine in one call for callers that cannot allocate: the split partials live in a
+    fixed array inside the library instead of caller memory.  q: [B][H_q][d] float16; out: [B][H_q][d]
+    float16 or float32.  Raises TqError(TQ_ERR_WORKSPACE) when B * H_q * d is too large for that array."""
+    assert q.is_contiguous() and q.dtype == torch.float16 and q.dim() == 3
+    assert out.shape == q.shape and out.dtype in (torch.float16, torch.float32) and out.is_contiguous()
+    cs = _cs(cache)
+    _check(_lib.tq_sdpa_int4_attend_static(C.byref(cs), _ptr(q), q.shape[1], float(attn_scale), _ptr(out),
+                                           int(out.dtype == torch.float32), _ptr(status), _stream(stream)),
+           "tq_sdpa_int4_attend_static")
 
 
 def alloc_partials(B, H_q, d, num_splits, device="cuda"):
