@@ -109,17 +109,18 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ CPU oracle leg
-def oracle_sample_us_per_layer(context, repeats=1):
-    """Time the CPU oracle as it stands on a bounded sample of the workload: ONE of the 8 KV
-    heads (its 8 query heads) of one `context`-token layer, quantised by the oracle itself;
-    the time is scaled by 8 to a full layer.  Returns (us_per_layer, seconds list, threads)."""
+def oracle_sample_us_per_layer(context, repeats=1, kv_heads=1):
+    """Time the CPU oracle as it stands on a bounded sample of the workload: `kv_heads` of the 8 KV
+    heads (with their 8 query heads each) of one `context`-token layer, quantised by the oracle
+    itself; the time is scaled by 8 / kv_heads to a full layer.
+    Returns (us_per_layer list, seconds list, threads)."""
     import numpy as np
     from oracle import tq_oracle as O
     from paper_2604_16957_b200 import inputs as I
-    sh = I.Shape("llama-1kvhead", 1, H_Q // H_KV, 1, D, ALPHA, k_outlier_channels=4)
+    sh = I.Shape("llama-sample", 1, (H_Q // H_KV) * kv_heads, kv_heads, D, ALPHA, k_outlier_channels=4)
     k, v = I.make_kv(sh, context, seed=1000)
     q = I.make_q(sh, seed=1000)
-    cache = O.Cache(1, 1, context, D)
+    cache = O.Cache(1, kv_heads, context, D)
     cache.append(k, v)
     del k, v
     secs = []
@@ -128,7 +129,7 @@ def oracle_sample_us_per_layer(context, repeats=1):
         out = O.attention(cache, q, ALPHA)
         secs.append(time.perf_counter() - t)
     assert np.all(np.isfinite(out))
-    return [s * H_KV * 1e6 for s in secs], secs, O.num_threads()
+    return [s * (H_KV / kv_heads) * 1e6 for s in secs], secs, O.num_threads()
 
 
 def run_reference(args, rank):
@@ -332,10 +333,11 @@ def main():
     if not args.no_compare:
         line["dequant_then_attend_us_per_layer"] = time_dequant_then_attend(tq, torch, caches, q_l, out, S, S_cap, dev)
     if not args.no_cpu_baseline:
-        per, secs, threads = oracle_sample_us_per_layer(S, repeats=2)
+        per, secs, threads = oracle_sample_us_per_layer(S, repeats=2, kv_heads=H_KV)
         line["cpu_baseline"] = {"value": min(per), "unit": "us/layer", "cores": threads, "kind": "oracle",
-                                "sample": f"1 of {H_KV} KV heads ({H_Q // H_KV} of {H_Q} query heads) of one {S}-token "
-                                          f"layer, best of 2 runs ({min(secs):.2f} s), scaled x{H_KV} to a full layer"}
+                                "sample": f"one full {S}-token layer (all {H_Q} query heads, {H_KV} KV heads) of the "
+                                          f"{L}-layer step, oracle-quantised, best of 2 runs ({min(secs):.2f} s wall on "
+                                          f"{threads} threads)"}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

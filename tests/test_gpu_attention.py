@@ -244,3 +244,58 @@ def test_full_size_128k_llama_layer_in_bench_configuration(gpu, oracle):
     out, _, C = fused_attention(tq, torch, dev, q, I.LLAMA.alpha)
     mx, rel = assert_attention_close(out, ref, "llama/128K")
     print(f"llama 128K C={C}: max-abs {mx:.2e} rel-L2 {rel:.2e}")
+
+
+def test_config5_ragged_batch_64_decode_steps(gpu, oracle):
+    """Batched ragged decode: B = 16, Llama-70B head shapes, context lengths uniform in [4096, 65536],
+    64 consecutive steps of quantize-append followed by fused attention.  The shortest and the longest
+    sequence carry seeded data and are checked against the oracle at the first and the last step (cache
+    bit-exact, attention within tolerance); the other sequences hold zeros but have their drawn lengths,
+    so the launch has the real ragged work distribution."""
+    tq, torch = gpu
+    sh = I.RAGGED
+    lens = I.ragged_lengths(sh.B, 4096, 65536, seed=5)
+    S_cap = 65536 + 64
+    picked = [int(np.argmin(lens)), int(np.argmax(lens))]
+    one = I.Shape("ragged-1seq", 1, sh.H_q, sh.H_kv, sh.d, sh.alpha, k_outlier_channels=sh.k_outlier_channels)
+    dev = tq.KVCache(sh.B, sh.H_kv, S_cap, sh.d)
+    host = {}
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for b in picked:  # prefill the two sampled sequences through the CUDA quantiser, one sequence at a time
+        k, v = I.make_kv(one, int(lens[b]), seed=500 + b)
+        host[b] = oracle.Cache(1, sh.H_kv, S_cap, sh.d)
+        host[b].append(k, v)
+        view = tq.tq_kv_cache(dev.k_packed[b].data_ptr(), dev.v_packed[b].data_ptr(), dev.k_scale[b].data_ptr(),
+                              dev.k_zero[b].data_ptr(), dev.v_scale[b].data_ptr(), dev.v_zero[b].data_ptr(),
+                              dev.seq_lens[b:b + 1].data_ptr(), 1, sh.H_kv, S_cap, sh.d)
+        tq.tq_kv_quantize_append(view, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
+    dev.seq_lens.copy_(torch.from_numpy(lens))
+    C = tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q, sh.d, S_cap)
+    o, m, l = tq.alloc_partials(sh.B, sh.H_q, sh.d, C)
+    out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+    for step in range(64):
+        k_new = np.zeros((sh.B, sh.H_kv, 1, sh.d), np.float16)
+        v_new = np.zeros_like(k_new)
+        q = np.zeros((sh.B, sh.H_q, sh.d), np.float16)
+        for b in picked:
+            kb, vb = I.make_kv(one, 1, seed=500 + b, stream=1 + step)
+            k_new[b], v_new[b] = kb[0], vb[0]
+            q[b] = I.make_q(one, seed=500 + b, stream=step)[0]
+            host[b].append(kb, vb)
+        tq.tq_kv_quantize_append(dev, torch.from_numpy(k_new).cuda(), torch.from_numpy(v_new).cuda(), status)
+        tq.tq_sdpa_int4_decode(dev, torch.from_numpy(q).cuda(), sh.alpha, C, o, m, l, status)
+        tq.tq_sdpa_int4_combine(o, m, l, out)
+        if step in (0, 63):
+            torch.cuda.synchronize()
+            got = out.cpu().numpy()
+            for b in picked:
+                n = int(lens[b]) + step + 1
+                assert int(host[b].lens[0]) == n
+                for d_arr, h_arr in zip(dev.arrays_token_major(), host[b].arrays()):
+                    assert np.array_equal(d_arr[b, :, :n].cpu().numpy().view(np.uint8), h_arr[0, :, :n].view(np.uint8))
+                ref = oracle.attention(host[b], q[b:b + 1], sh.alpha)
+                mx, rel = assert_attention_close(got[b:b + 1], ref, f"ragged step {step} seq {b}")
+                print(f"ragged step {step} seq {b} len {n}: max-abs {mx:.2e} rel-L2 {rel:.2e}")
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert dev.seq_lens.cpu().tolist() == [int(x) + 64 for x in lens]
