@@ -17,6 +17,8 @@ __global__ void __launch_bounds__(kThreads) combine_kernel(const float* __restri
   __shared__ float w[TQ_MAX_SPLITS];
   __shared__ float red[kThreads / 32];
   __shared__ float4 acc[kThreads];
+  pdl_wait();
+  pdl_launch_dependents();
   const long long bh = blockIdx.x;
   const float* m = m_part + bh * C;
   const float* l = l_part + bh * C;
@@ -77,8 +79,8 @@ __global__ void __launch_bounds__(kThreads) combine_kernel(const float* __restri
 
 cudaError_t launch_combine(const float* o_part, const float* m_part, const float* l_part, int B, int H_q, int d, int C,
                            void* out, bool out_fp32, cudaStream_t st) {
-  combine_kernel<<<B * H_q, kThreads, 0, st>>>(o_part, m_part, l_part, d, C, out, out_fp32 ? 1 : 0);
-  return cudaGetLastError();
+  return launch_kernel(combine_kernel, dim3(B * H_q), dim3(kThreads), 0, st, o_part, m_part, l_part, d, C, out,
+                       out_fp32 ? 1 : 0);
 }
 
 }  // namespace tq

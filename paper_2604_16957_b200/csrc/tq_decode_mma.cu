@@ -317,6 +317,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tid4 = lane & 3;
   const int h0 = kvh * G + tile * 8;         // first query head of this tile
   const int nh = min(8, G - tile * 8);       // heads in the tile; the rest of N = 8 is zero padding
+  pdl_wait();  // nothing global is read before this point
+  pdl_launch_dependents();
   const int len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
   int t0, t1;
   split_range(len, C, c, t0, t1);
@@ -500,8 +502,8 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, float attn_sc
   if (attr != cudaSuccess) return attr;
   const int G = H_q / c.H_kv;
   dim3 grid(C, c.H_kv * ((G + 7) / 8), c.B);
-  decode_mma_kernel<D><<<grid, kThreads, Cfg<D>::SMEM, st>>>(c, q, H_q, attn_scale, C, o_part, m_part, l_part, status);
-  return cudaGetLastError();
+  return launch_kernel(decode_mma_kernel<D>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, attn_scale, C, o_part,
+                       m_part, l_part, status);
 }
 
 }  // namespace

@@ -40,7 +40,34 @@ __device__ inline int checked_len(const int32_t* seq_lens, int b, int S_cap, int
   return len;
 }
 
-// host-side launchers (each returns cudaGetLastError() after its launches)
+// Programmatic dependent launch.  The three kernels of a decode step (append, phase 1, reduction) are
+// launched with the programmatic-stream-serialization attribute, so the launch latency of each one
+// overlaps the tail of the kernel before it in the stream.  Every kernel calls pdl_wait() before its
+// first global access (that wait returns once the preceding kernel has completed and its writes are
+// visible, so ordering is exactly stream order) and pdl_launch_dependents() right after, which lets
+// the next kernel be scheduled as soon as this one's blocks start to retire.  Both are no-ops when
+// the kernel was launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
+bool pdl_enabled();  // false when the environment has TQ_PDL=0
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// host-side launchers (each returns the launch error, if any)
 cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, const __half* v_new, int T,
                                    int32_t* status, cudaStream_t st);
 cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C, float* o_part,

@@ -106,6 +106,8 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
 // observe a length that another block of the same launch has already advanced.
 __global__ void __launch_bounds__(256) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
                                                             int T) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.y;
   const int len = c.seq_lens[b];
   if (len < 0 || len + T > c.S_cap) return;  // flagged by bump_lens_kernel
@@ -120,6 +122,8 @@ __global__ void __launch_bounds__(256) quantize_bulk_kernel(tq_kv_cache c, const
 }
 
 __global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= c.B) return;
   const int len = c.seq_lens[b];
@@ -134,6 +138,8 @@ __global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
 // then advances the length itself -- a single launch, and no block reads another's length.
 __global__ void __launch_bounds__(256) quantize_step_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
                                                             int T, int32_t* status) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.x;
   const int len = c.seq_lens[b];
   if (len < 0 || len + T > c.S_cap) {
@@ -161,14 +167,14 @@ cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, co
                                    int32_t* status, cudaStream_t st) {
   const long long per_seq = static_cast<long long>(c.H_kv) * T * (c.d >> 3);
   if (2 * per_seq <= 8192) {
-    quantize_step_kernel<<<c.B, 256, 0, st>>>(c, k_new, v_new, T, status);
+    return launch_kernel(quantize_step_kernel, dim3(c.B), dim3(256), 0, st, c, k_new, v_new, T, status);
   } else {
     const long long blocks = (per_seq + 255) / 256;
     dim3 grid(static_cast<unsigned>(blocks), c.B, 2);
-    quantize_bulk_kernel<<<grid, 256, 0, st>>>(c, k_new, v_new, T);
-    bump_lens_kernel<<<(c.B + 127) / 128, 128, 0, st>>>(c, T, status);
+    const cudaError_t e = launch_kernel(quantize_bulk_kernel, grid, dim3(256), 0, st, c, k_new, v_new, T);
+    if (e != cudaSuccess) return e;
+    return launch_kernel(bump_lens_kernel, dim3((c.B + 127) / 128), dim3(128), 0, st, c, T, status);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace tq
