@@ -23,6 +23,21 @@ __global__ void __launch_bounds__(kThreads) combine_kernel(const float* __restri
   const float* m = m_part + bh * C;
   const float* l = l_part + bh * C;
   const int tid = threadIdx.x;
+  const int nchunk = d >> 2;            // float4 chunks per row (8 .. 64)
+  const int nsl = kThreads / nchunk;    // split lanes
+  const int chunk = tid % nchunk, sl = tid / nchunk;
+  const float4* o = reinterpret_cast<const float4*>(o_part + bh * C * d) + chunk;
+
+  // The partial outputs do not depend on the weights: fetch this thread's first kPre of them now, so
+  // that their latency overlaps the (m, l) loads and the weight computation below.
+  constexpr int kPre = 8;
+  float4 pre[kPre];
+#pragma unroll
+  for (int i = 0; i < kPre; ++i) {
+    const int c = sl + i * nsl;
+    pre[i] = (sl < nsl && c < C) ? o[static_cast<long long>(c) * nchunk] : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+
   // global maximum over non-empty splits (C <= 256: one split per thread)
   const float lc = tid < C ? l[tid] : 0.f;
   const float mc = (tid < C && lc > 0.f) ? m[tid] : -INFINITY;
@@ -37,22 +52,25 @@ __global__ void __launch_bounds__(kThreads) combine_kernel(const float* __restri
   if (tid < C) w[tid] = lc > 0.f ? lc * __expf(mc - mg) : 0.f;
   __syncthreads();
 
-  const int nchunk = d >> 2;            // float4 chunks per row (8 .. 64)
-  const int nsl = kThreads / nchunk;    // split lanes
-  const int chunk = tid % nchunk, sl = tid / nchunk;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
   float den = 0.f;
   if (sl < nsl) {
-    const float4* o = reinterpret_cast<const float4*>(o_part + bh * C * d) + chunk;
-    for (int c = sl; c < C; c += nsl) {
+#pragma unroll
+    for (int i = 0; i < kPre; ++i) {
+      const int c = sl + i * nsl;
+      const float wc = c < C ? w[c] : 0.f;  // an empty split has weight 0 and o = 0
+      a.x = fmaf(wc, pre[i].x, a.x);
+      a.y = fmaf(wc, pre[i].y, a.y);
+      a.z = fmaf(wc, pre[i].z, a.z);
+      a.w = fmaf(wc, pre[i].w, a.w);
+    }
+    for (int c = sl + kPre * nsl; c < C; c += nsl) {
       const float wc = w[c];
-      if (wc > 0.f) {
-        const float4 v = o[static_cast<long long>(c) * nchunk];
-        a.x = fmaf(wc, v.x, a.x);
-        a.y = fmaf(wc, v.y, a.y);
-        a.z = fmaf(wc, v.z, a.z);
-        a.w = fmaf(wc, v.w, a.w);
-      }
+      const float4 v = o[static_cast<long long>(c) * nchunk];
+      a.x = fmaf(wc, v.x, a.x);
+      a.y = fmaf(wc, v.y, a.y);
+      a.z = fmaf(wc, v.z, a.z);
+      a.w = fmaf(wc, v.w, a.w);
     }
   }
   acc[tid] = a;
