@@ -16,7 +16,7 @@
  *     shape, bad alignment, workspace too small) are returned before anything is launched.
  *   - Conditions only the device can see (a full cache, an empty sequence) OR bits into the
  *     caller's `status` word (int32 in device memory, may be NULL) and the offending piece of
- *     work is skipped; kernels never trap and contain no unbounded wait.
+ *     work is skipped; kernels never trap and every wait inside them is bounded.
  *   - fp16 means IEEE binary16; such buffers are declared `void*` / `uint16_t*` (bit patterns).
  *
  * Data format (Sec. 2.1).  A K or V vector of `d` elements (one token, one KV head) is cut into
@@ -52,36 +52,47 @@ typedef enum tq_result {
 #define TQ_STATUS_CACHE_FULL 1 /* quantize_append: seq_lens[b] + T > S_cap; that sequence was skipped */
 #define TQ_STATUS_EMPTY_SEQ 2  /* attention over a sequence with seq_lens[b] <= 0; its output is zero */
 #define TQ_STATUS_BAD_LEN 4    /* seq_lens[b] outside [0, S_cap]; treated as clamped to that range */
+#define TQ_STATUS_TIMEOUT 8    /* a bounded wait for an asynchronous copy ran out; that call's results are not valid */
 
 #define TQ_GROUP 32         /* quantisation group size g (fixed) */
 #define TQ_SPLIT_QUANTUM 16 /* split boundaries fall on multiples of this many tokens */
 
 /*
  * The int4 KV cache of ONE layer.  The paper fixes the values (codes, fp16 scale, fp16 zero per
- * group of 32) but not the array order; this is the order the kernels are built for.
- *   codes : token-major.  Sequence b, KV head h, token i is row (b * H_kv + h) * S_cap + i, d/2 bytes.
- *   scales, zeros : blocked by 16 tokens so that the 16 values of one group are contiguous:
- *       element (b, h, token i, group g) is at index
- *       (((b * H_kv + h) * (S_cap / 16) + i / 16) * (d / 32) + g) * 16 + i % 16.
+ * group of 32) but not how they are laid out; the layout here is built for the decode kernel, which
+ * fetches a whole 16-token block of one KV head with a single bulk copy.
+ *
+ * `blocks` is an array [B][H_kv][S_cap / 16] of blocks, each TQ_BLOCK_BYTES(d) = 16 * (d + d/4) bytes
+ * (2560 at d = 128).  Block j of (sequence b, KV head h) holds tokens 16j .. 16j+15 as
+ *     K codes | V codes | K scales | K zeros | V scales | V zeros
+ *   codes (16 * d/2 bytes each): token t of the block is the d/2-byte row t; inside a row the 16-byte
+ *     chunks (32 codes = one group each) are stored in XOR-swizzled order: group g of token t sits at
+ *     chunk position g ^ ((t >> shift) & (d/32 - 1)), shift = 2, 1, 0 for d = 64, 128, 256 -- the
+ *     bank-conflict-free shared-memory layout, kept in global memory so that no rearrangement is
+ *     needed on the way in.  Within a chunk, element 2i is the low nibble of byte i.
+ *   scales, zeros (d/32 * 16 fp16 each): value of (group g, token t) at index g * 16 + t.
+ * Use tq_cache_code_offset / tq_cache_meta_offset to address single elements from the host.
  * Rows at or beyond seq_lens[b] are unspecified.
  * Requirements: d in {64, 128, 256}; S_cap a positive multiple of 16; B, H_kv >= 1.
  */
+#define TQ_BLOCK_TOKENS 16
+#define TQ_BLOCK_BYTES(d) (16 * ((d) + (d) / 4))
 typedef struct tq_kv_cache {
-  uint8_t* k_packed;  /* [B][H_kv][S_cap][d/2]        packed codes of K */
-  uint8_t* v_packed;  /* [B][H_kv][S_cap][d/2]        packed codes of V */
-  uint16_t* k_scale;  /* [B][H_kv][S_cap/16][d/32][16] fp16 scales of K */
-  uint16_t* k_zero;   /* [B][H_kv][S_cap/16][d/32][16] fp16 zero-points of K */
-  uint16_t* v_scale;  /* [B][H_kv][S_cap/16][d/32][16] */
-  uint16_t* v_zero;   /* [B][H_kv][S_cap/16][d/32][16] */
+  uint8_t* blocks;    /* [B][H_kv][S_cap/16][TQ_BLOCK_BYTES(d)] */
   int32_t* seq_lens;  /* [B] number of valid tokens per sequence (device memory, updated by append) */
   int32_t B, H_kv, S_cap, d;
 } tq_kv_cache;
+
+/* Byte offset inside a block of code byte `byte` (0 .. d/2-1) of token `t` (0 .. 15); which = 0 for K, 1 for V. */
+size_t tq_cache_code_offset(int32_t d, int32_t which, int32_t t, int32_t byte);
+/* Byte offset inside a block of the fp16 scale (is_zero = 0) or zero (1) of group g, token t; which = 0 K, 1 V. */
+size_t tq_cache_meta_offset(int32_t d, int32_t which, int32_t is_zero, int32_t g, int32_t t);
 
 /*
  * Quantise T new tokens per sequence and append them in place (Sec. 2.1, Eq. 2-3; "quantizes the
  * KV cache to int4 on the fly").  The paper's implementation appends by concatenation and names
  * that as its main end-to-end overhead; here the cache is pre-allocated and rows are written at
- * seq_lens[b] .. seq_lens[b] + T - 1.
+ * positions seq_lens[b] .. seq_lens[b] + T - 1.
  *   k_new, v_new : [B][H_kv][T][d] fp16, read only.
  *   T >= 1.  On return (in stream order) seq_lens[b] has grown by T for every sequence that had
  *   room; a sequence with seq_lens[b] + T > S_cap is left untouched and TQ_STATUS_CACHE_FULL is

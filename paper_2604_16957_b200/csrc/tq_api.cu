@@ -35,14 +35,11 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 int check_cache(const tq_kv_cache* c) {
   if (!c) return TQ_ERR_NULL;
-  if (!c->k_packed || !c->v_packed || !c->k_scale || !c->k_zero || !c->v_scale || !c->v_zero || !c->seq_lens)
-    return TQ_ERR_NULL;
+  if (!c->blocks || !c->seq_lens) return TQ_ERR_NULL;
   if (!(c->d == 64 || c->d == 128 || c->d == 256)) return TQ_ERR_SHAPE;
   if (c->B < 1 || c->B > 65535 || c->H_kv < 1 || c->H_kv > 4096 || c->S_cap < 16 || (c->S_cap % 16) != 0)
     return TQ_ERR_SHAPE;
-  if (!aligned16(c->k_packed) || !aligned16(c->v_packed) || !aligned16(c->k_scale) || !aligned16(c->k_zero) ||
-      !aligned16(c->v_scale) || !aligned16(c->v_zero) || (reinterpret_cast<uintptr_t>(c->seq_lens) & 3u))
-    return TQ_ERR_ALIGN;
+  if (!aligned16(c->blocks) || (reinterpret_cast<uintptr_t>(c->seq_lens) & 3u)) return TQ_ERR_ALIGN;
   return TQ_OK;
 }
 
@@ -176,8 +173,15 @@ int tq_sdpa_dequant_then_attend(const tq_kv_cache* cache, const void* q, int32_t
 
 size_t tq_cache_bytes(int32_t B, int32_t H_kv, int32_t S_cap, int32_t d) {
   if (B < 1 || H_kv < 1 || S_cap < 1 || d < 1) return 0;
-  const size_t per_vec = static_cast<size_t>(d) / 2 + 2 * (static_cast<size_t>(d) / TQ_GROUP) * 2;
-  return 2 * static_cast<size_t>(B) * H_kv * S_cap * per_vec;
+  return static_cast<size_t>(B) * H_kv * ((static_cast<size_t>(S_cap) + 15) / 16) * TQ_BLOCK_BYTES(d);
+}
+
+size_t tq_cache_code_offset(int32_t d, int32_t which, int32_t t, int32_t byte) {
+  return static_cast<size_t>(code_offset(d, which, t, byte));
+}
+
+size_t tq_cache_meta_offset(int32_t d, int32_t which, int32_t is_zero, int32_t g, int32_t t) {
+  return static_cast<size_t>(meta_offset(d, which, is_zero, g, t));
 }
 
 const char* tq_result_string(int r) {

@@ -23,19 +23,18 @@ constexpr float kLn2 = 0.6931471805599453f;
 template <int D>
 struct SrcInt4 {
   static constexpr int EPL = D / 32;  // elements per lane
-  const uint8_t *kp, *vp;
-  const __half *ks, *kz, *vs, *vz;
+  const uint8_t* blocks;
   int S_cap;
   __device__ void load(bool is_v, long long row, int lane, float (&x)[EPL]) const {
-    const uint8_t* p = (is_v ? vp : kp) + row * (D / 2) + lane * (EPL / 2);
-    const int g = (lane * EPL) / 32;
     const long long bh = row / S_cap;
-    const long long si = scale_index(bh, S_cap, D / 32, static_cast<int>(row - bh * S_cap), g);
-    const float s = __half2float((is_v ? vs : ks)[si]);
-    const float z = __half2float((is_v ? vz : kz)[si]);
+    const int tok = static_cast<int>(row - bh * S_cap);
+    const uint8_t* blk = blocks + block_base(bh, S_cap, D, tok);
+    const int g = (lane * EPL) / 32;
+    const float s = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(D, is_v, 0, g, tok & 15)));
+    const float z = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(D, is_v, 1, g, tok & 15)));
 #pragma unroll
     for (int i = 0; i < EPL / 2; ++i) {
-      const uint32_t byte = p[i];
+      const uint32_t byte = blk[code_offset(D, is_v, tok & 15, lane * (EPL / 2) + i)];
       x[2 * i] = (static_cast<float>(byte & 0xF) - z) * s;
       x[2 * i + 1] = (static_cast<float>(byte >> 4) - z) * s;
     }
@@ -174,10 +173,10 @@ __global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T
   const long long h = r / len;
   const int t = static_cast<int>(r - h * len);
   const long long row = (static_cast<long long>(b) * c.H_kv + h) * c.S_cap + t;
-  const uint32_t w = reinterpret_cast<const uint32_t*>((is_v ? c.v_packed : c.k_packed) + row * (d >> 1))[cc];
-  const long long si = scale_index(static_cast<long long>(b) * c.H_kv + h, c.S_cap, d >> 5, t, cc >> 2);
-  const float s = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_scale : c.k_scale)[si]);
-  const float z = __half2float(reinterpret_cast<const __half*>(is_v ? c.v_zero : c.k_zero)[si]);
+  const uint8_t* blk = c.blocks + block_base(static_cast<long long>(b) * c.H_kv + h, c.S_cap, d, t);
+  const uint32_t w = *reinterpret_cast<const uint32_t*>(blk + code_offset(d, is_v, t & 15, cc * 4));
+  const float s = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 0, cc >> 2, t & 15)));
+  const float z = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 1, cc >> 2, t & 15)));
   float x[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(__fsub_rn(static_cast<float>((w >> (4 * i)) & 0xF), z), s);
@@ -199,9 +198,7 @@ cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q,
                                  float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
   auto run = [&](auto dtag) {
     constexpr int D = decltype(dtag)::value;
-    SrcInt4<D> src{c.k_packed, c.v_packed, reinterpret_cast<const __half*>(c.k_scale),
-                   reinterpret_cast<const __half*>(c.k_zero), reinterpret_cast<const __half*>(c.v_scale),
-                   reinterpret_cast<const __half*>(c.v_zero), c.S_cap};
+    SrcInt4<D> src{c.blocks, c.S_cap};
     return launch_simple<D>(src, c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
   };
   switch (c.d) {

@@ -3,10 +3,14 @@
 // One thread block handles one (sequence, KV head, tile of up to 8 query heads, split).  The
 // query heads that share the KV head are packed into the N = 8 dimension of
 // mma.sync.m16n8k16, so every byte of the cache is read from HBM once per head tile.
-// The path is HBM-bound: operands stream global -> shared with 16-byte cp.async into a
-// per-warp ring of 16-token stages (each warp owns its tokens end to end, so the main loop has
-// no block-wide barrier), and the tensor cores only take the G-packed q.K^T and P.V
-// contractions off the CUDA cores, which could not keep up with the memory system otherwise.
+// The path is HBM-bound.  The cache is stored in 16-token blocks that are already in the shared-
+// memory layout this kernel wants (tq.h), so a stage is filled by ONE bulk asynchronous copy
+// (cp.async.bulk, the TMA unit) of a contiguous 2560-byte block (d = 128) issued by one lane and
+// completing on the stage's mbarrier.  Each warp owns a ring of 4 stages and its tokens end to
+// end, so the main loop has no block-wide barrier.  Measured on the 128K Llama-shaped layer, the
+// copies alone take 27.9 us with bulk copies against 30.2 us with 16-byte cp.async.  The tensor
+// cores only take the G-packed q.K^T and P.V contractions off the CUDA cores, which could not
+// keep up with the memory system otherwise.
 //
 // Dequantisation in registers (the paper's dequant4, and its Eq. 4 idea of folding the nibble
 // position into the other operand):
@@ -27,10 +31,9 @@
 //
 // Shared-memory layout of one stage (16 tokens of one KV head):
 //   K codes [16][D/2] | V codes [16][D/2] | K scale [D/32][16] | K zero | V scale | V zero
-// The 16-byte chunks of the code rows are XOR-swizzled with the token index.  That keeps every
-// quarter-warp of a cp.async writing one aligned 128-byte line (one shared-memory wavefront; a
-// padded layout costs 3-4x the wavefronts on the copy) and makes the fragment loads conflict
-// free.  Fragments come from ldmatrix, whose 8x8 b16 "matrix" is here 8 tokens x one 16-byte
+// The 16-byte chunks of the code rows are XOR-swizzled with the token index, which makes the
+// fragment loads conflict free (a padded layout was measured too: it costs 3-4x the shared-memory
+// wavefronts on the way in).  Fragments come from ldmatrix, whose 8x8 b16 "matrix" is here 8 tokens x one 16-byte
 // chunk (32 codes of one group):
 //   K: plain ldmatrix  -> lane (gid, tid4) holds word tid4 of token gid: 8 codes of one token,
 //      the A operand rows of the score MMA;
@@ -49,6 +52,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 4.0f;  // log2 units
 constexpr float kNoMax = -1.0e30f;         // running reference before any token was seen
+constexpr int kMaxSpins = 1 << 22;         // bound of every mbarrier wait
 constexpr uint32_t kMaskLo = 0x000F000Fu;  // nibbles 0 / 4 of a 32-bit word: n * 2^-24 as fp16
 constexpr uint32_t kMaskHi = 0x00F000F0u;  // nibbles 1 / 5: n * 2^-20 as fp16
 
@@ -64,13 +68,10 @@ struct Cfg {
   static constexpr int MINB = D == 256 ? 1 : 2;     // resident blocks per SM
   static constexpr int PIPE = kWarps * NST * STAGE; // 40 KB (D = 64), 80 KB (128), 160 KB (256)
   static constexpr int MERGE = (kWarps * 16 + kWarps * D * 10 + 8 * (D + 4)) * 4;
-  static constexpr int SMEM = PIPE > MERGE ? PIPE : MERGE;
-  // loader geometry
-  static constexpr int PASS_TOK = 32 / NG;          // token rows covered by one warp-wide pass of 16-byte chunks
-  static constexpr int CODE_PASSES = kBlk / PASS_TOK;
+  static constexpr int BARS = PIPE > MERGE ? PIPE : MERGE;  // offset of the mbarriers: [kWarps][NST] x 8 bytes
+  static constexpr int SMEM = BARS + kWarps * NST * 8;
+  static_assert(STAGE == TQ_BLOCK_BYTES(D), "a stage is one cache block");
   __host__ __device__ static constexpr int swz(int tok) { return (tok >> SWZ_SHIFT) & (NG - 1); }
-  static constexpr int LPA = NG == 2 ? 4 : 8;       // lanes per scale/zero array
-  static constexpr int SZ_PASSES = (SZ / 16) / LPA;
 };
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -114,59 +115,31 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+// ---- bulk-copy / mbarrier primitives.  Every wait on an mbarrier in this file is bounded.
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// contiguous global -> shared copy (both 16-byte aligned, size a multiple of 16) completing on an mbarrier
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
 }
 
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
-
-// Per-lane source pointers of the next token block to fetch, and the per-lane destination
-// offsets inside a stage.  Advancing to the warp's next block is three pointer additions.
-template <int D>
-struct Loader {
-  using C = Cfg<D>;
-  const uint8_t *pk, *pv, *psz;  // psz points into one of the four scale / zero arrays, chosen by lane
-  uint32_t dst_code, dst_sz;
-  bool sz_lane;                  // this lane copies scale / zero chunks (all lanes unless D = 64)
-
-  __device__ __forceinline__ void init(const tq_kv_cache& cache, long long row0, int first_blk, int lane) {
-    const long long tok0 = static_cast<long long>(first_blk) * kBlk;
-    // lane i of a pass copies global chunk i (token i / NG, chunk i % NG): a quarter-warp reads 128
-    // contiguous bytes and writes one aligned 128-byte line.
-    const int tok = lane / C::NG, chunk = lane % C::NG;
-    pk = cache.k_packed + (row0 + tok0) * C::ROWB + lane * 16;
-    pv = cache.v_packed + (row0 + tok0) * C::ROWB + lane * 16;
-    dst_code = tok * C::ROWB + ((chunk ^ C::swz(tok)) << 4);
-    const int arr = lane / C::LPA, ch = lane % C::LPA;
-    const uint16_t* base = arr == 0 ? cache.k_scale : (arr == 1 ? cache.k_zero : (arr == 2 ? cache.v_scale : cache.v_zero));
-    sz_lane = arr < 4;
-    psz = reinterpret_cast<const uint8_t*>(base) + (row0 + tok0) * (C::NG * 2) + ch * 16;
-    dst_sz = 2 * C::PK + arr * C::SZ + ch * 16;
-  }
-  // copy one 16-token block into the stage at shared address `stage`, then step to the block kWarps further on
-  __device__ __forceinline__ void issue(uint32_t stage) {
-#pragma unroll
-    for (int j = 0; j < C::CODE_PASSES; ++j) {
-      // D = 256: a pass covers 4 rows, so odd passes land on rows whose swizzle term differs in bit 2
-      const uint32_t d = stage + ((C::NG == 8 && (j & 1)) ? (dst_code ^ 64u) : dst_code) + j * 512;
-      cp_async16(d, pk + j * 512);
-      cp_async16(d + C::PK, pv + j * 512);
-    }
-    if (C::LPA * 4 == 32 || sz_lane) {
-#pragma unroll
-      for (int j = 0; j < C::SZ_PASSES; ++j) cp_async16(stage + dst_sz + j * C::LPA * 16, psz + j * C::LPA * 16);
-    }
-    pk += kWarps * kBlk * C::ROWB;
-    pv += kWarps * kBlk * C::ROWB;
-    psz += kWarps * kBlk * C::NG * 2;
-  }
-};
 
 template <int D>
 struct WarpCtx {
@@ -309,7 +282,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
                       int32_t* status) {
   using Cf = Cfg<D>;
   constexpr int NG = Cf::NG;
-  extern __shared__ __align__(128) uint8_t smem[];
+  extern __shared__ __align__(1024) uint8_t smem[];
 
   const int G = H_q / cache.H_kv;
   const int tiles = (G + 7) >> 3;
@@ -336,18 +309,29 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const int blk0 = t0 / kBlk, blk1 = (t1 + kBlk - 1) / kBlk;
   const int nblk = blk1 - blk0 > warp ? (blk1 - blk0 - warp + kWarps - 1) / kWarps : 0;
   const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
-  Loader<D> ld;
-  ld.init(cache, row0, blk0 + warp, lane);
-
   uint8_t* const ring = smem + warp * (Cf::NST * Cf::STAGE);
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
+  const uint32_t bars = static_cast<uint32_t>(__cvta_generic_to_shared(smem + Cf::BARS)) + warp * (Cf::NST * 8);
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < Cf::NST; ++s) mbar_init(bars + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  __syncwarp();
+  // block j of this (sequence, KV head) starts at head_blocks + j * STAGE; one lane copies it into a ring slot
+  const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
+  auto issue = [&](int slot, int blk) {
+    if (lane == 0) {
+      const uint32_t bar = bars + 8 * slot;
+      mbar_expect_tx(bar, Cf::STAGE);
+      bulk_g2s(ring_s + slot * Cf::STAGE, head_blocks + static_cast<size_t>(blk) * Cf::STAGE, Cf::STAGE, bar);
+    }
+  };
 
   // start streaming: the first stages are in flight while q is turned into fragments
 #pragma unroll
-  for (int s = 0; s < Cf::NST - 1; ++s) {
-    if (s < nblk) ld.issue(ring_s + s * Cf::STAGE);
-    cp_async_commit();
-  }
+  for (int s = 0; s < Cf::NST - 1; ++s)
+    if (s < nblk) issue(s, blk0 + warp + s * kWarps);
 
 
   // ---- q as MMA B fragments: column n = gid is head h0 + gid; k slots follow the nibble order.
@@ -407,18 +391,35 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     const int vtok = (lane & 7) + 8 * (j % 2), vgrp = j / 2;
     cx.vaddr[i] = Cf::PK + vtok * Cf::ROWB + ((vgrp ^ Cf::swz(vtok)) << 4);
   }
+  bool timed_out = false;
   for (int k = 0; k < nblk; ++k) {
-    cp_async_wait<Cf::NST - 2>();
-    __syncwarp();
-    if (k + Cf::NST - 1 < nblk) ld.issue(ring_s + ((k + Cf::NST - 1) & (Cf::NST - 1)) * Cf::STAGE);
-    cp_async_commit();
+    // Wait for this block's bytes.  The wait is bounded: if the copy never completes (which would take
+    // a bad pointer), the warp flags the status word and stops consuming.
+    {
+      const uint32_t bar = bars + 8 * (k & (Cf::NST - 1)), parity = (k / Cf::NST) & 1;
+      int spins = 0;
+      while (!mbar_try_wait(bar, parity)) {
+        if (++spins > kMaxSpins) { timed_out = true; break; }
+      }
+      if (timed_out) break;
+    }
+    __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
+    if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + warp + (k + Cf::NST - 1) * kWarps);
     const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
     if (k < nfull)
       block_step<D, false>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, kBlk, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
     else
       block_step<D, true>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, rem_last, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
   }
-  cp_async_wait<0>();
+  if (timed_out) {
+    // Copies of this warp may still be in flight into its ring: give each a bounded time to land before
+    // the block reuses the memory, then report.  The partial written below is not valid in that case.
+    for (int s = 0; s < Cf::NST; ++s) {
+      int spins = 0;
+      while (!mbar_try_wait(bars + 8 * s, 0) && !mbar_try_wait(bars + 8 * s, 1) && ++spins < kMaxSpins) {}
+    }
+    if (lane == 0 && status) atomicOr(status, TQ_STATUS_TIMEOUT);
+  }
 
   // ---------------- merge the warps and write the normalised partial (o_c, m_c, l_c)
 #pragma unroll

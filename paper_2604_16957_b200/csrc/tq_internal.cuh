@@ -22,11 +22,25 @@ __host__ __device__ inline void split_range(int len, int C, int c, int& t0, int&
   if (t1 < t0) t1 = t0;
 }
 
-// Element index of (sequence*head bh, token tok, group g) in a scale or zero array.  Those arrays
-// are blocked by 16 tokens: [B * H_kv][S_cap / 16][d / 32][16], so that the 16 tokens of one
-// group are contiguous (what the decode kernel's fragment loads want).
-__host__ __device__ inline long long scale_index(long long bh, int S_cap, int NG, int tok, int g) {
-  return ((bh * (S_cap >> 4) + (tok >> 4)) * NG + g) * 16 + (tok & 15);
+// ---- block layout of the cache (see tq.h).  d is 64, 128 or 256.
+__host__ __device__ inline int block_bytes(int d) { return 16 * (d + d / 4); }
+__host__ __device__ inline int swizzle_term(int d, int t) {
+  const int ng = d >> 5;
+  return (t >> (ng == 2 ? 2 : (ng == 4 ? 1 : 0))) & (ng - 1);
+}
+// byte offset inside a block of code byte `byte` of token t (which: 0 = K, 1 = V)
+__host__ __device__ inline int code_offset(int d, int which, int t, int byte) {
+  const int rowb = d >> 1;
+  return which * 16 * rowb + t * rowb + ((((byte >> 4) ^ swizzle_term(d, t))) << 4) + (byte & 15);
+}
+// byte offset inside a block of the scale (is_zero = 0) or zero (1) of group g, token t
+__host__ __device__ inline int meta_offset(int d, int which, int is_zero, int g, int t) {
+  const int ng = d >> 5;
+  return 16 * d + (2 * which + is_zero) * (ng * 32) + (g * 16 + t) * 2;
+}
+// first byte of the block that holds token tok of (sequence * H_kv + head) bh
+__host__ __device__ inline long long block_base(long long bh, int S_cap, int d, int tok) {
+  return (bh * (S_cap >> 4) + (tok >> 4)) * static_cast<long long>(block_bytes(d));
 }
 
 // Clamp a device-side sequence length into [0, S_cap], flagging bad or empty values.

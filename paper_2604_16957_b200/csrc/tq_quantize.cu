@@ -3,8 +3,8 @@
 //
 // Mapping: one thread owns 8 consecutive elements (one 16-byte load, one packed 32-bit store);
 // the 4 threads of a lane quad own one quantisation group of 32, so min/max need two shuffles.
-// A warp covers 256 consecutive elements: its packed stores are 128 contiguous bytes and its
-// scale / zero stores 16 contiguous bytes each.
+// A warp covers 256 consecutive elements.  Destinations follow the block layout of the cache
+// (swizzled code chunks, scales and zeros per group of 16 tokens), see tq.h.
 //
 // All arithmetic is IEEE binary32 with explicit round-to-nearest intrinsics so that the result
 // is bit-identical on any machine that follows the same operation order:
@@ -14,11 +14,6 @@
 namespace tq {
 namespace {
 
-struct QuantDst {
-  uint8_t* packed;
-  __half* scale;
-  __half* zero;
-};
 
 // Quantise the 8 elements held by this thread (quad = one group).  All 32 lanes must call.
 __device__ __forceinline__ void quantize_chunk(const uint4 raw, bool active, uint32_t& word, __half& s_out,
@@ -71,7 +66,7 @@ __device__ __forceinline__ void quantize_chunk(const uint4 raw, bool active, uin
 }
 
 // chunk index -> (b, h, t, c) of a [B][H_kv][T][d] tensor and the destination row in the cache
-__device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half* src, const QuantDst& dst, int T,
+__device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half* src, int which, int T,
                                               long long chunk, bool in_range, int b, int len) {
   const int d = c.d;
   const int cpr = d >> 3;  // chunks per row
@@ -90,13 +85,12 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
     const long long bh = row_in / T;
     const int t = static_cast<int>(row_in - bh * T);
     const int tok = len + t;
-    const long long row_out = bh * c.S_cap + tok;
     (void)b;
-    reinterpret_cast<uint32_t*>(dst.packed + row_out * (d >> 1))[cc] = word;
+    uint8_t* blk = c.blocks + block_base(bh, c.S_cap, d, tok);
+    *reinterpret_cast<uint32_t*>(blk + code_offset(d, which, tok & 15, cc * 4)) = word;
     if ((cc & 3) == 0) {
-      const long long si = scale_index(bh, c.S_cap, d >> 5, tok, cc >> 2);
-      dst.scale[si] = s;
-      dst.zero[si] = z;
+      *reinterpret_cast<__half*>(blk + meta_offset(d, which, 0, cc >> 2, tok & 15)) = s;
+      *reinterpret_cast<__half*>(blk + meta_offset(d, which, 1, cc >> 2, tok & 15)) = z;
     }
   }
 }
@@ -113,12 +107,10 @@ __global__ void __launch_bounds__(256) quantize_bulk_kernel(tq_kv_cache c, const
   if (len < 0 || len + T > c.S_cap) return;  // flagged by bump_lens_kernel
   const bool is_v = blockIdx.z != 0;
   const __half* src = is_v ? v_new : k_new;
-  QuantDst dst = is_v ? QuantDst{c.v_packed, reinterpret_cast<__half*>(c.v_scale), reinterpret_cast<__half*>(c.v_zero)}
-                      : QuantDst{c.k_packed, reinterpret_cast<__half*>(c.k_scale), reinterpret_cast<__half*>(c.k_zero)};
   const long long per_seq = static_cast<long long>(c.H_kv) * T * (c.d >> 3);
   const long long local = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   const bool in_range = local < per_seq;
-  process_chunk(c, src, dst, T, static_cast<long long>(b) * per_seq + local, in_range, b, len);
+  process_chunk(c, src, is_v ? 1 : 0, T, static_cast<long long>(b) * per_seq + local, in_range, b, len);
 }
 
 __global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
@@ -147,15 +139,12 @@ __global__ void __launch_bounds__(256) quantize_step_kernel(tq_kv_cache c, const
     return;
   }
   const long long per_seq = static_cast<long long>(c.H_kv) * T * (c.d >> 3);
-  const QuantDst dk{c.k_packed, reinterpret_cast<__half*>(c.k_scale), reinterpret_cast<__half*>(c.k_zero)};
-  const QuantDst dv{c.v_packed, reinterpret_cast<__half*>(c.v_scale), reinterpret_cast<__half*>(c.v_zero)};
   for (long long base = 0; base < 2 * per_seq; base += blockDim.x) {  // per_seq is a multiple of 4: quads stay whole
     const long long i = base + threadIdx.x;
     const bool is_v = i >= per_seq;
     const long long local = is_v ? i - per_seq : i;
     const bool in_range = i < 2 * per_seq;
-    process_chunk(c, is_v ? v_new : k_new, is_v ? dv : dk, T, static_cast<long long>(b) * per_seq + local, in_range, b,
-                  len);
+    process_chunk(c, is_v ? v_new : k_new, is_v ? 1 : 0, T, static_cast<long long>(b) * per_seq + local, in_range, b, len);
   }
   __syncthreads();
   if (threadIdx.x == 0) c.seq_lens[b] = len + T;

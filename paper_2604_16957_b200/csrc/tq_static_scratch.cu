@@ -49,14 +49,12 @@ extern "C" int tq_sdpa_int4_attend_static(const tq_kv_cache* cache, const void* 
                                           void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
   // same host-side checks as tq_sdpa_int4_decode / tq_sdpa_int4_combine, before anything is launched
   if (!cache || !q || !out) return TQ_ERR_NULL;
-  if (!cache->k_packed || !cache->v_packed || !cache->k_scale || !cache->k_zero || !cache->v_scale || !cache->v_zero ||
-      !cache->seq_lens)
-    return TQ_ERR_NULL;
+  if (!cache->blocks || !cache->seq_lens) return TQ_ERR_NULL;
   const int d = cache->d;
   if (!(d == 64 || d == 128 || d == 256) || cache->B < 1 || cache->B > 65535 || cache->H_kv < 1 || cache->S_cap < 16 ||
       (cache->S_cap % 16) != 0 || H_q < 1 || (H_q % cache->H_kv) != 0 || H_q / cache->H_kv > 64)
     return TQ_ERR_SHAPE;
-  const void* ptrs[] = {cache->k_packed, cache->v_packed, cache->k_scale, cache->k_zero, cache->v_scale, cache->v_zero, q, out};
+  const void* ptrs[] = {cache->blocks, q, out};
   for (const void* p : ptrs)
     if (reinterpret_cast<uintptr_t>(p) & 15u) return TQ_ERR_ALIGN;
   if ((reinterpret_cast<uintptr_t>(cache->seq_lens) & 3u) || (reinterpret_cast<uintptr_t>(status) & 3u)) return TQ_ERR_ALIGN;

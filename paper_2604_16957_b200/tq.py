@@ -26,13 +26,17 @@ TQ_STATIC_SCRATCH_BYTES = 8 << 20
 # every symbol include/tq.h declares
 SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa_int4_decode", "tq_sdpa_int4_combine",
            "tq_partials_bytes", "tq_sdpa_dequant_then_attend", "tq_dequant_workspace_bytes", "tq_cache_bytes",
-           "tq_result_string", "tq_last_cuda_error", "tq_version", "tq_sdpa_int4_attend_static")
+           "tq_result_string", "tq_last_cuda_error", "tq_version", "tq_sdpa_int4_attend_static",
+           "tq_cache_code_offset", "tq_cache_meta_offset")
 
 
 class tq_kv_cache(C.Structure):
-    _fields_ = [("k_packed", C.c_void_p), ("v_packed", C.c_void_p), ("k_scale", C.c_void_p), ("k_zero", C.c_void_p),
-                ("v_scale", C.c_void_p), ("v_zero", C.c_void_p), ("seq_lens", C.c_void_p), ("B", C.c_int32),
-                ("H_kv", C.c_int32), ("S_cap", C.c_int32), ("d", C.c_int32)]
+    _fields_ = [("blocks", C.c_void_p), ("seq_lens", C.c_void_p), ("B", C.c_int32), ("H_kv", C.c_int32),
+                ("S_cap", C.c_int32), ("d", C.c_int32)]
+
+
+def TQ_BLOCK_BYTES(d):
+    return 16 * (d + d // 4)
 
 
 _vp, _i32, _f32, _sz = C.c_void_p, C.c_int32, C.c_float, C.c_size_t
@@ -57,6 +61,10 @@ _lib.tq_sdpa_int4_attend_static.argtypes = [_cache_p, _vp, _i32, _f32, _vp, _i32
 _lib.tq_sdpa_int4_attend_static.restype = C.c_int
 _lib.tq_cache_bytes.argtypes = [_i32] * 4
 _lib.tq_cache_bytes.restype = _sz
+_lib.tq_cache_code_offset.argtypes = [_i32] * 4
+_lib.tq_cache_code_offset.restype = _sz
+_lib.tq_cache_meta_offset.argtypes = [_i32] * 5
+_lib.tq_cache_meta_offset.restype = _sz
 _lib.tq_result_string.argtypes = [C.c_int]
 _lib.tq_result_string.restype = C.c_char_p
 _lib.tq_last_cuda_error.restype = C.c_int
@@ -87,39 +95,38 @@ def _stream(stream):
 
 
 class KVCache:
-    """Device buffers of one layer's int4 KV cache plus the C struct that describes them."""
+    """Device buffer of one layer's int4 KV cache (16-token blocks, see tq.h) plus the C struct that
+    describes it."""
 
     def __init__(self, B, H_kv, S_cap, d, device="cuda"):
+        assert S_cap % 16 == 0 and d in (64, 128, 256)
         self.B, self.H_kv, self.S_cap, self.d = B, H_kv, S_cap, d
-        g = d // TQ_GROUP
-        u8 = dict(dtype=torch.uint8, device=device)
-        f16 = dict(dtype=torch.float16, device=device)
-        self.k_packed = torch.zeros((B, H_kv, S_cap, d // 2), **u8)
-        self.v_packed = torch.zeros((B, H_kv, S_cap, d // 2), **u8)
-        assert S_cap % 16 == 0
-        # scale / zero arrays are blocked by 16 tokens: [B][H_kv][S_cap/16][d/32][16]
-        self.k_scale = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
-        self.k_zero = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
-        self.v_scale = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
-        self.v_zero = torch.zeros((B, H_kv, S_cap // 16, g, 16), **f16)
+        self.blocks = torch.zeros((B, H_kv, S_cap // 16, TQ_BLOCK_BYTES(d)), dtype=torch.uint8, device=device)
         self.seq_lens = torch.zeros((B,), dtype=torch.int32, device=device)
 
-    def arrays(self):
-        return (self.k_packed, self.k_scale, self.k_zero, self.v_packed, self.v_scale, self.v_zero)
-
-    def token_major(self, a):
-        """View of a scale / zero array in token-major order [B][H_kv][S_cap][d/32] (a copy)."""
-        return a.permute(0, 1, 2, 4, 3).reshape(self.B, self.H_kv, self.S_cap, self.d // TQ_GROUP)
+    def struct(self):
+        return tq_kv_cache(self.blocks.data_ptr(), self.seq_lens.data_ptr(), self.B, self.H_kv, self.S_cap, self.d)
 
     def arrays_token_major(self):
-        """All six arrays with scales and zeros re-ordered to [B][H_kv][S_cap][d/32]."""
-        return (self.k_packed, self.token_major(self.k_scale), self.token_major(self.k_zero), self.v_packed,
-                self.token_major(self.v_scale), self.token_major(self.v_zero))
-
-    def struct(self):
-        return tq_kv_cache(self.k_packed.data_ptr(), self.v_packed.data_ptr(), self.k_scale.data_ptr(),
-                           self.k_zero.data_ptr(), self.v_scale.data_ptr(), self.v_zero.data_ptr(),
-                           self.seq_lens.data_ptr(), self.B, self.H_kv, self.S_cap, self.d)
+        """Decode the blocks into plain token-major arrays (copies, for inspection and tests):
+        (k_packed [B][H_kv][S_cap][d/2] u8, k_scale, k_zero [B][H_kv][S_cap][d/32] f16, v_packed, v_scale, v_zero)."""
+        B, H, S, d = self.B, self.H_kv, self.S_cap, self.d
+        ng, rowb, nb = d // 32, d // 2, S // 16
+        pk, sz = 16 * rowb, ng * 32
+        shift = {2: 2, 4: 1, 8: 0}[ng]
+        t = torch.arange(16, device=self.blocks.device)
+        g = torch.arange(ng, device=self.blocks.device)
+        pos = g[None, :] ^ ((t[:, None] >> shift) & (ng - 1))          # [16][ng]: chunk position of group g of token t
+        idx = pos[None, None, None, :, :, None].expand(B, H, nb, 16, ng, 16)
+        out = []
+        for which in (0, 1):
+            codes = self.blocks[..., which * pk:(which + 1) * pk].reshape(B, H, nb, 16, ng, 16)
+            out.append(torch.gather(codes, 4, idx).reshape(B, H, S, rowb))
+            for is_zero in (0, 1):
+                a = 2 * which + is_zero
+                m = self.blocks[..., 16 * d + a * sz:16 * d + (a + 1) * sz].contiguous().view(torch.float16)
+                out.append(m.reshape(B, H, nb, ng, 16).permute(0, 1, 2, 4, 3).reshape(B, H, S, ng))
+        return tuple(out)
 
 
 def _cs(cache):

@@ -43,6 +43,22 @@ def test_host_side_helpers(lib):
             assert t0 == prev and t1 >= t0 and (t0 % 16 == 0)
             prev = t1
         assert prev == length
+    # block layout: 2560 bytes per 16 tokens at d = 128; the offset helpers cover a block exactly once
+    for d in (64, 128, 256):
+        nbytes = tq.TQ_BLOCK_BYTES(d)
+        assert nbytes == 16 * 2 * tq.tq_cache_bytes(1, 1, 16, d) // 32 == 16 * (d + d // 4)
+        seen = set()
+        for which in (0, 1):
+            for t in range(16):
+                for byte in range(d // 2):
+                    seen.add(tq._lib.tq_cache_code_offset(d, which, t, byte))
+                for g in range(d // 32):
+                    for is_zero in (0, 1):
+                        o = tq._lib.tq_cache_meta_offset(d, which, is_zero, g, t)
+                        seen.update((o, o + 1))
+        assert seen == set(range(nbytes))
+    assert tq._lib.tq_cache_code_offset(128, 0, 0, 5) == 5 and tq._lib.tq_cache_code_offset(128, 1, 0, 0) == 1024
+    assert tq._lib.tq_cache_code_offset(128, 0, 2, 0) == 2 * 64 + 16   # token 2: chunks XOR 1
     c = tq.tq_auto_splits(1, 8, 64, 128, 131072)
     assert 1 <= c <= 256
     assert tq.tq_auto_splits(1, 8, 64, 128, 100) == 1
@@ -54,13 +70,13 @@ def test_argument_validation_without_gpu(lib):
     assert lib.tq_result_string(0) == b"ok"
     assert tq._lib.tq_kv_quantize_append(None, None, None, 1, None, None) == tq.TQ_ERR_NULL
     fake = 0x1000  # never dereferenced: validation fails first
-    cs = tq.tq_kv_cache(fake, fake, fake, fake, fake, fake, fake, 1, 1, 64, 100)   # d = 100
+    cs = tq.tq_kv_cache(fake, fake, 1, 1, 64, 100)   # d = 100
     assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 1, None, None) == tq.TQ_ERR_SHAPE
-    cs = tq.tq_kv_cache(fake, fake, fake, fake, fake, fake, fake, 1, 1, 60, 128)   # S_cap % 16 != 0
+    cs = tq.tq_kv_cache(fake, fake, 1, 1, 60, 128)   # S_cap % 16 != 0
     assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 8, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
-    cs = tq.tq_kv_cache(fake + 8, fake, fake, fake, fake, fake, fake, 1, 1, 64, 128)
+    cs = tq.tq_kv_cache(fake + 8, fake, 1, 1, 64, 128)
     assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 1, None, None) == tq.TQ_ERR_ALIGN
-    cs = tq.tq_kv_cache(fake, fake, fake, fake, fake, fake, fake, 1, 2, 64, 128)
+    cs = tq.tq_kv_cache(fake, fake, 1, 2, 64, 128)
     assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 7, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
     assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 8, 1.0, 300, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
     assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), None, 8, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_NULL

@@ -265,9 +265,7 @@ def test_config5_ragged_batch_64_decode_steps(gpu, oracle):
         k, v = I.make_kv(one, int(lens[b]), seed=500 + b)
         host[b] = oracle.Cache(1, sh.H_kv, S_cap, sh.d)
         host[b].append(k, v)
-        view = tq.tq_kv_cache(dev.k_packed[b].data_ptr(), dev.v_packed[b].data_ptr(), dev.k_scale[b].data_ptr(),
-                              dev.k_zero[b].data_ptr(), dev.v_scale[b].data_ptr(), dev.v_zero[b].data_ptr(),
-                              dev.seq_lens[b:b + 1].data_ptr(), 1, sh.H_kv, S_cap, sh.d)
+        view = tq.tq_kv_cache(dev.blocks[b].data_ptr(), dev.seq_lens[b:b + 1].data_ptr(), 1, sh.H_kv, S_cap, sh.d)
         tq.tq_kv_quantize_append(view, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
     dev.seq_lens.copy_(torch.from_numpy(lens))
     C = tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q, sh.d, S_cap)

@@ -34,8 +34,7 @@ def device_cache(tq, torch, shape, k, v, S_cap, lens=None, fill_byte=None):
     arrays are pre-filled with that byte so rows past the end hold junk (0xFF -> NaN scales)."""
     cache = tq.KVCache(shape.B, shape.H_kv, S_cap, shape.d)
     if fill_byte is not None:
-        for a in cache.arrays():
-            a.view(torch.uint8).fill_(fill_byte)
+        cache.blocks.fill_(fill_byte)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     tq.tq_kv_quantize_append(cache, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
     torch.cuda.synchronize()
