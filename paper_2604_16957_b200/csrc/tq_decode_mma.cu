@@ -392,6 +392,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     cx.vaddr[i] = Cf::PK + vtok * Cf::ROWB + ((vgrp ^ Cf::swz(vtok)) << 4);
   }
   bool timed_out = false;
+#pragma unroll 2  // measured: 34.3 -> 33.3 us per 128K layer (loop overhead shared by two blocks)
   for (int k = 0; k < nblk; ++k) {
     // Wait for this block's bytes.  The wait is bounded: if the copy never completes (which would take
     // a bad pointer), the warp flags the status word and stops consuming.
