@@ -114,7 +114,9 @@ int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t 
 /*
  * Token range of split c of a sequence of `len` tokens cut into C splits (host function): with
  * nb = ceil(len / 16), split c covers tokens [16 * floor(c * nb / C), min(len, 16 * floor((c + 1) * nb / C))).
- * This is the partition tq_sdpa_int4_decode uses; exposed so that partials can be checked.
+ * This is the partition tq_sdpa_int4_decode uses; exposed so that partials can be checked.  With a
+ * sliding window the same rule applies to the blocks that overlap [len - window, len), and the first
+ * split starts at len - window.
  */
 void tq_split_range(int32_t len, int32_t C, int32_t c, int32_t* t0 /* host */, int32_t* t1 /* host */);
 
@@ -137,6 +139,21 @@ void tq_split_range(int32_t len, int32_t C, int32_t c, int32_t* t0 /* host */, i
 int tq_sdpa_int4_decode(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
                         int32_t num_splits, float* o_part, float* m_part, float* l_part, int32_t* status,
                         void* stream);
+
+/*
+ * Phase 1 restricted to a sliding window (Appendix A: Gemma's sliding-attention layers, w = 1024,
+ * "handled by a conditional skip in the inner loop"): sequence b attends only its last `window`
+ * tokens, [max(0, seq_lens[b] - window), seq_lens[b]).  Here the skip is not per token: the splits
+ * partition the window only, so tokens outside it are never fetched.  window = 0 means no window
+ * (identical to tq_sdpa_int4_decode); window < 0 is TQ_ERR_SHAPE.  num_splits = 0 picks
+ * tq_auto_splits(B, H_kv, H_q, d, min(window, S_cap)).  Everything else as tq_sdpa_int4_decode; combine
+ * with tq_sdpa_int4_combine.  tq_split_range_window gives the partition.
+ */
+int tq_sdpa_int4_decode_window(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
+                               int32_t window, int32_t num_splits, float* o_part, float* m_part, float* l_part,
+                               int32_t* status, void* stream);
+void tq_split_range_window(int32_t len, int32_t window, int32_t C, int32_t c, int32_t* t0 /* host */,
+                           int32_t* t1 /* host */);
 
 /*
  * Phase 2, the reduction of Eq. 5:

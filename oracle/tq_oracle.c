@@ -15,6 +15,7 @@
  *   - a literal one-pass transcription of Algorithm 1 in fp64 (used only to pin the above)
  *   - split partials (o_c, m_c, l_c) and their reduction                      (Sec. 3.2, Eq. 5)
  *   - GQA head map kv_head = head / (H_q / H_kv)                              (Sec. 3.1)
+ *   - sliding window: only the last w tokens are attended                     (Appendix A)
  *   - KV cache size model                                                     (Eq. 1, Table 4)
  *
  * Precision: the quantiser is an encoding and runs in IEEE binary32, round-to-nearest-even,
@@ -33,8 +34,9 @@
  * Eq. 1 / Table 4 closed forms; |x - x^| <= s/2; nearest-code brute force; constant groups;
  * softmax weights sum to 1; constant-V, S = 1, q = 0, permutation, split and GQA invariances;
  * Algorithm 1 (literal) against the two-pass definition; a library fp64 attention on the
- * dequantised values.  The bit-level operation ORDER of the quantiser (which of several
- * mathematically equal float32 evaluation orders) is this build's reading and cannot be pinned
+ * dequantised values; the windowed form against full attention over a cache cut to the window.
+ * The bit-level operation ORDER of the quantiser (which of several mathematically equal float32
+ * evaluation orders) is this build's reading and cannot be pinned
  * by the paper, which prints no worked example.
  */
 #include <math.h>
@@ -293,6 +295,23 @@ void tqo_attention(const uint8_t* kp, const uint16_t* ks, const uint16_t* kz, co
     int64_t b = bh / nh, h = h_begin + bh % nh;
     double m, l;
     attend_range(&c, q16, H_q, alpha, b, h, 0, lens[b], out + (b * H_q + h) * d, &m, &l, NULL);
+  }
+}
+
+/* Sliding window (Appendix A): sequence b attends tokens [max(0, lens[b] - window), lens[b]);
+ * window <= 0 means all tokens.  out: [B][H_q][d] fp64. */
+void tqo_attention_window(const uint8_t* kp, const uint16_t* ks, const uint16_t* kz, const uint8_t* vp,
+                          const uint16_t* vs, const uint16_t* vz, const int32_t* lens, int64_t B, int64_t H_kv,
+                          int64_t S_cap, int64_t d, const uint16_t* q16, int64_t H_q, double alpha, int64_t window,
+                          double* out) {
+  tqo_cache c;
+  fill_cache(&c, kp, ks, kz, vp, vs, vz, lens, B, H_kv, S_cap, d);
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t bh = 0; bh < B * H_q; ++bh) {
+    int64_t b = bh / H_q, h = bh % H_q;
+    int64_t begin = (window > 0 && window < lens[b]) ? lens[b] - window : 0;
+    double m, l;
+    attend_range(&c, q16, H_q, alpha, b, h, begin, lens[b], out + (b * H_q + h) * d, &m, &l, NULL);
   }
 }
 

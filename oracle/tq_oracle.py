@@ -151,6 +151,15 @@ def attention(cache: Cache, q: np.ndarray, alpha: float, heads=None) -> np.ndarr
     return out
 
 
+def attention_window(cache: Cache, q: np.ndarray, alpha: float, window: int) -> np.ndarray:
+    """Attention over the last `window` tokens of every sequence (window <= 0: all tokens), fp64."""
+    q = np.ascontiguousarray(q, dtype=np.float16)
+    B, H_q, d = q.shape
+    out = np.zeros((B, H_q, d), np.float64)
+    lib().tqo_attention_window(*cache._cargs(), _p(q), _i64(H_q), C.c_double(alpha), _i64(window), _p(out))
+    return out
+
+
 def attention_weights(cache: Cache, q, alpha, b, h) -> np.ndarray:
     q = np.ascontiguousarray(q, dtype=np.float16)
     w = np.zeros((int(cache.lens[b]),), np.float64)

@@ -93,14 +93,24 @@ int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t 
 }
 
 void tq_split_range(int32_t len, int32_t C, int32_t c, int32_t* t0, int32_t* t1) {
+  tq_split_range_window(len, 0, C, c, t0, t1);
+}
+
+void tq_split_range_window(int32_t len, int32_t window, int32_t C, int32_t c, int32_t* t0, int32_t* t1) {
   int a = 0, b = 0;
-  if (C >= 1 && c >= 0 && c < C) split_range(len, C, c, a, b);
+  if (C >= 1 && c >= 0 && c < C) split_range(window_begin(len, window), len, C, c, a, b);
   if (t0) *t0 = a;
   if (t1) *t1 = b;
 }
 
 int tq_sdpa_int4_decode(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale, int32_t num_splits,
                         float* o_part, float* m_part, float* l_part, int32_t* status, void* stream) {
+  return tq_sdpa_int4_decode_window(cache, q, H_q, attn_scale, 0, num_splits, o_part, m_part, l_part, status, stream);
+}
+
+int tq_sdpa_int4_decode_window(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale, int32_t window,
+                               int32_t num_splits, float* o_part, float* m_part, float* l_part, int32_t* status,
+                               void* stream) {
   if (int r = check_cache(cache)) return r;
   if (!q || !o_part || !m_part || !l_part) return TQ_ERR_NULL;
   if (int r = check_heads(cache, H_q)) return r;
@@ -108,12 +118,14 @@ int tq_sdpa_int4_decode(const tq_kv_cache* cache, const void* q, int32_t H_q, fl
   if (!aligned16(q) || !aligned16(o_part) || (reinterpret_cast<uintptr_t>(m_part) & 3u) ||
       (reinterpret_cast<uintptr_t>(l_part) & 3u) || (reinterpret_cast<uintptr_t>(status) & 3u))
     return TQ_ERR_ALIGN;
-  const int C = num_splits ? num_splits : tq_auto_splits(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
+  if (window < 0) return TQ_ERR_SHAPE;
+  const int span = (window > 0 && window < cache->S_cap) ? window : cache->S_cap;  // most tokens a sequence attends
+  const int C = num_splits ? num_splits : tq_auto_splits(cache->B, cache->H_kv, H_q, cache->d, span);
   auto st = static_cast<cudaStream_t>(stream);
   auto qh = static_cast<const __half*>(q);
   if (use_simple_decode())
-    return finish(launch_decode_simple(*cache, qh, H_q, attn_scale, C, o_part, m_part, l_part, status, st));
-  return finish(launch_decode_mma(*cache, qh, H_q, attn_scale, C, o_part, m_part, l_part, status, st));
+    return finish(launch_decode_simple(*cache, qh, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st));
+  return finish(launch_decode_mma(*cache, qh, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st));
 }
 
 int tq_sdpa_int4_combine(const float* o_part, const float* m_part, const float* l_part, int32_t B, int32_t H_q,

@@ -59,7 +59,7 @@ struct SrcMat {
 template <int D, typename Src>
 __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, const int32_t* seq_lens, int H_kv,
                                                                     int S_cap, const __half* q, int H_q,
-                                                                    float attn_scale, int C, float* o_part,
+                                                                    float attn_scale, int window, int C, float* o_part,
                                                                     float* m_part, float* l_part, int32_t* status) {
   constexpr int EPL = D / 32;
   const int G = H_q / H_kv;
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
   pdl_launch_dependents();
   const int len = checked_len(seq_lens, b, S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
   int t0, t1;
-  split_range(len, C, c, t0, t1);
+  split_range(window_begin(len, window), len, C, c, t0, t1);
   const int h0 = kvh * G + tile * kHeadTile;
   const int nh = min(kHeadTile, G - tile * kHeadTile);
 
@@ -145,12 +145,13 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
 }
 
 template <int D, typename Src>
-cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C,
+cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window,
+                          int C,
                           float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
   const int G = H_q / c.H_kv;
   const int tiles = (G + kHeadTile - 1) / kHeadTile;
   dim3 grid(C, c.H_kv * tiles, c.B);
-  attend_simple_kernel<D, Src><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, attn_scale, C,
+  attend_simple_kernel<D, Src><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, attn_scale, window, C,
                                                              o_part, m_part, l_part, status);
   return cudaGetLastError();
 }
@@ -194,12 +195,12 @@ __global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T
 
 }  // namespace
 
-cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C,
+cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
                                  float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
   auto run = [&](auto dtag) {
     constexpr int D = decltype(dtag)::value;
     SrcInt4<D> src{c.blocks, c.S_cap};
-    return launch_simple<D>(src, c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
+    return launch_simple<D>(src, c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
   };
   switch (c.d) {
     case 64: return run(std::integral_constant<int, 64>{});
@@ -215,7 +216,7 @@ cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, 
     constexpr int D = decltype(dtag)::value;
     using T = decltype(ttag);
     SrcMat<D, T> src{static_cast<const T*>(k_mat), static_cast<const T*>(v_mat)};
-    return launch_simple<D>(src, c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
+    return launch_simple<D>(src, c, q, H_q, attn_scale, 0, C, o_part, m_part, l_part, status, st);
   };
   auto by_d = [&](auto ttag) {
     switch (c.d) {

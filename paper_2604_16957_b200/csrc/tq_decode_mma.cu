@@ -152,9 +152,9 @@ struct WarpCtx {
 };
 
 // One 16-token block: scores -> online softmax -> P.V, all in registers.  TAIL = the block
-// holding the end of the sequence: only its first `valid` tokens count.
+// holding an end of the attended range: only its tokens lo <= t < hi count.
 template <int D, bool TAIL>
-__device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, int valid,
+__device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, int lo, int hi,
                                            const uint32_t (&qf)[D / 32][4], const float (&qs)[D / 32][2],
                                            float (&oacc)[D / 16][4], float (&zacc)[D / 32][4], const float (&zero4)[4], float& m0, float& m1,
                                            float& l0, float& l1) {
@@ -165,7 +165,8 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
     __half* sz = reinterpret_cast<__half*>(const_cast<uint8_t*>(st) + 2 * Cf::PK);
     const int lane = threadIdx.x & 31;
     for (int i = lane; i < 4 * kBlk * NG; i += 32) {
-      if ((i % kBlk) >= valid) sz[i] = __ushort_as_half(0);  // arrays are [group][16 tokens]
+      const int t = i % kBlk;  // arrays are [group][16 tokens]
+      if (t < lo || t >= hi) sz[i] = __ushort_as_half(0);
     }
     __syncwarp();
   }
@@ -209,15 +210,15 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
   float d0 = fmaf(sc[0], cx.cs, -m0), d1 = fmaf(sc[1], cx.cs, -m1);
   float d2 = fmaf(sc[2], cx.cs, -m0), d3 = fmaf(sc[3], cx.cs, -m1);
   if (TAIL) {
-    if (cx.gid >= valid) d0 = d1 = -INFINITY;
-    if (cx.gid + 8 >= valid) d2 = d3 = -INFINITY;
+    if (cx.gid < lo || cx.gid >= hi) d0 = d1 = -INFINITY;
+    if (cx.gid + 8 < lo || cx.gid + 8 >= hi) d2 = d3 = -INFINITY;
   }
   const bool need = fmaxf(fmaxf(d0, d2), fmaxf(d1, d3)) > kRescaleThreshold;
   if (__any_sync(0xffffffffu, need)) {
     float a0 = sc[0] * cx.cs, a1 = sc[1] * cx.cs, a2 = sc[2] * cx.cs, a3 = sc[3] * cx.cs;
     if (TAIL) {
-      if (cx.gid >= valid) a0 = a1 = -INFINITY;
-      if (cx.gid + 8 >= valid) a2 = a3 = -INFINITY;
+      if (cx.gid < lo || cx.gid >= hi) a0 = a1 = -INFINITY;
+      if (cx.gid + 8 < lo || cx.gid + 8 >= hi) a2 = a3 = -INFINITY;
     }
     float bm0 = fmaxf(a0, a2), bm1 = fmaxf(a1, a3);
 #pragma unroll
@@ -275,9 +276,11 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
   }
 }
 
-template <int D>
+// WIN = a sliding window may be set (Appendix A); the instantiation without it carries none of the
+// window arithmetic into the block loop.
+template <int D, bool WIN>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
-    decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, float attn_scale, int C,
+    decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, float attn_scale, int window, int C,
                       float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
                       int32_t* status) {
   using Cf = Cfg<D>;
@@ -294,7 +297,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   pdl_launch_dependents();
   const int len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
   int t0, t1;
-  split_range(len, C, c, t0, t1);
+  split_range(WIN ? window_begin(len, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
 
   // ---- q first (a handful of loads that must not queue behind the cache stream), used further down
   uint4 qraw[NG];
@@ -379,8 +382,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
   // The block that holds the end of the sequence (if this warp owns it) is partial and goes
   // through the masking variant of the step; every other block through the plain one.
+  // Only the two blocks holding the ends of the range [t0, t1) can be partial: the last block of the warp
+  // that owns the end and, under a sliding window, the first block of warp 0 (the window may begin inside it).
   const int rem_last = t1 - (blk0 + warp + (nblk - 1) * kWarps) * kBlk;  // tokens in this warp's last block
   const int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;
+  const bool head = WIN && warp == 0 && (t0 & (kBlk - 1)) != 0 && nblk > 0;
   WarpCtx<D> cx;
   cx.ring = ring; cx.ksz_lane = ksz_lane; cx.vsz_lane = vsz_lane; cx.cs = cs; cx.gid = gid;
 #pragma unroll
@@ -407,10 +413,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
     if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + warp + (k + Cf::NST - 1) * kWarps);
     const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
-    if (k < nfull)
-      block_step<D, false>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, kBlk, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
-    else
-      block_step<D, true>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, rem_last, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
+    if (k < nfull && !(WIN && head && k == 0)) {
+      block_step<D, false>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, 0, kBlk, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
+    } else {
+      int lo = 0, hi = rem_last;
+      if (WIN) {
+        const int first = (blk0 + warp + k * kWarps) * kBlk;  // first token of this block
+        lo = max(t0 - first, 0);
+        hi = min(t1 - first, kBlk);
+      }
+      block_step<D, true>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, lo, hi, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
+    }
   }
   if (timed_out) {
     // Copies of this warp may still be in flight into its ring: give each a bounded time to land before
@@ -496,26 +509,33 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
 }
 
-template <int D>
-cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C, float* o_part,
+template <int D, bool WIN>
+cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C, float* o_part,
                    float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D, WIN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 Cfg<D>::SMEM);
   if (attr != cudaSuccess) return attr;
   const int G = H_q / c.H_kv;
   dim3 grid(C, c.H_kv * ((G + 7) / 8), c.B);
-  return launch_kernel(decode_mma_kernel<D>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, attn_scale, C, o_part,
-                       m_part, l_part, status);
+  return launch_kernel(decode_mma_kernel<D, WIN>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, attn_scale, window,
+                       C, o_part, m_part, l_part, status);
+}
+
+template <int D>
+cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C, float* o_part,
+                   float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+  return window > 0 ? launch<D, true>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st)
+                    : launch<D, false>(c, q, H_q, attn_scale, 0, C, o_part, m_part, l_part, status, st);
 }
 
 }  // namespace
 
-cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C, float* o_part,
-                              float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
+                              float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
   switch (c.d) {
-    case 64: return launch<64>(c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
-    case 128: return launch<128>(c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
-    default: return launch<256>(c, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
+    case 64: return launch<64>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    case 128: return launch<128>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    default: return launch<256>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
   }
 }
 

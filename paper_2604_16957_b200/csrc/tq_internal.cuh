@@ -11,15 +11,25 @@ namespace tq {
 constexpr int kGroup = TQ_GROUP;
 constexpr int kQuantum = TQ_SPLIT_QUANTUM;
 
-// Split partition shared by host and device: split c of C over a sequence of len tokens.
-__host__ __device__ inline void split_range(int len, int C, int c, int& t0, int& t1) {
+// Split partition shared by host and device: split c of C over the attended tokens [begin, len) of a
+// sequence (begin = 0 without a sliding window, max(0, len - window) with one).  Boundaries fall on
+// multiples of 16 tokens except the two ends.
+__host__ __device__ inline void split_range(int begin, int len, int C, int c, int& t0, int& t1) {
   if (len < 0) len = 0;
-  long long nb = (len + kQuantum - 1) / kQuantum;
-  long long b0 = (nb * c) / C, b1 = (nb * (c + 1)) / C;
-  t0 = (int)(b0 * kQuantum);
-  long long e = b1 * kQuantum;
-  t1 = (int)(e < len ? e : len);
-  if (t1 < t0) t1 = t0;
+  if (begin < 0) begin = 0;
+  if (begin > len) begin = len;
+  const long long nb0 = begin / kQuantum, nb1 = (len + kQuantum - 1) / kQuantum;
+  const long long n = nb1 - nb0;
+  const long long b0 = nb0 + (n * c) / C, b1 = nb0 + (n * (c + 1)) / C;
+  long long s = b0 * kQuantum, e = b1 * kQuantum;
+  if (s < begin) s = begin;
+  if (e > len) e = len;
+  if (e < s) e = s;
+  t0 = (int)s;
+  t1 = (int)e;
+}
+__host__ __device__ inline int window_begin(int len, int window) {
+  return (window > 0 && window < len) ? len - window : 0;
 }
 
 // ---- block layout of the cache (see tq.h).  d is 64, 128 or 256.
@@ -84,9 +94,9 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 // host-side launchers (each returns the launch error, if any)
 cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, const __half* v_new, int T,
                                    int32_t* status, cudaStream_t st);
-cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C, float* o_part,
-                              float* m_part, float* l_part, int32_t* status, cudaStream_t st);
-cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int C,
+cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
+                              float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
+cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
                                  float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
 cudaError_t launch_combine(const float* o_part, const float* m_part, const float* l_part, int B, int H_q, int d, int C,
                            void* out, bool out_fp32, cudaStream_t st);

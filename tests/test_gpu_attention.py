@@ -297,3 +297,35 @@ def test_config5_ragged_batch_64_decode_steps(gpu, oracle):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert dev.seq_lens.cpu().tolist() == [int(x) + 64 for x in lens]
+
+
+@pytest.mark.parametrize("d,H_q,H_kv", [(256, 32, 16), (128, 16, 2), (64, 4, 1)])
+def test_sliding_window_decode(gpu, oracle, d, H_q, H_kv):
+    """Appendix A: sliding-window layers (w = 1024 in the paper).  Windows that start inside a 16-token
+    block, are longer than the sequence, are a single token, plus ragged lengths and several split
+    counts; partial ranges are also checked against tq_split_range_window."""
+    tq, torch = gpu
+    sh = I.Shape("x", 4, H_q, H_kv, d, d ** -0.5 if d != 256 else 1.0, sigma_qk=1.0 if d != 256 else 0.25)
+    lens = [3000, 1024, 1029, 7]
+    host, dev = _both(gpu, oracle, sh, 3008, 51, S_cap=3008, lens=lens, fill_byte=0xFF)
+    q = I.make_q(sh, 51)
+    qd = torch.from_numpy(q).cuda()
+    for window, C in ((1024, 0), (1024, 5), (1000, 3), (1, 2), (17, 1), (5000, 4), (0, 2)):
+        ref = oracle.attention_window(host, q, sh.alpha, window)
+        Cn = C or tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q, sh.d, window or 3008)
+        o, m, l = tq.alloc_partials(sh.B, sh.H_q, sh.d, Cn)
+        out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        tq.tq_sdpa_int4_decode_window(dev, qd, sh.alpha, window, C, o, m, l, status)
+        tq.tq_sdpa_int4_combine(o, m, l, out)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert_attention_close(out.cpu().numpy(), ref, f"window {window} C {C}")
+    # the partition covers exactly the window
+    for length, window, Cn in ((3000, 1024, 5), (1029, 1024, 3), (7, 1024, 2), (100, 1, 4)):
+        prev = max(0, length - window)
+        for c in range(Cn):
+            t0, t1 = tq.tq_split_range_window(length, window, Cn, c)
+            assert t0 == prev and t1 >= t0
+            prev = t1
+        assert prev == length

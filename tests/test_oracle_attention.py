@@ -170,3 +170,31 @@ def test_zero_length_sequence_gives_zero(oracle):
     cache = _cache(oracle, sh, 10, 18, lens=[0, 10])
     out = oracle.attention(cache, I.make_q(sh, 18), sh.alpha)
     assert np.all(out[0] == 0) and np.abs(out[1]).max() > 0
+
+
+def test_sliding_window_equals_attention_over_the_last_w_tokens(oracle):
+    sh = I.Shape("t", 2, 4, 2, 64, 0.125)
+    lens = [100, 37]
+    cache = _cache(oracle, sh, 100, 19, lens=lens)
+    q = I.make_q(sh, 19)
+    full = oracle.attention(cache, q, sh.alpha)
+    # a window at least as long as the sequence, or none, changes nothing
+    assert np.array_equal(oracle.attention_window(cache, q, sh.alpha, 0), full)
+    assert np.array_equal(oracle.attention_window(cache, q, sh.alpha, 100), full)
+    assert np.array_equal(oracle.attention_window(cache, q, sh.alpha, 5000), full)
+    vd = oracle.dequant_rows(cache.v_packed, cache.v_scale, cache.v_zero)
+    # window 1: the last token's v^
+    w1 = oracle.attention_window(cache, q, sh.alpha, 1)
+    for b in range(2):
+        for h in range(4):
+            assert np.array_equal(w1[b, h], vd[b, h // 2, lens[b] - 1])
+    # window w: the same as full attention over a cache that holds only the last w tokens
+    for w in (7, 16, 40):
+        cut = oracle.Cache(sh.B, sh.H_kv, 100, sh.d)
+        for b in range(2):
+            n = min(w, lens[b])
+            for dst, src in zip(cut.arrays(), cache.arrays()):
+                dst[b, :, :n] = src[b, :, lens[b] - n:lens[b]]
+            cut.lens[b] = n
+        assert np.abs(oracle.attention_window(cache, q, sh.alpha, w) - oracle.attention(cut, q, sh.alpha)).max() < 1e-12
+        assert np.abs(oracle.attention_window(cache, q, sh.alpha, w) - full).max() > 1e-4
