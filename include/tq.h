@@ -104,9 +104,10 @@ int tq_kv_quantize_append(const tq_kv_cache* cache /* host */, const void* k_new
 
 /*
  * Number of sequence splits C the library would pick for a decode step over sequences of up to
- * `max_seq_len` tokens (host function, no CUDA call).  Chosen from the SM count so that
- * B * H_kv * ceil(G / 8) * C thread blocks fill the GPU in whole waves while every split keeps
- * enough tokens to stream efficiently.  Always in [1, TQ_MAX_SPLITS].
+ * `max_seq_len` tokens (host function, no CUDA call).  Chosen from the SM count: with few
+ * (sequence, KV head) pairs, B * H_kv * ceil(G / 8) * C thread blocks fill the GPU in one wave of
+ * equal splits (at least 512 tokens each); with a batch, in about four waves (splits of at least
+ * 2048 tokens), so that sequences of different lengths even out.  Always in [1, TQ_MAX_SPLITS].
  */
 #define TQ_MAX_SPLITS 256
 int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len);
@@ -154,6 +155,27 @@ int tq_sdpa_int4_decode_window(const tq_kv_cache* cache /* host */, const void* 
                                int32_t* status, void* stream);
 void tq_split_range_window(int32_t len, int32_t window, int32_t C, int32_t c, int32_t* t0 /* host */,
                            int32_t* t1 /* host */);
+
+/*
+ * Phase 1 for several query tokens per sequence (the S_q factor of the grid in Appendix A; speculative or
+ * chunked decode).  The S_q query tokens are the S_q newest tokens of each sequence and must already be in
+ * the cache (one tq_kv_quantize_append with T = S_q).  The paper does not say what each of them attends; here
+ * it is causal: query token s (0 = oldest) attends cached tokens [lo_s, hi_s) with
+ *   hi_s = seq_lens[b] - (S_q - 1 - s),   lo_s = max(0, hi_s - window)   (window = 0: lo_s = 0),
+ * each through its quantised K/V.  A query token with hi_s <= 0 attends nothing and gives o = 0, l = 0.
+ *   q       : device, fp16 [B][S_q][H_q][d]
+ *   o_part  : device, fp32 [B][S_q][H_q][C][d];  m_part, l_part : device, fp32 [B][S_q][H_q][C]
+ * i.e. the layouts of tq_sdpa_int4_decode with S_q * H_q in place of H_q, so tq_sdpa_int4_combine with
+ * H_q' = S_q * H_q reduces them to out [B][S_q][H_q][d].  The (query token, head) pairs that share a KV head
+ * are packed eight to a thread block like plain GQA heads, so S_q * (H_q / H_kv) <= 8 costs one pass over the
+ * cache.  Splits partition the tokens [lo_0, seq_lens[b]); num_splits = 0 picks
+ * tq_auto_splits(B, H_kv, S_q * H_q, d, span).  S_q = 1 is tq_sdpa_int4_decode_window.
+ * Errors as tq_sdpa_int4_decode, plus TQ_ERR_SHAPE for S_q outside 1..TQ_MAX_QUERY_TOKENS.
+ */
+#define TQ_MAX_QUERY_TOKENS 64
+int tq_sdpa_int4_decode_multi(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, int32_t S_q,
+                              float attn_scale, int32_t window, int32_t num_splits, float* o_part, float* m_part,
+                              float* l_part, int32_t* status, void* stream);
 
 /*
  * Phase 2, the reduction of Eq. 5:

@@ -160,6 +160,25 @@ def attention_window(cache: Cache, q: np.ndarray, alpha: float, window: int) -> 
     return out
 
 
+def attention_multi(cache: Cache, q: np.ndarray, alpha: float, window: int = 0) -> np.ndarray:
+    """Several query tokens per sequence, q [B][S_q][H_q][d]: the S_q newest cached tokens as queries.
+    The paper only names the S_q factor (Appendix A); the reading here is causal attention: query token s
+    sees the cache as it was when that token was the newest one, i.e. the first
+    lens[b] - (S_q - 1 - s) tokens (and of those the last `window`, if a window is set).
+    Returns [B][S_q][H_q][d] fp64."""
+    q = np.ascontiguousarray(q, dtype=np.float16)
+    B, S_q, H_q, d = q.shape
+    out = np.zeros((B, S_q, H_q, d), np.float64)
+    full = cache.lens.copy()
+    try:
+        for s in range(S_q):
+            cache.lens[:] = np.maximum(full - (S_q - 1 - s), 0)
+            out[:, s] = attention_window(cache, q[:, s], alpha, window)
+    finally:
+        cache.lens[:] = full
+    return out
+
+
 def attention_weights(cache: Cache, q, alpha, b, h) -> np.ndarray:
     q = np.ascontiguousarray(q, dtype=np.float16)
     w = np.zeros((int(cache.lens[b]),), np.float64)

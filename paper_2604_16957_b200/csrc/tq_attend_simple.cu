@@ -58,31 +58,40 @@ struct SrcMat {
 // grid: (C, H_kv * head_tiles, B); block: kWarps warps.
 template <int D, typename Src>
 __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, const int32_t* seq_lens, int H_kv,
-                                                                    int S_cap, const __half* q, int H_q,
+                                                                    int S_cap, const __half* q, int H_q, int S_q,
                                                                     float attn_scale, int window, int C, float* o_part,
                                                                     float* m_part, float* l_part, int32_t* status) {
   constexpr int EPL = D / 32;
   const int G = H_q / H_kv;
-  const int tiles = (G + kHeadTile - 1) / kHeadTile;
+  const int GV = G * S_q;  // (query token, head) pairs of one KV head: v = s * G + g
+  const int tiles = (GV + kHeadTile - 1) / kHeadTile;
   const int c = blockIdx.x, kvh = blockIdx.y / tiles, tile = blockIdx.y % tiles, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   pdl_wait();
   pdl_launch_dependents();
   const int len = checked_len(seq_lens, b, S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
   int t0, t1;
-  split_range(window_begin(len, window), len, C, c, t0, t1);
-  const int h0 = kvh * G + tile * kHeadTile;
-  const int nh = min(kHeadTile, G - tile * kHeadTile);
+  split_range(query_lo(len, S_q, 0, window), len, C, c, t0, t1);
+  const int v0 = tile * kHeadTile;
+  const int nh = min(kHeadTile, GV - v0);
+  auto q_row = [&](int v) -> long long {  // row of pair v in q and in the partial arrays, [B][S_q][H_q]
+    const int s = v / G;
+    return (static_cast<long long>(b) * S_q + s) * H_q + kvh * G + (v - s * G);
+  };
 
   float qr[kHeadTile][EPL], o[kHeadTile][EPL], m[kHeadTile], l[kHeadTile];
+  int lo[kHeadTile], hi[kHeadTile];  // tokens each pair attends (causal among the S_q query tokens)
 #pragma unroll
   for (int h = 0; h < kHeadTile; ++h) {
     m[h] = -INFINITY;
     l[h] = 0.f;
+    const int s = min((v0 + h) / G, S_q - 1);
+    hi[h] = query_hi(len, S_q, s);
+    lo[h] = window_begin(hi[h], window);
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
       o[h][e] = 0.f;
-      qr[h][e] = h < nh ? __half2float(q[(static_cast<long long>(b) * H_q + h0 + h) * D + lane * EPL + e]) : 0.f;
+      qr[h][e] = h < nh ? __half2float(q[q_row(v0 + h) * D + lane * EPL + e]) : 0.f;
     }
   }
   const long long row0 = (static_cast<long long>(b) * H_kv + kvh) * S_cap;
@@ -93,6 +102,7 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
     src.load(true, row0 + i, lane, vx);
 #pragma unroll
     for (int h = 0; h < kHeadTile; ++h) {
+      if (i < lo[h] || i >= hi[h]) continue;
       float dot = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) dot = fmaf(qr[h][e], kx[e], dot);
@@ -135,7 +145,7 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
         den += f * sm_l[w][h];
       }
     }
-    const long long pidx = (static_cast<long long>(b) * H_q + h0 + h) * C + c;
+    const long long pidx = q_row(v0 + h) * C + c;
     o_part[pidx * D + x] = den > 0.f ? num / den : 0.f;
     if (x == 0) {
       m_part[pidx] = M * kLn2;  // back to natural-log units of attn_scale * q.k
@@ -145,14 +155,14 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
 }
 
 template <int D, typename Src>
-cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window,
-                          int C,
-                          float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  const int G = H_q / c.H_kv;
-  const int tiles = (G + kHeadTile - 1) / kHeadTile;
+cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale,
+                          int window, int C, float* o_part, float* m_part, float* l_part, int32_t* status,
+                          cudaStream_t st) {
+  const int GV = (H_q / c.H_kv) * S_q;
+  const int tiles = (GV + kHeadTile - 1) / kHeadTile;
   dim3 grid(C, c.H_kv * tiles, c.B);
-  attend_simple_kernel<D, Src><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, attn_scale, window, C,
-                                                             o_part, m_part, l_part, status);
+  attend_simple_kernel<D, Src><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, S_q, attn_scale,
+                                                             window, C, o_part, m_part, l_part, status);
   return cudaGetLastError();
 }
 
@@ -195,12 +205,12 @@ __global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T
 
 }  // namespace
 
-cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
-                                 float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
+                                 int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
   auto run = [&](auto dtag) {
     constexpr int D = decltype(dtag)::value;
     SrcInt4<D> src{c.blocks, c.S_cap};
-    return launch_simple<D>(src, c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    return launch_simple<D>(src, c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
   };
   switch (c.d) {
     case 64: return run(std::integral_constant<int, 64>{});
@@ -216,7 +226,7 @@ cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, 
     constexpr int D = decltype(dtag)::value;
     using T = decltype(ttag);
     SrcMat<D, T> src{static_cast<const T*>(k_mat), static_cast<const T*>(v_mat)};
-    return launch_simple<D>(src, c, q, H_q, attn_scale, 0, C, o_part, m_part, l_part, status, st);
+    return launch_simple<D>(src, c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
   };
   auto by_d = [&](auto ttag) {
     switch (c.d) {

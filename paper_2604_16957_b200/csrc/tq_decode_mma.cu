@@ -1,6 +1,7 @@
 // Fused int4 decode attention, phase 1 (Sec. 3.1 Algorithm 1 per split, Sec. 3.2), for sm_100a.
 //
-// One thread block handles one (sequence, KV head, tile of up to 8 query heads, split).  The
+// One thread block handles one (sequence, KV head, tile of up to 8 query heads, split); with several query
+// tokens per sequence the tile holds (query token, head) pairs.  The
 // query heads that share the KV head are packed into the N = 8 dimension of
 // mma.sync.m16n8k16, so every byte of the cache is read from HBM once per head tile.
 // The path is HBM-bound.  The cache is stored in 16-token blocks that are already in the shared-
@@ -151,10 +152,17 @@ struct WarpCtx {
   int gid;
 };
 
-// One 16-token block: scores -> online softmax -> P.V, all in registers.  TAIL = the block
-// holding an end of the attended range: only its tokens lo <= t < hi count.
+// Which tokens of a block count, as rows relative to the block's first token.  Rows >= zrow lie past the
+// end of the sequence and hold unspecified bytes; column j (j = 0, 1: the thread's two score columns, i.e.
+// query heads 2*tid4 + j of the tile) attends rows lo[j] <= row < hi[j].
+struct RowMask {
+  int zrow, lo0, hi0, lo1, hi1;
+};
+
+// One 16-token block: scores -> online softmax -> P.V, all in registers.  TAIL = a block in which
+// some token does not count for some column (an end of the attended range falls inside it).
 template <int D, bool TAIL>
-__device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, int lo, int hi,
+__device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, const RowMask& mk,
                                            const uint32_t (&qf)[D / 32][4], const float (&qs)[D / 32][2],
                                            float (&oacc)[D / 16][4], float (&zacc)[D / 32][4], const float (&zero4)[4], float& m0, float& m1,
                                            float& l0, float& l1) {
@@ -165,8 +173,7 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
     __half* sz = reinterpret_cast<__half*>(const_cast<uint8_t*>(st) + 2 * Cf::PK);
     const int lane = threadIdx.x & 31;
     for (int i = lane; i < 4 * kBlk * NG; i += 32) {
-      const int t = i % kBlk;  // arrays are [group][16 tokens]
-      if (t < lo || t >= hi) sz[i] = __ushort_as_half(0);
+      if ((i % kBlk) >= mk.zrow) sz[i] = __ushort_as_half(0);  // arrays are [group][16 tokens]
     }
     __syncwarp();
   }
@@ -209,16 +216,24 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
   // reference is raised only when some d exceeds the threshold, so the common path is 4 FMAs.
   float d0 = fmaf(sc[0], cx.cs, -m0), d1 = fmaf(sc[1], cx.cs, -m1);
   float d2 = fmaf(sc[2], cx.cs, -m0), d3 = fmaf(sc[3], cx.cs, -m1);
+  // rows gid (d0, d1) and gid + 8 (d2, d3); columns 0 (d0, d2) and 1 (d1, d3)
+  const bool off0 = TAIL && (cx.gid < mk.lo0 || cx.gid >= mk.hi0), off1 = TAIL && (cx.gid < mk.lo1 || cx.gid >= mk.hi1);
+  const bool off2 = TAIL && (cx.gid + 8 < mk.lo0 || cx.gid + 8 >= mk.hi0);
+  const bool off3 = TAIL && (cx.gid + 8 < mk.lo1 || cx.gid + 8 >= mk.hi1);
   if (TAIL) {
-    if (cx.gid < lo || cx.gid >= hi) d0 = d1 = -INFINITY;
-    if (cx.gid + 8 < lo || cx.gid + 8 >= hi) d2 = d3 = -INFINITY;
+    if (off0) d0 = -INFINITY;
+    if (off1) d1 = -INFINITY;
+    if (off2) d2 = -INFINITY;
+    if (off3) d3 = -INFINITY;
   }
   const bool need = fmaxf(fmaxf(d0, d2), fmaxf(d1, d3)) > kRescaleThreshold;
   if (__any_sync(0xffffffffu, need)) {
     float a0 = sc[0] * cx.cs, a1 = sc[1] * cx.cs, a2 = sc[2] * cx.cs, a3 = sc[3] * cx.cs;
     if (TAIL) {
-      if (cx.gid < lo || cx.gid >= hi) a0 = a1 = -INFINITY;
-      if (cx.gid + 8 < lo || cx.gid + 8 >= hi) a2 = a3 = -INFINITY;
+      if (off0) a0 = -INFINITY;
+      if (off1) a1 = -INFINITY;
+      if (off2) a2 = -INFINITY;
+      if (off3) a3 = -INFINITY;
     }
     float bm0 = fmaxf(a0, a2), bm1 = fmaxf(a1, a3);
 #pragma unroll
@@ -276,28 +291,38 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
   }
 }
 
-// WIN = a sliding window may be set (Appendix A); the instantiation without it carries none of the
-// window arithmetic into the block loop.
-template <int D, bool WIN>
+// GEN = the general form: a sliding window (Appendix A) and / or several query tokens per sequence
+// (S_q > 1, the grid's S_q factor in Appendix A).  With S_q query tokens the "heads" of a KV head are its
+// G * S_q (query token, head) pairs, v = s * G + g, packed into MMA columns like plain heads; query token s
+// is the (S_q - 1 - s)-th newest cached token and attends causally: tokens [lo_s, hi_s) with
+// hi_s = len - (S_q - 1 - s), lo_s = max(0, hi_s - window).  The plain instantiation carries none of this
+// arithmetic into the block loop.
+template <int D, bool GEN>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
-    decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, float attn_scale, int window, int C,
-                      float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
+    decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, int S_q, float attn_scale, int window,
+                      int C, float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
                       int32_t* status) {
   using Cf = Cfg<D>;
   constexpr int NG = Cf::NG;
   extern __shared__ __align__(1024) uint8_t smem[];
 
   const int G = H_q / cache.H_kv;
-  const int tiles = (G + 7) >> 3;
+  const int GV = GEN ? G * S_q : G;  // columns of this KV head
+  const int tiles = (GV + 7) >> 3;
   const int c = blockIdx.x, kvh = blockIdx.y / tiles, tile = blockIdx.y - kvh * tiles, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tid4 = lane & 3;
-  const int h0 = kvh * G + tile * 8;         // first query head of this tile
-  const int nh = min(8, G - tile * 8);       // heads in the tile; the rest of N = 8 is zero padding
+  const int v0 = tile * 8;                   // first column of this tile
+  const int nh = min(8, GV - v0);            // columns in the tile; the rest of N = 8 is zero padding
+  // row of column v in q and in the partial arrays: [B][S_q][H_q]
+  auto q_row = [&](int v) -> long long {
+    const int s = GEN ? v / G : 0;
+    return (static_cast<long long>(b) * (GEN ? S_q : 1) + s) * H_q + kvh * G + (v - s * G);
+  };
   pdl_wait();  // nothing global is read before this point
   pdl_launch_dependents();
   const int len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
   int t0, t1;
-  split_range(WIN ? window_begin(len, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
+  split_range(GEN ? query_lo(len, S_q, 0, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
 
   // ---- q first (a handful of loads that must not queue behind the cache stream), used further down
   uint4 qraw[NG];
@@ -305,11 +330,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   for (int g = 0; g < NG; ++g) {
     qraw[g] = make_uint4(0, 0, 0, 0);
     if (gid < nh)
-      qraw[g] = *reinterpret_cast<const uint4*>(q + (static_cast<long long>(b) * H_q + h0 + gid) * D + g * 32 + tid4 * 8);
+      qraw[g] = *reinterpret_cast<const uint4*>(q + q_row(v0 + gid) * D + g * 32 + tid4 * 8);
   }
 
   // ---- this warp's token blocks: blk0 + warp, blk0 + warp + kWarps, ...
-  const int blk0 = t0 / kBlk, blk1 = (t1 + kBlk - 1) / kBlk;
+  const int blk0 = t0 / kBlk, blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
   const int nblk = blk1 - blk0 > warp ? (blk1 - blk0 - warp + kWarps - 1) / kWarps : 0;
   const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
   uint8_t* const ring = smem + warp * (Cf::NST * Cf::STAGE);
@@ -337,7 +362,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     if (s < nblk) issue(s, blk0 + warp + s * kWarps);
 
 
-  // ---- q as MMA B fragments: column n = gid is head h0 + gid; k slots follow the nibble order.
+  // ---- q as MMA B fragments: column n = gid is column v0 + gid of the tile; k slots follow the nibble order.
   // qs[g][j] = 2^-24 * sum of q over group g for heads 2*tid4 + j (the zero-point term of the scores).
   uint32_t qf[NG][4];
   float qs[NG][2];
@@ -380,13 +405,23 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const uint32_t ksz_lane = 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32;
   const uint32_t vsz_lane = 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16;
 
-  // The block that holds the end of the sequence (if this warp owns it) is partial and goes
-  // through the masking variant of the step; every other block through the plain one.
-  // Only the two blocks holding the ends of the range [t0, t1) can be partial: the last block of the warp
-  // that owns the end and, under a sliding window, the first block of warp 0 (the window may begin inside it).
+  // Blocks in which every token counts for every column go through the plain step, the others through the
+  // masking one.  Plain decode: only the block holding the end of the sequence is partial.  General form:
+  // blocks that reach beyond the oldest query's end, or begin before the newest query's window start.
   const int rem_last = t1 - (blk0 + warp + (nblk - 1) * kWarps) * kBlk;  // tokens in this warp's last block
-  const int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;
-  const bool head = WIN && warp == 0 && (t0 & (kBlk - 1)) != 0 && nblk > 0;
+  int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;           // this warp's blocks k < nfull are full
+  int nhead = 0;                                                         // ... and blocks k < nhead are masked
+  int lo0 = 0, hi0 = 0, lo1 = 0, hi1 = 0;                                // token ranges of this thread's two columns
+  if (GEN) {
+    const int s0 = min((v0 + 2 * tid4) / G, S_q - 1), s1 = min((v0 + 2 * tid4 + 1) / G, S_q - 1);
+    hi0 = query_hi(len, S_q, s0); lo0 = window_begin(hi0, window);
+    hi1 = query_hi(len, S_q, s1); lo1 = window_begin(hi1, window);
+    const int full_end = min(t1, query_hi(len, S_q, 0)) >> 4;                   // blocks below it end inside every range
+    const int full_begin = (query_lo(len, S_q, S_q - 1, window) + kBlk - 1) >> 4;  // blocks from it on begin inside
+    const int first_blk = blk0 + warp;
+    nfull = full_end > first_blk ? min(nblk, (full_end - first_blk + kWarps - 1) / kWarps) : 0;
+    nhead = full_begin > first_blk ? min(nblk, (full_begin - first_blk + kWarps - 1) / kWarps) : 0;
+  }
   WarpCtx<D> cx;
   cx.ring = ring; cx.ksz_lane = ksz_lane; cx.vsz_lane = vsz_lane; cx.cs = cs; cx.gid = gid;
 #pragma unroll
@@ -413,16 +448,16 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
     if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + warp + (k + Cf::NST - 1) * kWarps);
     const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
-    if (k < nfull && !(WIN && head && k == 0)) {
-      block_step<D, false>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, 0, kBlk, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
+    if (k < nfull && !(GEN && k < nhead)) {
+      const RowMask all{kBlk, 0, kBlk, 0, kBlk};
+      block_step<D, false>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, all, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
     } else {
-      int lo = 0, hi = rem_last;
-      if (WIN) {
+      RowMask mk{rem_last, 0, rem_last, 0, rem_last};
+      if (GEN) {
         const int first = (blk0 + warp + k * kWarps) * kBlk;  // first token of this block
-        lo = max(t0 - first, 0);
-        hi = min(t1 - first, kBlk);
+        mk = RowMask{t1 - first, lo0 - first, min(hi0, t1) - first, lo1 - first, min(hi1, t1) - first};
       }
-      block_step<D, true>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, lo, hi, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
+      block_step<D, true>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, mk, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
     }
   }
   if (timed_out) {
@@ -492,7 +527,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   __syncthreads();
   for (int idx = threadIdx.x; idx < nh * D; idx += kThreads) {  // coalesced: one head row after the other
     const int h = idx / D, x = idx - h * D;
-    const long long pidx = (static_cast<long long>(b) * H_q + h0 + h) * C + c;
+    const long long pidx = q_row(v0 + h) * C + c;
     o_part[pidx * D + x] = tb[h * kRowPitch + x];
   }
   if (warp == 0 && gid == 0) {  // lanes 0..3 hold heads 2*tid4, 2*tid4+1
@@ -501,7 +536,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       const int h = 2 * tid4 + j;
       if (h < nh) {
         const float den = j ? den1 : den0, M = j ? M1 : M0;
-        const long long pidx = (static_cast<long long>(b) * H_q + h0 + h) * C + c;
+        const long long pidx = q_row(v0 + h) * C + c;
         m_part[pidx] = den > 0.f ? M * kLn2 : -INFINITY;  // natural-log units of attn_scale * q.k^
         l_part[pidx] = den;
       }
@@ -509,33 +544,33 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
 }
 
-template <int D, bool WIN>
-cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C, float* o_part,
-                   float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D, WIN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <int D, bool GEN>
+cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
+                   float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 Cfg<D>::SMEM);
   if (attr != cudaSuccess) return attr;
-  const int G = H_q / c.H_kv;
-  dim3 grid(C, c.H_kv * ((G + 7) / 8), c.B);
-  return launch_kernel(decode_mma_kernel<D, WIN>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, attn_scale, window,
-                       C, o_part, m_part, l_part, status);
+  const int GV = (H_q / c.H_kv) * S_q;
+  dim3 grid(C, c.H_kv * ((GV + 7) / 8), c.B);
+  return launch_kernel(decode_mma_kernel<D, GEN>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, S_q, attn_scale,
+                       window, C, o_part, m_part, l_part, status);
 }
 
 template <int D>
-cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C, float* o_part,
-                   float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  return window > 0 ? launch<D, true>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st)
-                    : launch<D, false>(c, q, H_q, attn_scale, 0, C, o_part, m_part, l_part, status, st);
+cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
+                   float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+  return (window > 0 || S_q > 1) ? launch<D, true>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st)
+                                 : launch<D, false>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
 }
 
 }  // namespace
 
-cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
-                              float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
+                              int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
   switch (c.d) {
-    case 64: return launch<64>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
-    case 128: return launch<128>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
-    default: return launch<256>(c, q, H_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    default: return launch<256>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
   }
 }
 

@@ -32,6 +32,16 @@ __host__ __device__ inline int window_begin(int len, int window) {
   return (window > 0 && window < len) ? len - window : 0;
 }
 
+// Several query tokens per sequence (S_q >= 1): query token s is the (S_q - 1 - s)-th newest cached token and
+// attends causally the tokens [query_lo, query_hi).
+__host__ __device__ inline int query_hi(int len, int S_q, int s) {
+  const int hi = len - (S_q - 1 - s);
+  return hi > 0 ? hi : 0;
+}
+__host__ __device__ inline int query_lo(int len, int S_q, int s, int window) {
+  return window_begin(query_hi(len, S_q, s), window);
+}
+
 // ---- block layout of the cache (see tq.h).  d is 64, 128 or 256.
 __host__ __device__ inline int block_bytes(int d) { return 16 * (d + d / 4); }
 __host__ __device__ inline int swizzle_term(int d, int t) {
@@ -94,10 +104,10 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 // host-side launchers (each returns the launch error, if any)
 cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, const __half* v_new, int T,
                                    int32_t* status, cudaStream_t st);
-cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
-                              float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
-cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, float attn_scale, int window, int C,
-                                 float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
+cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
+                              int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
+cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
+                                 int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
 cudaError_t launch_combine(const float* o_part, const float* m_part, const float* l_part, int B, int H_q, int d, int C,
                            void* out, bool out_fp32, cudaStream_t st);
 cudaError_t launch_dequant(const tq_kv_cache& c, void* k_mat, void* v_mat, bool fp32, cudaStream_t st);

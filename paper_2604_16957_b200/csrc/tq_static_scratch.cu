@@ -78,7 +78,7 @@ extern "C" int tq_sdpa_int4_attend_static(const tq_kv_cache* cache, const void* 
   auto st = static_cast<cudaStream_t>(stream);
   // Every partial of every (sequence, head, split) is written by phase 1, empty splits included, so
   // nothing in the scratch has to be cleared between calls.
-  e = launch_decode_mma(*cache, static_cast<const __half*>(q), H_q, attn_scale, 0, C, o_part, m_part, l_part, status, st);
+  e = launch_decode_mma(*cache, static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
   if (e != cudaSuccess) return TQ_ERR_CUDA;
   e = launch_combine(o_part, m_part, l_part, cache->B, H_q, d, C, out, out_is_fp32 != 0, st);
   return e == cudaSuccess ? TQ_OK : TQ_ERR_CUDA;

@@ -329,3 +329,37 @@ def test_sliding_window_decode(gpu, oracle, d, H_q, H_kv):
             assert t0 == prev and t1 >= t0
             prev = t1
         assert prev == length
+
+
+@pytest.mark.parametrize("d,H_q,H_kv,S_q", [(256, 32, 16, 4), (128, 64, 8, 3), (64, 4, 1, 5), (128, 8, 4, 16)])
+@pytest.mark.parametrize("impl", ["mma", "simple"])
+def test_multi_query_decode(gpu, oracle, d, H_q, H_kv, S_q, impl):
+    """Several query tokens per sequence (the S_q factor of Appendix A), causal among themselves, with and
+    without a sliding window: one tile (G * S_q = 8), several tiles, a partly filled last tile; lengths
+    whose newest S_q tokens straddle a 16-token block, and a sequence shorter than S_q."""
+    tq, torch = gpu
+    sh = I.Shape("x", 4, H_q, H_kv, d, d ** -0.5 if d != 256 else 1.0, sigma_qk=1.0 if d != 256 else 0.25)
+    lens = [2000, 1026, 2, 48]
+    host, dev = _both(gpu, oracle, sh, 2000, 61, S_cap=2000, lens=lens, fill_byte=0xFF)
+    q = np.ascontiguousarray(np.stack([I.make_q(sh, 61, stream=s) for s in range(S_q)], axis=1))
+    qd = torch.from_numpy(q).cuda()
+    if impl == "simple":
+        os.environ["TQ_DECODE_IMPL"] = "simple"
+    try:
+        for window, C in ((0, 0), (0, 3), (1024, 0), (20, 2), (1, 1)):
+            ref = oracle.attention_multi(host, q, sh.alpha, window)
+            Cn = C or tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q * S_q, sh.d, window or 2000)
+            o, m, l = tq.alloc_partials(sh.B, sh.H_q * S_q, sh.d, Cn)
+            out = torch.empty((sh.B, S_q, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            tq.tq_sdpa_int4_decode_multi(dev, qd, sh.alpha, window, C, o, m, l, status)
+            tq.tq_sdpa_int4_combine(o, m, l, out.view(sh.B, S_q * sh.H_q, sh.d))
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            got = out.cpu().numpy()
+            for s in range(S_q):  # query tokens older than the sequence attend nothing
+                if 2 - (S_q - 1 - s) <= 0:
+                    assert not got[2, s].any() and not ref[2, s].any()
+            assert_attention_close(got.reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d), f"S_q {S_q} window {window} C {C}")
+    finally:
+        os.environ.pop("TQ_DECODE_IMPL", None)

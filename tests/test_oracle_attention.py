@@ -198,3 +198,35 @@ def test_sliding_window_equals_attention_over_the_last_w_tokens(oracle):
             cut.lens[b] = n
         assert np.abs(oracle.attention_window(cache, q, sh.alpha, w) - oracle.attention(cut, q, sh.alpha)).max() < 1e-12
         assert np.abs(oracle.attention_window(cache, q, sh.alpha, w) - full).max() > 1e-4
+
+
+def test_multi_query_is_causal_attention_of_each_query_token(oracle):
+    sh = I.Shape("t", 2, 4, 2, 64, 0.125)
+    lens = [60, 2]
+    cache = _cache(oracle, sh, 64, 23, lens=lens)
+    S_q = 3
+    q = np.stack([I.make_q(sh, 23, stream=s) for s in range(S_q)], axis=1)  # [B][S_q][H_q][d]
+    out = oracle.attention_multi(cache, q, sh.alpha)
+    assert np.array_equal(cache.lens, np.array(lens, np.int32))  # the lengths are restored
+    # the newest query token sees everything; one query token is plain attention
+    assert np.array_equal(out[:, S_q - 1], oracle.attention(cache, q[:, S_q - 1], sh.alpha))
+    assert np.array_equal(oracle.attention_multi(cache, q[:, :1], sh.alpha)[:, 0], oracle.attention(cache, q[:, 0], sh.alpha))
+    # query token s: brute force over the first len - (S_q - 1 - s) tokens from the dequantised cache
+    kd = oracle.dequant_rows(cache.k_packed, cache.k_scale, cache.k_zero)
+    vd = oracle.dequant_rows(cache.v_packed, cache.v_scale, cache.v_zero)
+    for b in range(2):
+        for s in range(S_q):
+            n = max(lens[b] - (S_q - 1 - s), 0)
+            for h in range(4):
+                if n == 0:
+                    assert not out[b, s, h].any()
+                    continue
+                a = sh.alpha * kd[b, h // 2, :n] @ q[b, s, h].astype(np.float64)
+                w = np.exp(a - a.max())
+                ref = (w / w.sum()) @ vd[b, h // 2, :n]
+                assert np.abs(out[b, s, h] - ref).max() < 1e-12
+    # with a window, the same over the last w of those tokens
+    outw = oracle.attention_multi(cache, q, sh.alpha, window=10)
+    a = sh.alpha * kd[0, 1, 48:58] @ q[0, 0, 3].astype(np.float64)
+    w = np.exp(a - a.max())
+    assert np.abs(outw[0, 0, 3] - (w / w.sum()) @ vd[0, 1, 48:58]).max() < 1e-12
