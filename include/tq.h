@@ -67,13 +67,14 @@ typedef enum tq_result {
  *     K codes | V codes | K scales | K zeros | V scales | V zeros
  *   codes (16 * d/2 bytes each): token t of the block is the d/2-byte row t; inside a row the 16-byte
  *     chunks (32 codes = one group each) are stored in XOR-swizzled order: group g of token t sits at
- *     chunk position g ^ ((t >> shift) & (d/32 - 1)), shift = 2, 1, 0 for d = 64, 128, 256 -- the
+ *     chunk position g ^ ((t >> shift) & (d/32 - 1)), shift = 2, 1, 0, 0 for d = 64, 128, 256, 512 -- the
  *     bank-conflict-free shared-memory layout, kept in global memory so that no rearrangement is
  *     needed on the way in.  Within a chunk, element 2i is the low nibble of byte i.
  *   scales, zeros (d/32 * 16 fp16 each): value of (group g, token t) at index g * 16 + t.
  * Use tq_cache_code_offset / tq_cache_meta_offset to address single elements from the host.
  * Rows at or beyond seq_lens[b] are unspecified.
- * Requirements: d in {64, 128, 256}; S_cap a positive multiple of 16; B, H_kv >= 1.
+ * Requirements: d in {64, 128, 256, 512} (512: the paper's Gemma global layers, Table 7); S_cap a
+ * positive multiple of 16; B, H_kv >= 1.
  */
 #define TQ_BLOCK_TOKENS 16
 #define TQ_BLOCK_BYTES(d) (16 * ((d) + (d) / 4))
@@ -182,7 +183,7 @@ int tq_sdpa_int4_decode_multi(const tq_kv_cache* cache /* host */, const void* q
  *   out[b][h][:] = sum_c w_c * o_part[b][h][c][:] / sum_c w_c,   w_c = l_c * exp(m_c - max_c m_c),
  * skipping splits with l_c = 0; if all are empty the output row is zero.
  *   out : [B][H_q][d], fp16 (out_is_fp32 = 0) or fp32 (out_is_fp32 = 1).
- * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE (B, H_q, num_splits < 1, d not a multiple of 32 or > 256), TQ_ERR_ALIGN,
+ * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE (B, H_q, num_splits < 1, d not a multiple of 32 or > 512), TQ_ERR_ALIGN,
  * TQ_ERR_CUDA.
  */
 int tq_sdpa_int4_combine(const float* o_part, const float* m_part, const float* l_part, int32_t B, int32_t H_q,

@@ -36,7 +36,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 int check_cache(const tq_kv_cache* c) {
   if (!c) return TQ_ERR_NULL;
   if (!c->blocks || !c->seq_lens) return TQ_ERR_NULL;
-  if (!(c->d == 64 || c->d == 128 || c->d == 256)) return TQ_ERR_SHAPE;
+  if (!(c->d == 64 || c->d == 128 || c->d == 256 || c->d == 512)) return TQ_ERR_SHAPE;
   if (c->B < 1 || c->B > 65535 || c->H_kv < 1 || c->H_kv > 4096 || c->S_cap < 16 || (c->S_cap % 16) != 0)
     return TQ_ERR_SHAPE;
   if (!aligned16(c->blocks) || (reinterpret_cast<uintptr_t>(c->seq_lens) & 3u)) return TQ_ERR_ALIGN;
@@ -151,7 +151,7 @@ int tq_sdpa_int4_decode_multi(const tq_kv_cache* cache, const void* q, int32_t H
 int tq_sdpa_int4_combine(const float* o_part, const float* m_part, const float* l_part, int32_t B, int32_t H_q,
                          int32_t d, int32_t num_splits, void* out, int32_t out_is_fp32, void* stream) {
   if (!o_part || !m_part || !l_part || !out) return TQ_ERR_NULL;
-  if (B < 1 || H_q < 1 || num_splits < 1 || num_splits > TQ_MAX_SPLITS || d < 32 || d > 256 || (d % 32) != 0 ||
+  if (B < 1 || H_q < 1 || num_splits < 1 || num_splits > TQ_MAX_SPLITS || d < 32 || d > 512 || (d % 32) != 0 ||
       static_cast<long long>(B) * H_q > 0x7fffffffLL)
     return TQ_ERR_SHAPE;
   if (!aligned16(o_part) || !aligned16(out) || (reinterpret_cast<uintptr_t>(m_part) & 3u) ||

@@ -16,7 +16,11 @@ namespace tq {
 namespace {
 
 constexpr int kWarps = 4;
-constexpr int kHeadTile = 8;
+// (query token, head) pairs per thread block: 8, or 4 at d = 512 where a pair's registers double
+template <int D>
+struct HeadTile {
+  static constexpr int value = D > 256 ? 4 : 8;
+};
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -62,6 +66,7 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
                                                                     float attn_scale, int window, int C, float* o_part,
                                                                     float* m_part, float* l_part, int32_t* status) {
   constexpr int EPL = D / 32;
+  constexpr int kHeadTile = HeadTile<D>::value;
   const int G = H_q / H_kv;
   const int GV = G * S_q;  // (query token, head) pairs of one KV head: v = s * G + g
   const int tiles = (GV + kHeadTile - 1) / kHeadTile;
@@ -158,6 +163,7 @@ template <int D, typename Src>
 cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale,
                           int window, int C, float* o_part, float* m_part, float* l_part, int32_t* status,
                           cudaStream_t st) {
+  constexpr int kHeadTile = HeadTile<D>::value;
   const int GV = (H_q / c.H_kv) * S_q;
   const int tiles = (GV + kHeadTile - 1) / kHeadTile;
   dim3 grid(C, c.H_kv * tiles, c.B);
@@ -215,6 +221,7 @@ cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q,
   switch (c.d) {
     case 64: return run(std::integral_constant<int, 64>{});
     case 128: return run(std::integral_constant<int, 128>{});
+    case 512: return run(std::integral_constant<int, 512>{});
     default: return run(std::integral_constant<int, 256>{});
   }
 }
@@ -232,6 +239,7 @@ cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, 
     switch (c.d) {
       case 64: return run(std::integral_constant<int, 64>{}, ttag);
       case 128: return run(std::integral_constant<int, 128>{}, ttag);
+      case 512: return run(std::integral_constant<int, 512>{}, ttag);
       default: return run(std::integral_constant<int, 256>{}, ttag);
     }
   };

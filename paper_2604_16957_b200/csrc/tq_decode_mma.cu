@@ -8,7 +8,8 @@
 // memory layout this kernel wants (tq.h), so a stage is filled by ONE bulk asynchronous copy
 // (cp.async.bulk, the TMA unit) of a contiguous 2560-byte block (d = 128) issued by one lane and
 // completing on the stage's mbarrier.  Each warp owns a ring of 4 stages and its tokens end to
-// end, so the main loop has no block-wide barrier.  Measured on the 128K Llama-shaped layer, the
+// end, so the main loop has no block-wide barrier.  (Head dimensions 256 and 512 are split over teams
+// of 2 and 4 warps that share a ring and exchange their partial scores once per token block.)  Measured on the 128K Llama-shaped layer, the
 // copies alone take 27.9 us with bulk copies against 30.2 us with 16-byte cp.async.  The tensor
 // cores only take the G-packed q.K^T and P.V contractions off the CUDA cores, which could not
 // keep up with the memory system otherwise.
@@ -64,14 +65,24 @@ struct Cfg {
   static constexpr int PK = kBlk * ROWB;            // code bytes per stage, K or V
   static constexpr int SWZ_SHIFT = NG == 2 ? 2 : (NG == 4 ? 1 : 0);  // chunk' = chunk ^ ((tok >> SHIFT) & (NG - 1))
   static constexpr int SZ = kBlk * NG * 2;          // bytes of one scale or zero array per stage
-  static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1280 / 2560 / 5120 bytes
-  static constexpr int NST = 4;                     // stages in the per-warp ring (power of two)
-  static constexpr int MINB = D == 256 ? 1 : 2;     // resident blocks per SM
-  static constexpr int PIPE = kWarps * NST * STAGE; // 40 KB (D = 64), 80 KB (128), 160 KB (256)
-  static constexpr int MERGE = (kWarps * 16 + kWarps * D * 10 + 8 * (D + 4)) * 4;
-  static constexpr int BARS = PIPE > MERGE ? PIPE : MERGE;  // offset of the mbarriers: [kWarps][NST] x 8 bytes
-  static constexpr int SMEM = BARS + kWarps * NST * 8;
+  static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1280 / 2560 / 5120 / 10240 bytes
+  static constexpr int NST = 4;                     // stages in a ring (power of two)
+  // Head dimensions above 128 are split over DS warps (a "team") that work on the same token block, each
+  // on DW = 128 channels: the accumulators of one warp stay within 128 registers per thread, so two
+  // blocks fit an SM at every head dimension.  A team owns one ring; the kernel has NTEAM teams.
+  static constexpr int DS = D <= 128 ? 1 : D / 128;
+  static constexpr int DW = D / DS;                 // channels per warp
+  static constexpr int NGW = DW / 32;               // groups per warp
+  static constexpr int NTEAM = kWarps / DS;
+  static constexpr int MINB = 2;                    // resident blocks per SM
+  static constexpr int PIPE = NTEAM * NST * STAGE;  // 40 KB (D = 64), 80 KB otherwise
+  static constexpr int MERGE = (NTEAM * 16 + NTEAM * D * 10 + 8 * (D + 4)) * 4;
+  static constexpr int BARS = PIPE > MERGE ? PIPE : MERGE;  // offset of the mbarriers: [NTEAM][NST] x 8 bytes
+  static constexpr int XCH = BARS + NTEAM * NST * 8;        // score exchange of the teams: [NTEAM][2][DS][32] float4 + flags
+  static constexpr int XCH_TEAM = DS > 1 ? 2 * DS * 32 * 16 + 2 * DS * 4 : 0;
+  static constexpr int SMEM = XCH + NTEAM * XCH_TEAM;
   static_assert(STAGE == TQ_BLOCK_BYTES(D), "a stage is one cache block");
+  static_assert(kWarps % DS == 0 && XCH % 16 == 0, "teams tile the block");
   __host__ __device__ static constexpr int swz(int tok) { return (tok >> SWZ_SHIFT) & (NG - 1); }
 };
 
@@ -145,8 +156,8 @@ __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_c
 template <int D>
 struct WarpCtx {
   uint8_t* ring;
-  uint32_t kaddr[D / 64];  // ldmatrix row address (offset in a stage) this lane supplies, per K load
-  uint32_t vaddr[D / 64];  // same for the V loads
+  uint32_t kaddr[Cfg<D>::NGW / 2];  // ldmatrix row address (offset in a stage) this lane supplies, per K load
+  uint32_t vaddr[Cfg<D>::NGW / 2];  // same for the V loads
   uint32_t ksz_lane, vsz_lane;
   float cs;
   int gid;
@@ -159,59 +170,63 @@ struct RowMask {
   int zrow, lo0, hi0, lo1, hi1;
 };
 
-// One 16-token block: scores -> online softmax -> P.V, all in registers.  TAIL = a block in which
-// some token does not count for some column (an end of the attended range falls inside it).
+// First half of one 16-token block: this warp's share of the scores S[token][head] (over its DW channels;
+// they carry a factor 2^-24).  TAIL = a block in which some token does not count for some column.
 template <int D, bool TAIL>
-__device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, const RowMask& mk,
-                                           const uint32_t (&qf)[D / 32][4], const float (&qs)[D / 32][2],
-                                           float (&oacc)[D / 16][4], float (&zacc)[D / 32][4], const float (&zero4)[4], float& m0, float& m1,
-                                           float& l0, float& l1) {
+__device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, const RowMask& mk,
+                                             const uint32_t (&qf)[Cfg<D>::NGW][4], const float (&qs)[Cfg<D>::NGW][2],
+                                             const float (&zero4)[4], float (&sc)[4]) {
   using Cf = Cfg<D>;
-  constexpr int NG = Cf::NG;
+  constexpr int NGW = Cf::NGW;
   if (TAIL) {
     // rows past the end hold unspecified bytes: give them scale = zero = 0 so they dequantise to 0
+    // (every warp of a team clears all of them before its own reads; the stores are idempotent)
     __half* sz = reinterpret_cast<__half*>(const_cast<uint8_t*>(st) + 2 * Cf::PK);
     const int lane = threadIdx.x & 31;
-    for (int i = lane; i < 4 * kBlk * NG; i += 32) {
+    for (int i = lane; i < 4 * kBlk * Cf::NG; i += 32) {
       if ((i % kBlk) >= mk.zrow) sz[i] = __ushort_as_half(0);  // arrays are [group][16 tokens]
     }
     __syncwarp();
   }
-
-  // ---------------- scores: S[token][head] over this block's 16 tokens (carry a factor 2^-24)
-  float sc[4];
-  {
-    // matrix j = 4 * i + m of load i is (tokens 8 * (j / NG) .., group j % NG)
-    uint32_t kw[NG / 2][4], ksz[4];
+  // matrix j = 4 * i + m of load i is (tokens 8 * (j / NGW) .., group j % NGW of this warp)
+  uint32_t kw[NGW / 2][4], ksz[4];
 #pragma unroll
-    for (int i = 0; i < NG / 2; ++i) ldmatrix_x4(kw[i], st_s + cx.kaddr[i]);
+  for (int i = 0; i < NGW / 2; ++i) ldmatrix_x4(kw[i], st_s + cx.kaddr[i]);
 #pragma unroll
-    for (int g = 0; g < NG; ++g) {
-      const uint32_t w0 = kw[g / 4][g % 4];                      // token gid
-      const uint32_t w8 = kw[(NG + g) / 4][(NG + g) % 4];        // token gid + 8
-      float acc[4];
-      mma16816_first(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1], zero4);
-      const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
-      mma16816(acc, y0 & kMaskLo, y8 & kMaskLo, y0 & kMaskHi, y8 & kMaskHi, qf[g][2], qf[g][3]);
-      // Scales and zeros of tokens gid and gid + 8 for groups g, g+1 by one transposing ldmatrix: its
-      // matrices are (scale | tokens 0-7), (scale | 8-15), (zero | 0-7), (zero | 8-15), each with rows
-      // alternating between the 16-byte chunks of groups g and g+1, so every lane receives element gid
-      // of both chunks: half2 (x[g][token], x[g+1][token]).
-      if ((g & 1) == 0) ldmatrix_x4_trans(ksz, st_s + cx.ksz_lane + 32 * g);
-      const float s_lo = (g & 1) ? __high2float(u32_as_h2(ksz[0])) : __low2float(u32_as_h2(ksz[0]));
-      const float s_hi = (g & 1) ? __high2float(u32_as_h2(ksz[1])) : __low2float(u32_as_h2(ksz[1]));
-      const float z_lo = (g & 1) ? __high2float(u32_as_h2(ksz[2])) : __low2float(u32_as_h2(ksz[2]));
-      const float z_hi = (g & 1) ? __high2float(u32_as_h2(ksz[3])) : __low2float(u32_as_h2(ksz[3]));
-      const float t0 = fmaf(-z_lo, qs[g][0], acc[0]), t1 = fmaf(-z_lo, qs[g][1], acc[1]);
-      const float t2 = fmaf(-z_hi, qs[g][0], acc[2]), t3 = fmaf(-z_hi, qs[g][1], acc[3]);
-      if (g == 0) {
-        sc[0] = s_lo * t0; sc[1] = s_lo * t1; sc[2] = s_hi * t2; sc[3] = s_hi * t3;
-      } else {
-        sc[0] = fmaf(s_lo, t0, sc[0]); sc[1] = fmaf(s_lo, t1, sc[1]);
-        sc[2] = fmaf(s_hi, t2, sc[2]); sc[3] = fmaf(s_hi, t3, sc[3]);
-      }
+  for (int g = 0; g < NGW; ++g) {
+    const uint32_t w0 = kw[g / 4][g % 4];                      // token gid
+    const uint32_t w8 = kw[(NGW + g) / 4][(NGW + g) % 4];      // token gid + 8
+    float acc[4];
+    mma16816_first(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1], zero4);
+    const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
+    mma16816(acc, y0 & kMaskLo, y8 & kMaskLo, y0 & kMaskHi, y8 & kMaskHi, qf[g][2], qf[g][3]);
+    // Scales and zeros of tokens gid and gid + 8 for groups g, g+1 by one transposing ldmatrix: its
+    // matrices are (scale | tokens 0-7), (scale | 8-15), (zero | 0-7), (zero | 8-15), each with rows
+    // alternating between the 16-byte chunks of groups g and g+1, so every lane receives element gid
+    // of both chunks: half2 (x[g][token], x[g+1][token]).
+    if ((g & 1) == 0) ldmatrix_x4_trans(ksz, st_s + cx.ksz_lane + 32 * g);
+    const float s_lo = (g & 1) ? __high2float(u32_as_h2(ksz[0])) : __low2float(u32_as_h2(ksz[0]));
+    const float s_hi = (g & 1) ? __high2float(u32_as_h2(ksz[1])) : __low2float(u32_as_h2(ksz[1]));
+    const float z_lo = (g & 1) ? __high2float(u32_as_h2(ksz[2])) : __low2float(u32_as_h2(ksz[2]));
+    const float z_hi = (g & 1) ? __high2float(u32_as_h2(ksz[3])) : __low2float(u32_as_h2(ksz[3]));
+    const float t0 = fmaf(-z_lo, qs[g][0], acc[0]), t1 = fmaf(-z_lo, qs[g][1], acc[1]);
+    const float t2 = fmaf(-z_hi, qs[g][0], acc[2]), t3 = fmaf(-z_hi, qs[g][1], acc[3]);
+    if (g == 0) {
+      sc[0] = s_lo * t0; sc[1] = s_lo * t1; sc[2] = s_hi * t2; sc[3] = s_hi * t3;
+    } else {
+      sc[0] = fmaf(s_lo, t0, sc[0]); sc[1] = fmaf(s_lo, t1, sc[1]);
+      sc[2] = fmaf(s_hi, t2, sc[2]); sc[3] = fmaf(s_hi, t3, sc[3]);
     }
   }
+}
+
+// Second half: online softmax on the complete scores, then P.V for this warp's DW output channels.
+template <int D, bool TAIL>
+__device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t st_s, const RowMask& mk,
+                                                 const float (&sc)[4], float (&oacc)[Cfg<D>::DW / 16][4],
+                                                 float (&zacc)[Cfg<D>::NGW][4], float& m0, float& m1, float& l0,
+                                                 float& l1) {
+  constexpr int NGW = Cfg<D>::NGW;
   // ---------------- online softmax in the log2 domain.  d = score - running reference m; the
   // reference is raised only when some d exceeds the threshold, so the common path is 4 FMAs.
   float d0 = fmaf(sc[0], cx.cs, -m0), d1 = fmaf(sc[1], cx.cs, -m1);
@@ -248,11 +263,11 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
     l0 *= f0;
     l1 *= f1;
 #pragma unroll
-    for (int i = 0; i < D / 16; ++i) {
+    for (int i = 0; i < Cfg<D>::DW / 16; ++i) {
       oacc[i][0] *= f0; oacc[i][1] *= f1; oacc[i][2] *= f0; oacc[i][3] *= f1;
     }
 #pragma unroll
-    for (int g = 0; g < NG; ++g) {
+    for (int g = 0; g < NGW; ++g) {
       zacc[g][0] *= f0; zacc[g][1] *= f1;
     }
     d0 = a0 - m0; d1 = a1 - m1; d2 = a2 - m0; d3 = a3 - m1;
@@ -265,30 +280,37 @@ __device__ __forceinline__ void block_step(const WarpCtx<D>& cx, const uint8_t* 
   const uint32_t pt1 = movmatrix_trans(h2_as_u32(__floats2half2_rn(p2, p3)));
 
   // ---------------- P.V: O^T[channel][head] += V^T[channel][token] * (P * s)[token][head]
-  {
-    // matrix j = 4 * i + m of load i is (group j / 2, tokens 8 * (j % 2) ..)
-    uint32_t vw[4];
+  // matrix j = 4 * i + m of load i is (group j / 2 of this warp, tokens 8 * (j % 2) ..)
+  uint32_t vw[4];
 #pragma unroll
-    for (int g = 0; g < NG; ++g) {
-      // Scales / zeros of token pairs (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9) of group g: an ldmatrix
-      // whose eight row addresses are equal hands every lane word tid4 of that 16-byte chunk; the four
-      // matrices are (zero | tokens 0-7), (scale | 0-7), (zero | 8-15), (scale | 8-15).  In that order the
-      // four result registers are, as they stand, the A operand of the zero-point MMA: rows 0-7 hold z_g
-      // (c0, c1 accumulate sum_tok z_g * B_g), rows 8-15 hold the scales and produce values never read.
-      uint32_t vsz[4];
-      ldmatrix_x4(vsz, st_s + cx.vsz_lane + 32 * g);
-      const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vsz[1])));
-      const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vsz[3])));
-      mma16816(zacc[g], vsz[0], vsz[1], vsz[2], vsz[3], b0, b1);
-      // r1 = (tokens 2*tid4, 2*tid4+1), r2 = (tokens 2*tid4+8, +9): 16-bit lane gid of chunk g, i.e. codes of
-      // channels 32g + 4*gid .. +3 of two tokens side by side
-      if ((g & 1) == 0) ldmatrix_x4_trans(vw, st_s + cx.vaddr[g / 2]);
-      const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
-      mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
-      const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
-      mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1 & kMaskHi, y2 & kMaskLo, y2 & kMaskHi, b0, b1);
-    }
+  for (int g = 0; g < NGW; ++g) {
+    // Scales / zeros of token pairs (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9) of group g: an ldmatrix
+    // whose eight row addresses are equal hands every lane word tid4 of that 16-byte chunk; the four
+    // matrices are (zero | tokens 0-7), (scale | 0-7), (zero | 8-15), (scale | 8-15).  In that order the
+    // four result registers are, as they stand, the A operand of the zero-point MMA: rows 0-7 hold z_g
+    // (c0, c1 accumulate sum_tok z_g * B_g), rows 8-15 hold the scales and produce values never read.
+    uint32_t vsz[4];
+    ldmatrix_x4(vsz, st_s + cx.vsz_lane + 32 * g);
+    const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vsz[1])));
+    const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vsz[3])));
+    mma16816(zacc[g], vsz[0], vsz[1], vsz[2], vsz[3], b0, b1);
+    // r1 = (tokens 2*tid4, 2*tid4+1), r2 = (tokens 2*tid4+8, +9): 16-bit lane gid of chunk g, i.e. codes of
+    // channels 32g + 4*gid .. +3 of two tokens side by side
+    if ((g & 1) == 0) ldmatrix_x4_trans(vw, st_s + cx.vaddr[g / 2]);
+    const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
+    mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
+    const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
+    mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1 & kMaskHi, y2 & kMaskLo, y2 & kMaskHi, b0, b1);
   }
+}
+
+// Bounded wait on an mbarrier phase; false if the copy did not complete within the limit.
+__device__ __forceinline__ bool wait_stage(uint32_t bar, uint32_t parity) {
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if (++spins > kMaxSpins) return false;
+  }
+  return true;
 }
 
 // GEN = the general form: a sliding window (Appendix A) and / or several query tokens per sequence
@@ -303,7 +325,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
                       int C, float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
                       int32_t* status) {
   using Cf = Cfg<D>;
-  constexpr int NG = Cf::NG;
+  constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
   extern __shared__ __align__(1024) uint8_t smem[];
 
   const int G = H_q / cache.H_kv;
@@ -311,6 +333,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const int tiles = (GV + 7) >> 3;
   const int c = blockIdx.x, kvh = blockIdx.y / tiles, tile = blockIdx.y - kvh * tiles, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tid4 = lane & 3;
+  const int team = warp / DS, sub = warp - team * DS;  // this warp works on channels [sub * DW, (sub + 1) * DW)
   const int v0 = tile * 8;                   // first column of this tile
   const int nh = min(8, GV - v0);            // columns in the tile; the rest of N = 8 is zero padding
   // row of column v in q and in the partial arrays: [B][S_q][H_q]
@@ -325,31 +348,32 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   split_range(GEN ? query_lo(len, S_q, 0, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
 
   // ---- q first (a handful of loads that must not queue behind the cache stream), used further down
-  uint4 qraw[NG];
+  uint4 qraw[NGW];
 #pragma unroll
-  for (int g = 0; g < NG; ++g) {
+  for (int g = 0; g < NGW; ++g) {
     qraw[g] = make_uint4(0, 0, 0, 0);
     if (gid < nh)
-      qraw[g] = *reinterpret_cast<const uint4*>(q + q_row(v0 + gid) * D + g * 32 + tid4 * 8);
+      qraw[g] = *reinterpret_cast<const uint4*>(q + q_row(v0 + gid) * D + (sub * NGW + g) * 32 + tid4 * 8);
   }
 
-  // ---- this warp's token blocks: blk0 + warp, blk0 + warp + kWarps, ...
+  // ---- this team's token blocks: blk0 + team, blk0 + team + NTEAM, ...
   const int blk0 = t0 / kBlk, blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
-  const int nblk = blk1 - blk0 > warp ? (blk1 - blk0 - warp + kWarps - 1) / kWarps : 0;
+  const int nblk = blk1 - blk0 > team ? (blk1 - blk0 - team + NTEAM - 1) / NTEAM : 0;
   const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
-  uint8_t* const ring = smem + warp * (Cf::NST * Cf::STAGE);
+  uint8_t* const ring = smem + team * (Cf::NST * Cf::STAGE);
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
-  const uint32_t bars = static_cast<uint32_t>(__cvta_generic_to_shared(smem + Cf::BARS)) + warp * (Cf::NST * 8);
-  if (lane == 0) {
+  const uint32_t bars = static_cast<uint32_t>(__cvta_generic_to_shared(smem + Cf::BARS)) + team * (Cf::NST * 8);
+  if (sub == 0 && lane == 0) {
 #pragma unroll
     for (int s = 0; s < Cf::NST; ++s) mbar_init(bars + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  __syncwarp();
-  // block j of this (sequence, KV head) starts at head_blocks + j * STAGE; one lane copies it into a ring slot
+  if (DS > 1) __syncthreads();  // the team's other warps wait on these barriers too
+  else __syncwarp();
+  // block j of this (sequence, KV head) starts at head_blocks + j * STAGE; one lane of the team copies it into a slot
   const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
   auto issue = [&](int slot, int blk) {
-    if (lane == 0) {
+    if (sub == 0 && lane == 0) {
       const uint32_t bar = bars + 8 * slot;
       mbar_expect_tx(bar, Cf::STAGE);
       bulk_g2s(ring_s + slot * Cf::STAGE, head_blocks + static_cast<size_t>(blk) * Cf::STAGE, Cf::STAGE, bar);
@@ -359,15 +383,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // start streaming: the first stages are in flight while q is turned into fragments
 #pragma unroll
   for (int s = 0; s < Cf::NST - 1; ++s)
-    if (s < nblk) issue(s, blk0 + warp + s * kWarps);
-
+    if (s < nblk) issue(s, blk0 + team + s * NTEAM);
 
   // ---- q as MMA B fragments: column n = gid is column v0 + gid of the tile; k slots follow the nibble order.
   // qs[g][j] = 2^-24 * sum of q over group g for heads 2*tid4 + j (the zero-point term of the scores).
-  uint32_t qf[NG][4];
-  float qs[NG][2];
+  uint32_t qf[NGW][4];
+  float qs[NGW][2];
 #pragma unroll
-  for (int g = 0; g < NG; ++g) {
+  for (int g = 0; g < NGW; ++g) {
     const uint4 raw = qraw[g];
     const __half2 sixteenth = __float2half2_rn(0.0625f);
     qf[g][0] = __byte_perm(raw.x, raw.z, 0x5410);                                            // (c0, c4)
@@ -388,80 +411,114 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     qs[g][1] = __shfl_sync(0xffffffffu, sum, (2 * tid4 + 1) * 4);
   }
 
-  float oacc[D / 16][4];  // [M tile][c0..c3]: rows = channels, cols = heads 2*tid4, 2*tid4+1
-  float zacc[NG][4];      // sum_tok B_g * z_g: [0], [1] are heads 2*tid4, 2*tid4+1; [2], [3] are not used
-  float zero4[4];         // four registers holding 0, opaque to the compiler: the C operand of accumulator-less MMAs
+  float oacc[Cf::DW / 16][4];  // [M tile][c0..c3]: rows = channels, cols = heads 2*tid4, 2*tid4+1
+  float zacc[NGW][4];          // sum_tok B_g * z_g: [0], [1] are heads 2*tid4, 2*tid4+1; [2], [3] are not used
+  float zero4[4];              // four registers holding 0, opaque to the compiler: the C operand of accumulator-less MMAs
 #pragma unroll
   for (int i = 0; i < 4; ++i) asm volatile("mov.f32 %0, 0f00000000;\n" : "=f"(zero4[i]));
 #pragma unroll
-  for (int i = 0; i < D / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+  for (int i = 0; i < Cf::DW / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
 #pragma unroll
-  for (int g = 0; g < NG; ++g) zacc[g][0] = zacc[g][1] = zacc[g][2] = zacc[g][3] = 0.f;
+  for (int g = 0; g < NGW; ++g) zacc[g][0] = zacc[g][1] = zacc[g][2] = zacc[g][3] = 0.f;
   float m0 = kNoMax, m1 = kNoMax, l0 = 0.f, l1 = 0.f;
   const float cs = attn_scale * kLog2e * 16777216.0f;  // scores carry 2^-24 from the code operands
-
-  // per-lane byte offsets inside a stage (everything else is a compile-time offset from these)
-  // ldmatrix row addresses (offsets in a stage) for the scale / zero fragments, see block_step
-  const uint32_t ksz_lane = 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32;
-  const uint32_t vsz_lane = 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16;
 
   // Blocks in which every token counts for every column go through the plain step, the others through the
   // masking one.  Plain decode: only the block holding the end of the sequence is partial.  General form:
   // blocks that reach beyond the oldest query's end, or begin before the newest query's window start.
-  const int rem_last = t1 - (blk0 + warp + (nblk - 1) * kWarps) * kBlk;  // tokens in this warp's last block
-  int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;           // this warp's blocks k < nfull are full
-  int nhead = 0;                                                         // ... and blocks k < nhead are masked
-  int lo0 = 0, hi0 = 0, lo1 = 0, hi1 = 0;                                // token ranges of this thread's two columns
+  const int rem_last = t1 - (blk0 + team + (nblk - 1) * NTEAM) * kBlk;  // tokens in this team's last block
+  int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;          // this team's blocks k < nfull are full
+  int nhead = 0;                                                        // ... and blocks k < nhead are masked
+  int lo0 = 0, hi0 = 0, lo1 = 0, hi1 = 0;                               // token ranges of this thread's two columns
   if (GEN) {
     const int s0 = min((v0 + 2 * tid4) / G, S_q - 1), s1 = min((v0 + 2 * tid4 + 1) / G, S_q - 1);
     hi0 = query_hi(len, S_q, s0); lo0 = window_begin(hi0, window);
     hi1 = query_hi(len, S_q, s1); lo1 = window_begin(hi1, window);
     const int full_end = min(t1, query_hi(len, S_q, 0)) >> 4;                   // blocks below it end inside every range
     const int full_begin = (query_lo(len, S_q, S_q - 1, window) + kBlk - 1) >> 4;  // blocks from it on begin inside
-    const int first_blk = blk0 + warp;
-    nfull = full_end > first_blk ? min(nblk, (full_end - first_blk + kWarps - 1) / kWarps) : 0;
-    nhead = full_begin > first_blk ? min(nblk, (full_begin - first_blk + kWarps - 1) / kWarps) : 0;
+    const int first_blk = blk0 + team;
+    nfull = full_end > first_blk ? min(nblk, (full_end - first_blk + NTEAM - 1) / NTEAM) : 0;
+    nhead = full_begin > first_blk ? min(nblk, (full_begin - first_blk + NTEAM - 1) / NTEAM) : 0;
   }
+  // per-lane byte offsets inside a stage: ldmatrix row addresses of the code, scale and zero fragments of
+  // this warp's channel groups sub * NGW .. (see block_scores / block_softmax_pv)
   WarpCtx<D> cx;
-  cx.ring = ring; cx.ksz_lane = ksz_lane; cx.vsz_lane = vsz_lane; cx.cs = cs; cx.gid = gid;
+  cx.ring = ring; cx.cs = cs; cx.gid = gid;
+  cx.ksz_lane = 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32 + sub * NGW * 32;
+  cx.vsz_lane = 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
 #pragma unroll
-  for (int i = 0; i < NG / 2; ++i) {
+  for (int i = 0; i < NGW / 2; ++i) {
     const int j = 4 * i + (lane >> 3);
-    const int ktok = (lane & 7) + 8 * (j / NG), kgrp = j % NG;
+    const int ktok = (lane & 7) + 8 * (j / NGW), kgrp = sub * NGW + j % NGW;
     cx.kaddr[i] = ktok * Cf::ROWB + ((kgrp ^ Cf::swz(ktok)) << 4);
-    const int vtok = (lane & 7) + 8 * (j % 2), vgrp = j / 2;
+    const int vtok = (lane & 7) + 8 * (j % 2), vgrp = sub * NGW + j / 2;
     cx.vaddr[i] = Cf::PK + vtok * Cf::ROWB + ((vgrp ^ Cf::swz(vtok)) << 4);
   }
+  // score exchange of a team: [2 (parity of k)][DS][32 lanes] float4, then [2][DS] timeout flags
+  float4* const xch = reinterpret_cast<float4*>(smem + Cf::XCH + team * Cf::XCH_TEAM);
+  int* const xflag = reinterpret_cast<int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
+
   bool timed_out = false;
 #pragma unroll 2  // measured: 34.3 -> 33.3 us per 128K layer (loop overhead shared by two blocks)
   for (int k = 0; k < nblk; ++k) {
     // Wait for this block's bytes.  The wait is bounded: if the copy never completes (which would take
     // a bad pointer), the warp flags the status word and stops consuming.
-    {
-      const uint32_t bar = bars + 8 * (k & (Cf::NST - 1)), parity = (k / Cf::NST) & 1;
-      int spins = 0;
-      while (!mbar_try_wait(bar, parity)) {
-        if (++spins > kMaxSpins) { timed_out = true; break; }
-      }
-      if (timed_out) break;
+    const bool arrived = wait_stage(bars + 8 * (k & (Cf::NST - 1)), (k / Cf::NST) & 1);
+    if (DS == 1) {
+      if (!arrived) { timed_out = true; break; }
+      __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
+      if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + team + (k + Cf::NST - 1) * NTEAM);
     }
-    __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
-    if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + warp + (k + Cf::NST - 1) * kWarps);
+    const uint32_t st_s = ring_s + (k & (Cf::NST - 1)) * Cf::STAGE;
     const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
-    if (k < nfull && !(GEN && k < nhead)) {
-      const RowMask all{kBlk, 0, kBlk, 0, kBlk};
-      block_step<D, false>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, all, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
-    } else {
+    const bool plain = k < nfull && !(GEN && k < nhead);
+    auto mask_of_block = [&]() {
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
       if (GEN) {
-        const int first = (blk0 + warp + k * kWarps) * kBlk;  // first token of this block
+        const int first = (blk0 + team + k * NTEAM) * kBlk;  // first token of this block
         mk = RowMask{t1 - first, lo0 - first, min(hi0, t1) - first, lo1 - first, min(hi1, t1) - first};
       }
-      block_step<D, true>(cx, st, ring_s + (k & (Cf::NST - 1)) * Cf::STAGE, mk, qf, qs, oacc, zacc, zero4, m0, m1, l0, l1);
+      return mk;
+    };
+    const RowMask all{kBlk, 0, kBlk, 0, kBlk};
+    float sc[4];
+    if (DS == 1) {
+      if (plain) {
+        block_scores<D, false>(cx, st, st_s, all, qf, qs, zero4, sc);
+        block_softmax_pv<D, false>(cx, st_s, all, sc, oacc, zacc, m0, m1, l0, l1);
+      } else {
+        const RowMask mk = mask_of_block();
+        block_scores<D, true>(cx, st, st_s, mk, qf, qs, zero4, sc);
+        block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
+      }
+    } else {
+      const RowMask mk = plain ? all : mask_of_block();
+      if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, zero4, sc);
+      else block_scores<D, true>(cx, st, st_s, mk, qf, qs, zero4, sc);
+      // The warps of the team each hold the scores over their own channels: exchange and add them in a fixed
+      // order, so that every warp of the team continues with bit-identical scores.  The barrier of
+      // iteration k also tells that every warp is done with the slot of iteration k - 1, which is refilled
+      // after it; a warp whose wait ran out says so here and the whole team stops together.
+      float4* const xb = xch + (k & 1) * (DS * 32);
+      xb[sub * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
+      if (lane == 0) xflag[(k & 1) * DS + sub] = arrived ? 0 : 1;
+      asm volatile("bar.sync %0, %1;\n" ::"r"(1 + team), "r"(32 * DS) : "memory");
+      int bad = 0;
+      sc[0] = sc[1] = sc[2] = sc[3] = 0.f;
+#pragma unroll
+      for (int w = 0; w < DS; ++w) {
+        const float4 part = xb[w * 32 + lane];
+        sc[0] += part.x; sc[1] += part.y; sc[2] += part.z; sc[3] += part.w;
+        bad |= xflag[(k & 1) * DS + w];
+      }
+      if (bad) { timed_out = true; break; }
+      if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + team + (k + Cf::NST - 1) * NTEAM);
+      if (plain) block_softmax_pv<D, false>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
+      else block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
     }
   }
   if (timed_out) {
-    // Copies of this warp may still be in flight into its ring: give each a bounded time to land before
+    // Copies of this team may still be in flight into its ring: give each a bounded time to land before
     // the block reuses the memory, then report.  The partial written below is not valid in that case.
     for (int s = 0; s < Cf::NST; ++s) {
       int spins = 0;
@@ -470,46 +527,46 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     if (lane == 0 && status) atomicOr(status, TQ_STATUS_TIMEOUT);
   }
 
-  // ---------------- merge the warps and write the normalised partial (o_c, m_c, l_c)
+  // ---------------- merge the teams and write the normalised partial (o_c, m_c, l_c)
 #pragma unroll
   for (int off = 4; off <= 16; off <<= 1) {
     l0 += __shfl_xor_sync(0xffffffffu, l0, off);
     l1 += __shfl_xor_sync(0xffffffffu, l1, off);
   }
   __syncthreads();  // every warp is done with its ring; the memory is reused below
-  // layout (floats): wml[kWarps][16] = each warp's m[8], l[8] | slab[kWarps][D][kChPitch] | tb[8][kRowPitch]
+  // layout (floats): wml[NTEAM][16] = each team's m[8], l[8] | slab[NTEAM][D][kChPitch] | tb[8][kRowPitch]
   constexpr int kChPitch = 10;       // 8 heads per channel row, padded: the float2 fragment stores are conflict free
   constexpr int kRowPitch = D + 4;   // transposed [head][channel] tile, conflict free for the writes below
   float* const wml = reinterpret_cast<float*>(smem);
-  float* const slab = wml + kWarps * 16;
-  float* const tb = slab + kWarps * D * kChPitch;
-  if (gid == 0) {
-    wml[warp * 16 + 2 * tid4] = m0;
-    wml[warp * 16 + 2 * tid4 + 1] = m1;
-    wml[warp * 16 + 8 + 2 * tid4] = l0;
-    wml[warp * 16 + 8 + 2 * tid4 + 1] = l1;
+  float* const slab = wml + NTEAM * 16;
+  float* const tb = slab + NTEAM * D * kChPitch;
+  if (gid == 0 && sub == 0) {  // the warps of a team hold identical m and l
+    wml[team * 16 + 2 * tid4] = m0;
+    wml[team * 16 + 2 * tid4 + 1] = m1;
+    wml[team * 16 + 8 + 2 * tid4] = l0;
+    wml[team * 16 + 8 + 2 * tid4 + 1] = l1;
   }
   __syncthreads();
-  // every thread: unit-wide reference M, denominator and this warp's weight for its two heads
+  // every thread: unit-wide reference M, denominator and this team's weight for its two heads
   float M0 = kNoMax, M1 = kNoMax;
 #pragma unroll
-  for (int w = 0; w < kWarps; ++w) {
+  for (int w = 0; w < NTEAM; ++w) {
     M0 = fmaxf(M0, wml[w * 16 + 2 * tid4]);
     M1 = fmaxf(M1, wml[w * 16 + 2 * tid4 + 1]);
   }
   float den0 = 0.f, den1 = 0.f;
 #pragma unroll
-  for (int w = 0; w < kWarps; ++w) {  // a warp that saw no token has m = -1e30 and l = 0
+  for (int w = 0; w < NTEAM; ++w) {  // a team that saw no token has m = -1e30 and l = 0
     den0 = fmaf(ex2(wml[w * 16 + 2 * tid4] - M0), wml[w * 16 + 8 + 2 * tid4], den0);
     den1 = fmaf(ex2(wml[w * 16 + 2 * tid4 + 1] - M1), wml[w * 16 + 8 + 2 * tid4 + 1], den1);
   }
   const float f0 = den0 > 0.f ? ex2(m0 - M0) / den0 : 0.f;
   const float f1 = den1 > 0.f ? ex2(m1 - M1) / den1 : 0.f;
-  float* const mo = slab + warp * D * kChPitch;
+  float* const mo = slab + team * D * kChPitch;
 #pragma unroll
-  for (int mt = 0; mt < D / 16; ++mt) {
+  for (int mt = 0; mt < Cf::DW / 16; ++mt) {
     const int g = mt >> 1;
-    const int ch = 32 * g + 4 * gid + 2 * (mt & 1);
+    const int ch = sub * Cf::DW + 32 * g + 4 * gid + 2 * (mt & 1);
     // even channel: codes carried 2^-24; odd channel (high nibble): 2^-20
     *reinterpret_cast<float2*>(mo + ch * kChPitch + 2 * tid4) =
         make_float2((oacc[mt][0] * 16777216.0f - zacc[g][0]) * f0, (oacc[mt][1] * 16777216.0f - zacc[g][1]) * f1);
@@ -521,7 +578,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     const int x = idx >> 3, h = idx & 7;  // consecutive threads take consecutive heads of one channel
     float sum = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) sum += slab[(w * D + x) * kChPitch + h];
+    for (int w = 0; w < NTEAM; ++w) sum += slab[(w * D + x) * kChPitch + h];
     tb[h * kRowPitch + x] = sum;
   }
   __syncthreads();
@@ -570,6 +627,7 @@ cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, in
   switch (c.d) {
     case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
     case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    case 512: return launch<512>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
     default: return launch<256>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
   }
 }

@@ -126,9 +126,9 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
 // grid: (blocks touched per sequence, B * H_kv, {K, V}); 2 * d threads (one per 8 elements).
 // seq_lens is read only here and bumped by bump_lens_kernel afterwards, so that no block can observe a
 // length that another block of the same launch has already advanced.
-__global__ void __launch_bounds__(512) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
+__global__ void __launch_bounds__(1024) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
                                                             int T) {
-  __shared__ __align__(16) __half sm_meta[2][8][16];  // [scale | zero][group][token]
+  __shared__ __align__(16) __half sm_meta[2][16][16];  // [scale | zero][group][token], up to d = 512
   pdl_wait();
   pdl_launch_dependents();
   const int d = c.d, cpr = d >> 3, ng = d >> 5;

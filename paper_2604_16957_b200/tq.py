@@ -106,7 +106,7 @@ class KVCache:
     describes it."""
 
     def __init__(self, B, H_kv, S_cap, d, device="cuda"):
-        assert S_cap % 16 == 0 and d in (64, 128, 256)
+        assert S_cap % 16 == 0 and d in (64, 128, 256, 512)
         self.B, self.H_kv, self.S_cap, self.d = B, H_kv, S_cap, d
         self.blocks = torch.zeros((B, H_kv, S_cap // 16, TQ_BLOCK_BYTES(d)), dtype=torch.uint8, device=device)
         self.seq_lens = torch.zeros((B,), dtype=torch.int32, device=device)
@@ -120,7 +120,7 @@ class KVCache:
         B, H, S, d = self.B, self.H_kv, self.S_cap, self.d
         ng, rowb, nb = d // 32, d // 2, S // 16
         pk, sz = 16 * rowb, ng * 32
-        shift = {2: 2, 4: 1, 8: 0}[ng]
+        shift = {2: 2, 4: 1, 8: 0, 16: 0}[ng]
         t = torch.arange(16, device=self.blocks.device)
         g = torch.arange(ng, device=self.blocks.device)
         pos = g[None, :] ^ ((t[:, None] >> shift) & (ng - 1))          # [16][ng]: chunk position of group g of token t

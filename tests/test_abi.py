@@ -44,7 +44,7 @@ def test_host_side_helpers(lib):
             prev = t1
         assert prev == length
     # block layout: 2560 bytes per 16 tokens at d = 128; the offset helpers cover a block exactly once
-    for d in (64, 128, 256):
+    for d in (64, 128, 256, 512):
         nbytes = tq.TQ_BLOCK_BYTES(d)
         assert nbytes == 16 * 2 * tq.tq_cache_bytes(1, 1, 16, d) // 32 == 16 * (d + d // 4)
         seen = set()

@@ -363,3 +363,36 @@ def test_multi_query_decode(gpu, oracle, d, H_q, H_kv, S_q, impl):
             assert_attention_close(got.reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d), f"S_q {S_q} window {window} C {C}")
     finally:
         os.environ.pop("TQ_DECODE_IMPL", None)
+
+
+@pytest.mark.parametrize("impl", ["mma", "simple"])
+def test_head_dim_512(gpu, oracle, impl):
+    """Table 7's Gemma global layers: d = 512, 32 query heads per KV head (four head tiles).  Decode after a
+    bulk fill and a T = 1 append, with ragged lengths, explicit and automatic splits, a window and several
+    query tokens."""
+    tq, torch = gpu
+    sh = I.Shape("global512", 2, 64, 2, 512, 1.0, sigma_qk=0.2)
+    lens = [1500, 333]
+    host, dev = _both(gpu, oracle, sh, 1500, 71, S_cap=1520, lens=lens, fill_byte=0xFF)
+    k1, v1 = I.make_kv(sh, 1, 71, stream=1)
+    host.append(k1, v1)
+    tq.tq_kv_quantize_append(dev, torch.from_numpy(k1).cuda(), torch.from_numpy(v1).cuda())
+    assert_cache_bits_equal(dev, host)
+    q = I.make_q(sh, 71)
+    if impl == "simple":
+        os.environ["TQ_DECODE_IMPL"] = "simple"
+    try:
+        for C in (0, 1, 5):
+            out, _, _ = fused_attention(tq, torch, dev, q, sh.alpha, num_splits=C)
+            assert_attention_close(out, oracle.attention(host, q, sh.alpha), f"d512 C={C}")
+        q3 = np.ascontiguousarray(np.stack([I.make_q(sh, 71, stream=s) for s in range(3)], axis=1))
+        for window in (0, 100):
+            o, m, l = tq.alloc_partials(sh.B, sh.H_q * 3, sh.d, 4)
+            out = torch.empty((sh.B, 3, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+            tq.tq_sdpa_int4_decode_multi(dev, torch.from_numpy(q3).cuda(), sh.alpha, window, 4, o, m, l)
+            tq.tq_sdpa_int4_combine(o, m, l, out.view(sh.B, 3 * sh.H_q, sh.d))
+            torch.cuda.synchronize()
+            ref = oracle.attention_multi(host, q3, sh.alpha, window)
+            assert_attention_close(out.cpu().numpy().reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d), f"d512 w={window}")
+    finally:
+        os.environ.pop("TQ_DECODE_IMPL", None)

@@ -17,7 +17,8 @@ def gpu():
 
 
 @pytest.mark.parametrize("shape,S,seed", [(I.TINY, 256, 1), (I.LLAMA, 1024, 2), (I.LLAMA, 4096 + 48, 3),
-                                          (I.GEMMA, 512, 4), (I.Shape("b3", 3, 8, 2, 64, 0.125), 100, 6)])
+                                          (I.GEMMA, 512, 4), (I.Shape("b3", 3, 8, 2, 64, 0.125), 100, 6),
+                                          (I.Shape("global512", 2, 32, 1, 512, 1.0, sigma_qk=0.25), 300, 7)])
 def test_bulk_quantise_bit_exact(gpu, oracle, shape, S, seed):
     tq, torch = gpu
     k, v = I.make_kv(shape, S, seed)
