@@ -208,6 +208,21 @@ size_t tq_dequant_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t 
                                   int32_t ws_is_fp32);
 
 /*
+ * K-versus-V precision ablation (Sec. 5: int4 K with full-precision V loses less than full-precision K
+ * with int4 V, because key errors pass through the softmax while value errors reach the output
+ * directly).  Phase 1 with each of K and V taken either from the int4 cache or from an unquantised
+ * matrix: k_fp16 / v_fp16 are device fp16 [B][H_kv][S_cap][d] (rows below seq_lens[b] are read), or
+ * NULL to take that side from the cache.  Both NULL is the plain fused attention; both given ignores
+ * the cache's contents (its lengths still apply) and is full-precision attention.  Same partials as
+ * tq_sdpa_int4_decode (combine with tq_sdpa_int4_combine).  A scalar kernel meant for the experiment,
+ * not for speed.  num_splits = 0 picks tq_auto_splits(B, H_kv, H_q, d, S_cap).
+ * Errors and status as tq_sdpa_int4_decode.
+ */
+int tq_sdpa_mixed_precision_attend(const tq_kv_cache* cache /* host */, const void* k_fp16, const void* v_fp16,
+                                   const void* q, int32_t H_q, float attn_scale, int32_t num_splits, float* o_part,
+                                   float* m_part, float* l_part, int32_t* status, void* stream);
+
+/*
  * Fused attention for callers that cannot allocate (the paper has no counterpart for this entry
  * point; it exists for integration, not for the method).  Some hosts of this library may not call
  * cudaMalloc at the point where attention runs: an inference server that hands all device memory

@@ -179,6 +179,30 @@ def attention_multi(cache: Cache, q: np.ndarray, alpha: float, window: int = 0) 
     return out
 
 
+def attention_mixed(cache: Cache, k16, v16, q: np.ndarray, alpha: float) -> np.ndarray:
+    """K-versus-V precision ablation (Sec. 5): softmax(alpha q K^T) V in fp64 with K and V each either the
+    dequantised cache (argument None) or the given unquantised fp16 values [B][H_kv][>= len][d].
+    Returns [B][H_q][d]."""
+    q = np.asarray(q, dtype=np.float16).astype(np.float64)
+    B, H_q, d = q.shape
+    G = H_q // cache.H_kv
+    kd = dequant_rows(cache.k_packed, cache.k_scale, cache.k_zero) if k16 is None else None
+    vd = dequant_rows(cache.v_packed, cache.v_scale, cache.v_zero) if v16 is None else None
+    out = np.zeros((B, H_q, d), np.float64)
+    for b in range(B):
+        n = int(cache.lens[b])
+        if n == 0:
+            continue
+        for h in range(H_q):
+            kv = h // G
+            K = (kd[b, kv, :n] if k16 is None else np.asarray(k16[b, kv, :n], dtype=np.float16).astype(np.float64))
+            V = (vd[b, kv, :n] if v16 is None else np.asarray(v16[b, kv, :n], dtype=np.float16).astype(np.float64))
+            a = alpha * (K @ q[b, h])
+            w = np.exp(a - a.max())
+            out[b, h] = (w / w.sum()) @ V
+    return out
+
+
 def attention_weights(cache: Cache, q, alpha, b, h) -> np.ndarray:
     q = np.ascontiguousarray(q, dtype=np.float16)
     w = np.zeros((int(cache.lens[b]),), np.float64)

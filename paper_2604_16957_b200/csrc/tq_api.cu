@@ -203,6 +203,23 @@ int tq_sdpa_dequant_then_attend(const tq_kv_cache* cache, const void* q, int32_t
   return finish(launch_combine(o_part, m_part, l_part, cache->B, H_q, d, C, out, out_is_fp32 != 0, st));
 }
 
+int tq_sdpa_mixed_precision_attend(const tq_kv_cache* cache, const void* k_fp16, const void* v_fp16, const void* q,
+                                   int32_t H_q, float attn_scale, int32_t num_splits, float* o_part, float* m_part,
+                                   float* l_part, int32_t* status, void* stream) {
+  if (int r = check_cache(cache)) return r;
+  if (!q || !o_part || !m_part || !l_part) return TQ_ERR_NULL;
+  if (int r = check_heads(cache, H_q)) return r;
+  if (num_splits < 0 || num_splits > TQ_MAX_SPLITS) return TQ_ERR_SHAPE;
+  if (!aligned16(q) || !aligned16(o_part) || !aligned16(k_fp16) || !aligned16(v_fp16) ||
+      (reinterpret_cast<uintptr_t>(m_part) & 3u) || (reinterpret_cast<uintptr_t>(l_part) & 3u) ||
+      (reinterpret_cast<uintptr_t>(status) & 3u))
+    return TQ_ERR_ALIGN;
+  const int C = num_splits ? num_splits : tq_auto_splits(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
+  return finish(launch_attend_mixed(*cache, static_cast<const __half*>(k_fp16), static_cast<const __half*>(v_fp16),
+                                    static_cast<const __half*>(q), H_q, attn_scale, C, o_part, m_part, l_part, status,
+                                    static_cast<cudaStream_t>(stream)));
+}
+
 size_t tq_cache_bytes(int32_t B, int32_t H_kv, int32_t S_cap, int32_t d) {
   if (B < 1 || H_kv < 1 || S_cap < 1 || d < 1) return 0;
   return static_cast<size_t>(B) * H_kv * ((static_cast<size_t>(S_cap) + 15) / 16) * TQ_BLOCK_BYTES(d);

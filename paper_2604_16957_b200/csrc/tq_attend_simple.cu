@@ -59,6 +59,20 @@ struct SrcMat {
   }
 };
 
+// K and V from different places: each either the int4 cache or an unquantised fp16 matrix
+// [B][H_kv][S_cap][D].  This is the K-versus-V precision ablation of Sec. 5 (int4 K with full-precision
+// V against full-precision K with int4 V).
+template <int D>
+struct SrcMixed {
+  static constexpr int EPL = D / 32;
+  SrcInt4<D> cache;
+  SrcMat<D, __half> mat;  // a null k or v means "take that side from the cache"
+  __device__ void load(bool is_v, long long row, int lane, float (&x)[EPL]) const {
+    if ((is_v ? mat.v : mat.k) != nullptr) mat.load(is_v, row, lane, x);
+    else cache.load(is_v, row, lane, x);
+  }
+};
+
 // grid: (C, H_kv * head_tiles, B); block: kWarps warps.
 template <int D, typename Src>
 __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, const int32_t* seq_lens, int H_kv,
@@ -244,6 +258,22 @@ cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, 
     }
   };
   return fp32 ? by_d(float{}) : by_d(__half{});
+}
+
+cudaError_t launch_attend_mixed(const tq_kv_cache& c, const __half* k_fp16, const __half* v_fp16, const __half* q, int H_q,
+                                float attn_scale, int C, float* o_part, float* m_part, float* l_part, int32_t* status,
+                                cudaStream_t st) {
+  auto run = [&](auto dtag) {
+    constexpr int D = decltype(dtag)::value;
+    SrcMixed<D> src{SrcInt4<D>{c.blocks, c.S_cap}, SrcMat<D, __half>{k_fp16, v_fp16}};
+    return launch_simple<D>(src, c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
+  };
+  switch (c.d) {
+    case 64: return run(std::integral_constant<int, 64>{});
+    case 128: return run(std::integral_constant<int, 128>{});
+    case 512: return run(std::integral_constant<int, 512>{});
+    default: return run(std::integral_constant<int, 256>{});
+  }
 }
 
 cudaError_t launch_dequant(const tq_kv_cache& c, void* k_mat, void* v_mat, bool fp32, cudaStream_t st) {

@@ -114,6 +114,9 @@ cudaError_t launch_dequant(const tq_kv_cache& c, void* k_mat, void* v_mat, bool 
 cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, const void* v_mat, bool fp32,
                                        const __half* q, int H_q, float attn_scale, int C, float* o_part, float* m_part,
                                        float* l_part, int32_t* status, cudaStream_t st);
+cudaError_t launch_attend_mixed(const tq_kv_cache& c, const __half* k_fp16, const __half* v_fp16, const __half* q, int H_q,
+                                float attn_scale, int C, float* o_part, float* m_part, float* l_part, int32_t* status,
+                                cudaStream_t st);
 int device_sm_count();
 
 }  // namespace tq

@@ -28,7 +28,7 @@ SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa
            "tq_partials_bytes", "tq_sdpa_dequant_then_attend", "tq_dequant_workspace_bytes", "tq_cache_bytes",
            "tq_result_string", "tq_last_cuda_error", "tq_version", "tq_sdpa_int4_attend_static",
            "tq_cache_code_offset", "tq_cache_meta_offset", "tq_sdpa_int4_decode_window", "tq_split_range_window",
-           "tq_sdpa_int4_decode_multi")
+           "tq_sdpa_int4_decode_multi", "tq_sdpa_mixed_precision_attend")
 
 
 class tq_kv_cache(C.Structure):
@@ -54,6 +54,8 @@ _lib.tq_sdpa_int4_decode_window.argtypes = [_cache_p, _vp, _i32, _f32, _i32, _i3
 _lib.tq_sdpa_int4_decode_window.restype = C.c_int
 _lib.tq_sdpa_int4_decode_multi.argtypes = [_cache_p, _vp, _i32, _i32, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.tq_sdpa_int4_decode_multi.restype = C.c_int
+_lib.tq_sdpa_mixed_precision_attend.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp]
+_lib.tq_sdpa_mixed_precision_attend.restype = C.c_int
 _lib.tq_split_range_window.argtypes = [_i32, _i32, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.tq_split_range_window.restype = None
 _lib.tq_sdpa_int4_combine.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _i32, _vp, _i32, _vp]
@@ -202,6 +204,20 @@ def tq_sdpa_int4_decode_multi(cache, q, attn_scale, window, num_splits, o_part, 
     _check(_lib.tq_sdpa_int4_decode_multi(C.byref(cs), _ptr(q), q.shape[2], q.shape[1], float(attn_scale),
                                           int(window), int(num_splits), _ptr(o_part), _ptr(m_part), _ptr(l_part),
                                           _ptr(status), _stream(stream)), "tq_sdpa_int4_decode_multi")
+
+
+def tq_sdpa_mixed_precision_attend(cache, k_fp16, v_fp16, q, attn_scale, num_splits, o_part, m_part, l_part,
+                                   status=None, stream=None):
+    """Phase 1 with K and / or V from unquantised fp16 [B][H_kv][S_cap][d] (None: from the int4 cache)."""
+    assert q.is_contiguous() and q.dtype == torch.float16 and q.dim() == 3
+    for t in (k_fp16, v_fp16):
+        assert t is None or (t.is_contiguous() and t.dtype == torch.float16 and
+                             tuple(t.shape) == (cache.B, cache.H_kv, cache.S_cap, cache.d))
+    cs = _cs(cache)
+    _check(_lib.tq_sdpa_mixed_precision_attend(C.byref(cs), _ptr(k_fp16), _ptr(v_fp16), _ptr(q), q.shape[1],
+                                               float(attn_scale), int(num_splits), _ptr(o_part), _ptr(m_part),
+                                               _ptr(l_part), _ptr(status), _stream(stream)),
+           "tq_sdpa_mixed_precision_attend")
 
 
 def tq_split_range_window(length, window, C_, c):

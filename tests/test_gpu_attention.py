@@ -396,3 +396,25 @@ def test_head_dim_512(gpu, oracle, impl):
             assert_attention_close(out.cpu().numpy().reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d), f"d512 w={window}")
     finally:
         os.environ.pop("TQ_DECODE_IMPL", None)
+
+
+def test_mixed_precision_attend_matches_oracle(gpu, oracle):
+    """Sec. 5 ablation path: K and V each from the int4 cache or from the unquantised fp16 values."""
+    tq, torch = gpu
+    sh = I.Shape("x", 2, 16, 2, 128, 128 ** -0.5, k_outlier_channels=4)
+    k, v = I.make_kv(sh, 600, 81)
+    lens = [600, 77]
+    host = oracle_cache(oracle, sh, k, v, 608, lens)
+    dev = device_cache(tq, torch, sh, k, v, 608, lens)
+    pad = lambda a: np.ascontiguousarray(np.pad(a, ((0, 0), (0, 0), (0, 8), (0, 0))))
+    kf, vf = torch.from_numpy(pad(k)).cuda(), torch.from_numpy(pad(v)).cuda()
+    q = I.make_q(sh, 81)
+    qd = torch.from_numpy(q).cuda()
+    for use_k, use_v in ((False, False), (True, False), (False, True), (True, True)):
+        o, m, l = tq.alloc_partials(sh.B, sh.H_q, sh.d, 3)
+        out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+        tq.tq_sdpa_mixed_precision_attend(dev, kf if use_k else None, vf if use_v else None, qd, sh.alpha, 3, o, m, l)
+        tq.tq_sdpa_int4_combine(o, m, l, out)
+        torch.cuda.synchronize()
+        ref = oracle.attention_mixed(host, k if use_k else None, v if use_v else None, q, sh.alpha)
+        assert_attention_close(out.cpu().numpy(), ref, f"mixed k_fp16={use_k} v_fp16={use_v}")

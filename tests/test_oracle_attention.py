@@ -230,3 +230,33 @@ def test_multi_query_is_causal_attention_of_each_query_token(oracle):
     a = sh.alpha * kd[0, 1, 48:58] @ q[0, 0, 3].astype(np.float64)
     w = np.exp(a - a.max())
     assert np.abs(outw[0, 0, 3] - (w / w.sum()) @ vd[0, 1, 48:58]).max() < 1e-12
+
+
+def test_mixed_precision_attention_reduces_to_its_two_ends(oracle):
+    sh = I.Shape("t", 2, 4, 2, 64, 0.125)
+    k, v = I.make_kv(sh, 80, 29)
+    cache = oracle.Cache(sh.B, sh.H_kv, 80, sh.d)
+    cache.append(k, v)
+    cache.lens[:] = [80, 33]
+    q = I.make_q(sh, 29)
+    # both sides from the cache: the C implementation of the definition
+    assert np.abs(oracle.attention_mixed(cache, None, None, q, sh.alpha) - oracle.attention(cache, q, sh.alpha)).max() < 1e-12
+    # both sides unquantised: attention on the fp16 inputs, independent of the cache contents
+    full = oracle.attention_mixed(cache, k, v, q, sh.alpha)
+    other = oracle.Cache(sh.B, sh.H_kv, 80, sh.d)
+    other.lens[:] = cache.lens
+    assert np.array_equal(oracle.attention_mixed(other, k, v, q, sh.alpha), full)
+    # one side each: equal to plain attention over a cache whose other side is exact, which is the case
+    # for values that int4 represents exactly (here V in {0..15}/4 per group with min 0 and max 15/4)
+    rng = np.random.default_rng(3)
+    v_exact = (rng.integers(0, 16, size=v.shape) / 4.0).astype(np.float16)
+    v_exact[..., 0::32] = 0.0
+    v_exact[..., 1::32] = 3.75
+    c2 = oracle.Cache(sh.B, sh.H_kv, 80, sh.d)
+    c2.append(k, v_exact)
+    vd = oracle.dequant_rows(c2.v_packed, c2.v_scale, c2.v_zero)
+    assert np.array_equal(vd, v_exact.astype(np.float64))
+    assert np.abs(oracle.attention_mixed(c2, None, v_exact, q, sh.alpha) - oracle.attention(c2, q, sh.alpha)).max() < 1e-12
+    # and the ablation's ordering is measurable: each variant differs from the unquantised result
+    for kk, vv in ((None, v), (k, None)):
+        assert np.abs(oracle.attention_mixed(cache, kk, vv, q, sh.alpha) - full).max() > 1e-4
