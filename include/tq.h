@@ -53,6 +53,7 @@ typedef enum tq_result {
 #define TQ_STATUS_EMPTY_SEQ 2  /* attention over a sequence with seq_lens[b] <= 0; its output is zero */
 #define TQ_STATUS_BAD_LEN 4    /* seq_lens[b] outside [0, S_cap]; treated as clamped to that range */
 #define TQ_STATUS_TIMEOUT 8    /* a bounded wait for an asynchronous copy ran out; that call's results are not valid */
+#define TQ_STATUS_BAD_PAGE 16  /* a page-table entry outside [0, num_pages) was met */
 
 #define TQ_GROUP 32         /* quantisation group size g (fixed) */
 #define TQ_SPLIT_QUANTUM 16 /* split boundaries fall on multiples of this many tokens */
@@ -79,9 +80,22 @@ typedef enum tq_result {
 #define TQ_BLOCK_TOKENS 16
 #define TQ_BLOCK_BYTES(d) (16 * ((d) + (d) / 4))
 typedef struct tq_kv_cache {
-  uint8_t* blocks;    /* [B][H_kv][S_cap/16][TQ_BLOCK_BYTES(d)] */
+  uint8_t* blocks;    /* [B][H_kv][S_cap/16][TQ_BLOCK_BYTES(d)]; with paging: the page pool, see below */
   int32_t* seq_lens;  /* [B] number of valid tokens per sequence (device memory, updated by append) */
   int32_t B, H_kv, S_cap, d;
+  /*
+   * Paging (optional; the paper's cache is one growing tensor per layer and it names cache management as its
+   * end-to-end overhead, Sec. 5 and 6.3; pages are the usual way to serve ragged batches from one pool).
+   * page_table == NULL: the contiguous layout above, the three integers are ignored.  Otherwise `blocks` is a
+   * pool [num_pages][H_kv][page_tokens/16][TQ_BLOCK_BYTES(d)], page_table is device memory
+   * [B][max_pages] int32, entry (b, i) names the pool page that holds tokens i*page_tokens ..
+   * (i+1)*page_tokens - 1 of sequence b (for all KV heads), and S_cap must equal max_pages * page_tokens.
+   * Only the entries below ceil(seq_lens[b] / page_tokens) (after an append: of the new length) are read.
+   * An entry outside [0, num_pages) sets TQ_STATUS_BAD_PAGE and is treated as page 0 by readers and
+   * skipped by writers.  page_tokens is a multiple of 16.  Every entry point takes either form.
+   */
+  const int32_t* page_table;
+  int32_t page_tokens, max_pages, num_pages;
 } tq_kv_cache;
 
 /* Byte offset inside a block of code byte `byte` (0 .. d/2-1) of token `t` (0 .. 15); which = 0 for K, 1 for V. */

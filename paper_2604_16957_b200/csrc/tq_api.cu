@@ -40,6 +40,12 @@ int check_cache(const tq_kv_cache* c) {
   if (c->B < 1 || c->B > 65535 || c->H_kv < 1 || c->H_kv > 4096 || c->S_cap < 16 || (c->S_cap % 16) != 0)
     return TQ_ERR_SHAPE;
   if (!aligned16(c->blocks) || (reinterpret_cast<uintptr_t>(c->seq_lens) & 3u)) return TQ_ERR_ALIGN;
+  if (c->page_table) {
+    if (c->page_tokens < 16 || (c->page_tokens % 16) != 0 || c->max_pages < 1 || c->num_pages < 1 ||
+        static_cast<long long>(c->page_tokens) * c->max_pages != c->S_cap)
+      return TQ_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(c->page_table) & 3u) return TQ_ERR_ALIGN;
+  }
   return TQ_OK;
 }
 

@@ -27,12 +27,14 @@ constexpr float kLn2 = 0.6931471805599453f;
 template <int D>
 struct SrcInt4 {
   static constexpr int EPL = D / 32;  // elements per lane
-  const uint8_t* blocks;
-  int S_cap;
+  tq_kv_cache c;
+  // row = (b * H_kv + kvh) * S_cap + token
   __device__ void load(bool is_v, long long row, int lane, float (&x)[EPL]) const {
-    const long long bh = row / S_cap;
-    const int tok = static_cast<int>(row - bh * S_cap);
-    const uint8_t* blk = blocks + block_base(bh, S_cap, D, tok);
+    const long long bh = row / c.S_cap;
+    const int tok = static_cast<int>(row - bh * c.S_cap);
+    const int b = static_cast<int>(bh / c.H_kv);
+    bool ok;
+    const uint8_t* blk = cache_block(c, b, static_cast<int>(bh - static_cast<long long>(b) * c.H_kv), tok, nullptr, ok);
     const int g = (lane * EPL) / 32;
     const float s = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(D, is_v, 0, g, tok & 15)));
     const float z = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(D, is_v, 1, g, tok & 15)));
@@ -204,7 +206,8 @@ __global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T
   const long long h = r / len;
   const int t = static_cast<int>(r - h * len);
   const long long row = (static_cast<long long>(b) * c.H_kv + h) * c.S_cap + t;
-  const uint8_t* blk = c.blocks + block_base(static_cast<long long>(b) * c.H_kv + h, c.S_cap, d, t);
+  bool ok;
+  const uint8_t* blk = cache_block(c, b, static_cast<int>(h), t, nullptr, ok);
   const uint32_t w = *reinterpret_cast<const uint32_t*>(blk + code_offset(d, is_v, t & 15, cc * 4));
   const float s = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 0, cc >> 2, t & 15)));
   const float z = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 1, cc >> 2, t & 15)));
@@ -229,7 +232,7 @@ cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q,
                                  int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
   auto run = [&](auto dtag) {
     constexpr int D = decltype(dtag)::value;
-    SrcInt4<D> src{c.blocks, c.S_cap};
+    SrcInt4<D> src{c};
     return launch_simple<D>(src, c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
   };
   switch (c.d) {
@@ -265,7 +268,7 @@ cudaError_t launch_attend_mixed(const tq_kv_cache& c, const __half* k_fp16, cons
                                 cudaStream_t st) {
   auto run = [&](auto dtag) {
     constexpr int D = decltype(dtag)::value;
-    SrcMixed<D> src{SrcInt4<D>{c.blocks, c.S_cap}, SrcMat<D, __half>{k_fp16, v_fp16}};
+    SrcMixed<D> src{SrcInt4<D>{c}, SrcMat<D, __half>{k_fp16, v_fp16}};
     return launch_simple<D>(src, c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
   };
   switch (c.d) {

@@ -318,14 +318,16 @@ __device__ __forceinline__ bool wait_stage(uint32_t bar, uint32_t parity) {
 // G * S_q (query token, head) pairs, v = s * G + g, packed into MMA columns like plain heads; query token s
 // is the (S_q - 1 - s)-th newest cached token and attends causally: tokens [lo_s, hi_s) with
 // hi_s = len - (S_q - 1 - s), lo_s = max(0, hi_s - window).  The plain instantiation carries none of this
-// arithmetic into the block loop.
-template <int D, bool GEN>
+// arithmetic into the block loop.  MODE: 0 plain, 1 general, 2 general over a paged cache (tq.h): the block
+// addresses then come from the page table, each entry fetched one block ahead of its use.
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, int S_q, float attn_scale, int window,
                       int C, float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
                       int32_t* status) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
+  constexpr bool GEN = MODE != 0, PAGED = MODE == 2;
   extern __shared__ __align__(1024) uint8_t smem[];
 
   const int G = H_q / cache.H_kv;
@@ -370,20 +372,50 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   if (DS > 1) __syncthreads();  // the team's other warps wait on these barriers too
   else __syncwarp();
-  // block j of this (sequence, KV head) starts at head_blocks + j * STAGE; one lane of the team copies it into a slot
+  // The team's n-th block is block blk0 + team + n * NTEAM of this (sequence, KV head); one lane of the team
+  // copies it into ring slot n mod NST.  Contiguous cache: it starts at head_blocks + block * STAGE.  Paged:
+  // page `pg` (the table entry, fetched ahead) holds [H_kv][page_tokens / 16] blocks.
   const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
-  auto issue = [&](int slot, int blk) {
+  const int bpp = PAGED ? cache.page_tokens >> 4 : 1;
+  auto page_of = [&](int n) -> int {
+    return cache.page_table[static_cast<long long>(b) * cache.max_pages + (blk0 + team + n * NTEAM) / bpp];
+  };
+  auto issue = [&](int n, int pg) {
     if (sub == 0 && lane == 0) {
+      const int slot = n & (Cf::NST - 1), blk = blk0 + team + n * NTEAM;
+      const uint8_t* src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
+      if (PAGED) {
+        if (pg < 0 || pg >= cache.num_pages) {
+          if (status) atomicOr(status, TQ_STATUS_BAD_PAGE);
+          pg = 0;
+        }
+        src = cache.blocks + ((static_cast<size_t>(pg) * cache.H_kv + kvh) * bpp + blk % bpp) * Cf::STAGE;
+      }
       const uint32_t bar = bars + 8 * slot;
       mbar_expect_tx(bar, Cf::STAGE);
-      bulk_g2s(ring_s + slot * Cf::STAGE, head_blocks + static_cast<size_t>(blk) * Cf::STAGE, Cf::STAGE, bar);
+      bulk_g2s(ring_s + slot * Cf::STAGE, src, Cf::STAGE, bar);
     }
   };
 
   // start streaming: the first stages are in flight while q is turned into fragments
+  int pg_next = 0;  // paged: table entry of the next block to be issued
+  {
+    int pre = 0;
+    if (PAGED && lane < Cf::NST && lane < nblk) pre = page_of(lane);  // the first entries, fetched side by side
 #pragma unroll
-  for (int s = 0; s < Cf::NST - 1; ++s)
-    if (s < nblk) issue(s, blk0 + team + s * NTEAM);
+    for (int s = 0; s < Cf::NST - 1; ++s) {
+      const int pg = PAGED ? __shfl_sync(0xffffffffu, pre, s) : 0;
+      if (s < nblk) issue(s, pg);
+    }
+    if (PAGED) pg_next = __shfl_sync(0xffffffffu, pre, Cf::NST - 1);
+  }
+  // issue the team's n-th block (if it has one) and fetch the table entry of the one after it
+  auto refill = [&](int n) {
+    if (n < nblk) {
+      issue(n, pg_next);
+      if (PAGED && n + 1 < nblk) pg_next = page_of(n + 1);
+    }
+  };
 
   // ---- q as MMA B fragments: column n = gid is column v0 + gid of the tile; k slots follow the nibble order.
   // qs[g][j] = 2^-24 * sum of q over group g for heads 2*tid4 + j (the zero-point term of the scores).
@@ -467,7 +499,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     if (DS == 1) {
       if (!arrived) { timed_out = true; break; }
       __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
-      if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + team + (k + Cf::NST - 1) * NTEAM);
+      refill(k + Cf::NST - 1);
     }
     const uint32_t st_s = ring_s + (k & (Cf::NST - 1)) * Cf::STAGE;
     const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
@@ -512,7 +544,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         bad |= xflag[(k & 1) * DS + w];
       }
       if (bad) { timed_out = true; break; }
-      if (k + Cf::NST - 1 < nblk) issue((k + Cf::NST - 1) & (Cf::NST - 1), blk0 + team + (k + Cf::NST - 1) * NTEAM);
+      refill(k + Cf::NST - 1);
       if (plain) block_softmax_pv<D, false>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       else block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
     }
@@ -601,23 +633,24 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
 }
 
-template <int D, bool GEN>
+template <int D, int MODE>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
                    float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D, GEN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 Cfg<D>::SMEM);
   if (attr != cudaSuccess) return attr;
   const int GV = (H_q / c.H_kv) * S_q;
   dim3 grid(C, c.H_kv * ((GV + 7) / 8), c.B);
-  return launch_kernel(decode_mma_kernel<D, GEN>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, S_q, attn_scale,
+  return launch_kernel(decode_mma_kernel<D, MODE>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, S_q, attn_scale,
                        window, C, o_part, m_part, l_part, status);
 }
 
 template <int D>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
                    float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  return (window > 0 || S_q > 1) ? launch<D, true>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st)
-                                 : launch<D, false>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
+  if (c.page_table != nullptr) return launch<D, 2>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+  return (window > 0 || S_q > 1) ? launch<D, 1>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st)
+                                 : launch<D, 0>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
 }
 
 }  // namespace

@@ -63,6 +63,27 @@ __host__ __device__ inline long long block_base(long long bh, int S_cap, int d, 
   return (bh * (S_cap >> 4) + (tok >> 4)) * static_cast<long long>(block_bytes(d));
 }
 
+// Index (in units of blocks) of the block that holds logical 16-token block j of (sequence b, KV head kvh),
+// contiguous or paged (see tq.h).  ok = false (paged only) when the page-table entry is outside the pool;
+// the index returned then refers to page 0.
+__device__ inline long long cache_block_index(const tq_kv_cache& c, int b, int kvh, int j, bool& ok) {
+  ok = true;
+  if (c.page_table == nullptr) return (static_cast<long long>(b) * c.H_kv + kvh) * (c.S_cap >> 4) + j;
+  const int bpp = c.page_tokens >> 4;
+  const int i = j / bpp;
+  int p = c.page_table[static_cast<long long>(b) * c.max_pages + i];
+  if (p < 0 || p >= c.num_pages) {
+    ok = false;
+    p = 0;
+  }
+  return (static_cast<long long>(p) * c.H_kv + kvh) * bpp + (j - i * bpp);
+}
+__device__ inline uint8_t* cache_block(const tq_kv_cache& c, int b, int kvh, int tok, int32_t* status, bool& ok) {
+  const long long idx = cache_block_index(c, b, kvh, tok >> 4, ok);
+  if (!ok && status) atomicOr(status, TQ_STATUS_BAD_PAGE);
+  return c.blocks + idx * block_bytes(c.d);
+}
+
 // Clamp a device-side sequence length into [0, S_cap], flagging bad or empty values.
 __device__ inline int checked_len(const int32_t* seq_lens, int b, int S_cap, int32_t* status) {
   int len = seq_lens[b];

@@ -92,7 +92,7 @@ __device__ __forceinline__ void quantize_chunk(const uint4 raw, bool active, uin
 
 // chunk index -> (b, h, t, c) of a [B][H_kv][T][d] tensor and the destination row in the cache
 __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half* src, int which, int T,
-                                              long long chunk, bool in_range, int b, int len) {
+                                              long long chunk, bool in_range, int b, int len, int32_t* status) {
   const int d = c.d;
   const int cpr = d >> 3;  // chunks per row
   uint4 raw = make_uint4(0, 0, 0, 0);
@@ -110,8 +110,9 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
     const long long bh = row_in / T;
     const int t = static_cast<int>(row_in - bh * T);
     const int tok = len + t;
-    (void)b;
-    uint8_t* blk = c.blocks + block_base(bh, c.S_cap, d, tok);
+    bool ok;
+    uint8_t* blk = cache_block(c, b, static_cast<int>(bh - static_cast<long long>(b) * c.H_kv), tok, status, ok);
+    if (!ok) return;  // a page outside the pool: nothing is written
     *reinterpret_cast<uint32_t*>(blk + code_offset(d, which, tok & 15, cc * 4)) = word;
     if ((cc & 3) == 0) {
       *reinterpret_cast<__half*>(blk + meta_offset(d, which, 0, cc >> 2, tok & 15)) = s;
@@ -127,7 +128,7 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
 // seq_lens is read only here and bumped by bump_lens_kernel afterwards, so that no block can observe a
 // length that another block of the same launch has already advanced.
 __global__ void __launch_bounds__(1024) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
-                                                            int T) {
+                                                             int T, int32_t* status) {
   __shared__ __align__(16) __half sm_meta[2][16][16];  // [scale | zero][group][token], up to d = 512
   pdl_wait();
   pdl_launch_dependents();
@@ -148,7 +149,10 @@ __global__ void __launch_bounds__(1024) quantize_bulk_kernel(tq_kv_cache c, cons
   uint32_t word;
   __half s, z;
   quantize_chunk(raw, active, word, s, z);
-  uint8_t* blk = c.blocks + block_base(bh, c.S_cap, d, 16 * j);
+  bool page_ok;
+  uint8_t* blk = cache_block(c, b, static_cast<int>(bh - static_cast<long long>(b) * c.H_kv), 16 * j,
+                             threadIdx.x == 0 ? status : nullptr, page_ok);
+  if (!page_ok) return;  // a page outside the pool: nothing is written (uniform over the block)
   if (active) *reinterpret_cast<uint32_t*>(blk + code_offset(d, which, t, cc * 4)) = word;
   const bool whole = tok_lo == 16 * j && tok_hi == 16 * j + 16;
   if ((cc & 3) == 0) {
@@ -202,7 +206,8 @@ __global__ void __launch_bounds__(256) quantize_step_kernel(tq_kv_cache c, const
     const bool is_v = i >= per_seq;
     const long long local = is_v ? i - per_seq : i;
     const bool in_range = i < 2 * per_seq;
-    process_chunk(c, is_v ? v_new : k_new, is_v ? 1 : 0, T, static_cast<long long>(b) * per_seq + local, in_range, b, len);
+    process_chunk(c, is_v ? v_new : k_new, is_v ? 1 : 0, T, static_cast<long long>(b) * per_seq + local, in_range, b, len,
+                  status);
   }
   __syncthreads();
   if (threadIdx.x == 0) c.seq_lens[b] = len + T;
@@ -217,7 +222,7 @@ cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, co
     return launch_kernel(quantize_step_kernel, dim3(c.B), dim3(256), 0, st, c, k_new, v_new, T, status);
   } else {
     dim3 grid(static_cast<unsigned>((T + 15) / 16 + 1), static_cast<unsigned>(c.B * c.H_kv), 2);
-    const cudaError_t e = launch_kernel(quantize_bulk_kernel, grid, dim3(2 * c.d), 0, st, c, k_new, v_new, T);
+    const cudaError_t e = launch_kernel(quantize_bulk_kernel, grid, dim3(2 * c.d), 0, st, c, k_new, v_new, T, status);
     if (e != cudaSuccess) return e;
     return launch_kernel(bump_lens_kernel, dim3((c.B + 127) / 128), dim3(128), 0, st, c, T, status);
   }

@@ -33,7 +33,8 @@ SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa
 
 class tq_kv_cache(C.Structure):
     _fields_ = [("blocks", C.c_void_p), ("seq_lens", C.c_void_p), ("B", C.c_int32), ("H_kv", C.c_int32),
-                ("S_cap", C.c_int32), ("d", C.c_int32)]
+                ("S_cap", C.c_int32), ("d", C.c_int32), ("page_table", C.c_void_p), ("page_tokens", C.c_int32),
+                ("max_pages", C.c_int32), ("num_pages", C.c_int32)]
 
 
 def TQ_BLOCK_BYTES(d):
@@ -114,7 +115,8 @@ class KVCache:
         self.seq_lens = torch.zeros((B,), dtype=torch.int32, device=device)
 
     def struct(self):
-        return tq_kv_cache(self.blocks.data_ptr(), self.seq_lens.data_ptr(), self.B, self.H_kv, self.S_cap, self.d)
+        return tq_kv_cache(self.blocks.data_ptr(), self.seq_lens.data_ptr(), self.B, self.H_kv, self.S_cap, self.d,
+                           None, 0, 0, 0)
 
     def arrays_token_major(self):
         """Decode the blocks into plain token-major arrays (copies, for inspection and tests):
@@ -136,6 +138,35 @@ class KVCache:
                 m = self.blocks[..., 16 * d + a * sz:16 * d + (a + 1) * sz].contiguous().view(torch.float16)
                 out.append(m.reshape(B, H, nb, ng, 16).permute(0, 1, 2, 4, 3).reshape(B, H, S, ng))
         return tuple(out)
+
+
+class PagedKVCache:
+    """The same cache served from a pool of pages: `blocks` is [num_pages][H_kv][page_tokens/16][block bytes],
+    `page_table` [B][max_pages] int32 names the pool page of every page_tokens-token stretch of a sequence."""
+
+    def __init__(self, B, H_kv, page_tokens, max_pages, num_pages, d, device="cuda"):
+        assert page_tokens % 16 == 0 and d in (64, 128, 256, 512)
+        self.B, self.H_kv, self.d = B, H_kv, d
+        self.page_tokens, self.max_pages, self.num_pages = page_tokens, max_pages, num_pages
+        self.S_cap = page_tokens * max_pages
+        self.blocks = torch.zeros((num_pages, H_kv, page_tokens // 16, TQ_BLOCK_BYTES(d)), dtype=torch.uint8, device=device)
+        self.page_table = torch.zeros((B, max_pages), dtype=torch.int32, device=device)
+        self.seq_lens = torch.zeros((B,), dtype=torch.int32, device=device)
+
+    def struct(self):
+        return tq_kv_cache(self.blocks.data_ptr(), self.seq_lens.data_ptr(), self.B, self.H_kv, self.S_cap, self.d,
+                           self.page_table.data_ptr(), self.page_tokens, self.max_pages, self.num_pages)
+
+    def contiguous(self):
+        """A KVCache holding the same logical contents (a copy gathered through the page table)."""
+        out = KVCache(self.B, self.H_kv, self.S_cap, self.d, device=self.blocks.device)
+        pages = self.blocks[self.page_table.long().clamp(0, self.num_pages - 1)]  # [B][max_pages][H_kv][bpp][bytes]
+        out.blocks.copy_(pages.permute(0, 2, 1, 3, 4).reshape(out.blocks.shape))
+        out.seq_lens.copy_(self.seq_lens)
+        return out
+
+    def arrays_token_major(self):
+        return self.contiguous().arrays_token_major()
 
 
 def _cs(cache):

@@ -418,3 +418,83 @@ def test_mixed_precision_attend_matches_oracle(gpu, oracle):
         torch.cuda.synchronize()
         ref = oracle.attention_mixed(host, k if use_k else None, v if use_v else None, q, sh.alpha)
         assert_attention_close(out.cpu().numpy(), ref, f"mixed k_fp16={use_k} v_fp16={use_v}")
+
+
+def _paged(tq, torch, sh, page_tokens, max_pages, seed):
+    """A paged cache whose page table is a seeded random assignment of distinct pool pages."""
+    num_pages = sh.B * max_pages + 3
+    cache = tq.PagedKVCache(sh.B, sh.H_kv, page_tokens, max_pages, num_pages, sh.d)
+    perm = np.random.default_rng(seed).permutation(num_pages)[:sh.B * max_pages].astype(np.int32)
+    cache.page_table.copy_(torch.from_numpy(perm.reshape(sh.B, max_pages)))
+    cache.blocks.fill_(0xFF)
+    return cache
+
+
+@pytest.mark.parametrize("d,H_q,H_kv,page_tokens", [(128, 16, 2, 64), (256, 8, 4, 16), (64, 4, 1, 48), (512, 32, 1, 32)])
+def test_paged_cache_append_and_decode(gpu, oracle, d, H_q, H_kv, page_tokens):
+    """The cache served from a pool of pages through a page table (random page assignment): bulk and
+    single-token appends are bit-exact against the oracle, decode (plain, windowed, several query tokens)
+    and the comparison path match it, and the result equals the contiguous cache's bit for bit."""
+    tq, torch = gpu
+    sh = I.Shape("x", 3, H_q, H_kv, d, d ** -0.5 if d < 256 else 1.0, sigma_qk=1.0 if d < 256 else 0.25)
+    S = 700
+    max_pages = (S + 40 + page_tokens - 1) // page_tokens
+    k, v = I.make_kv(sh, S, 91)
+    host = oracle.Cache(sh.B, sh.H_kv, page_tokens * max_pages, sh.d)
+    host.append(k, v)
+    dev = _paged(tq, torch, sh, page_tokens, max_pages, 91)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tq.tq_kv_quantize_append(dev, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
+    for step in range(3):
+        k1, v1 = I.make_kv(sh, 1, 91, stream=1 + step)
+        host.append(k1, v1)
+        tq.tq_kv_quantize_append(dev, torch.from_numpy(k1).cuda(), torch.from_numpy(v1).cuda(), status)
+    assert_cache_bits_equal(dev, host)
+    flat = dev.contiguous()
+    q = I.make_q(sh, 91)
+    for C in (0, 3):
+        out, o_p, _ = fused_attention(tq, torch, dev, q, sh.alpha, num_splits=C)
+        assert_attention_close(out, oracle.attention(host, q, sh.alpha), f"paged C={C}")
+        out_flat, o_f, _ = fused_attention(tq, torch, flat, q, sh.alpha, num_splits=C)
+        assert np.array_equal(out, out_flat)
+    q3 = np.ascontiguousarray(np.stack([I.make_q(sh, 91, stream=s) for s in range(3)], axis=1))
+    for window in (0, 100):
+        o, m, l = tq.alloc_partials(sh.B, sh.H_q * 3, sh.d, 2)
+        out = torch.empty((sh.B, 3, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+        tq.tq_sdpa_int4_decode_multi(dev, torch.from_numpy(q3).cuda(), sh.alpha, window, 2, o, m, l, status)
+        tq.tq_sdpa_int4_combine(o, m, l, out.view(sh.B, 3 * sh.H_q, sh.d))
+        ref = oracle.attention_multi(host, q3, sh.alpha, window)
+        assert_attention_close(out.cpu().numpy().reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d), f"paged w={window}")
+    # comparison path through the page table
+    need = tq.tq_dequant_workspace_bytes(sh.B, sh.H_kv, sh.H_q, dev.S_cap, sh.d, False)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+    tq.tq_sdpa_dequant_then_attend(dev, torch.from_numpy(q).cuda(), sh.alpha, ws, False, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert_attention_close(out.cpu().numpy(), oracle.attention(host, q, sh.alpha), "paged dequant-then-attend")
+
+
+def test_paged_cache_bad_page_is_flagged_not_followed(gpu, oracle):
+    tq, torch = gpu
+    sh = I.Shape("x", 2, 8, 2, 128, 0.1)
+    dev = _paged(tq, torch, sh, 32, 4, 5)
+    k, v = I.make_kv(sh, 100, 5)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tq.tq_kv_quantize_append(dev, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    before = dev.blocks.clone()
+    dev.page_table[1, 1] = dev.num_pages + 7   # tokens 32..63 of sequence 1
+    dev.page_table[0, 3] = -1                  # tokens 96..127 of sequence 0 (the next append lands there)
+    q = I.make_q(sh, 5)
+    out, _, _ = fused_attention(tq, torch, dev, q, sh.alpha, num_splits=2, status=status)
+    assert int(status.item()) & 16                 # flagged; the reads went to pool page 0, not out of bounds
+    assert np.all(np.isfinite(out[0]))             # sequence 0's bad entry lies beyond its length and is never read
+    status.zero_()
+    k1, v1 = I.make_kv(sh, 1, 5, stream=1)
+    tq.tq_kv_quantize_append(dev, torch.from_numpy(k1).cuda(), torch.from_numpy(v1).cuda(), status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & 16
+    changed = (dev.blocks != before).flatten(1).any(dim=1).cpu().numpy()
+    assert changed.sum() == 1 and changed[int(dev.page_table[1, 3])]  # only sequence 1's page was written
