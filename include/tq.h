@@ -92,7 +92,7 @@ typedef struct tq_kv_cache {
    * (i+1)*page_tokens - 1 of sequence b (for all KV heads), and S_cap must equal max_pages * page_tokens.
    * Only the entries below ceil(seq_lens[b] / page_tokens) (after an append: of the new length) are read.
    * An entry outside [0, num_pages) sets TQ_STATUS_BAD_PAGE and is treated as page 0 by readers and
-   * skipped by writers.  page_tokens is a multiple of 16.  Every entry point takes either form.
+   * skipped by writers.  page_tokens is a power of two, at least 16.  Every entry point takes either form.
    */
   const int32_t* page_table;
   int32_t page_tokens, max_pages, num_pages;

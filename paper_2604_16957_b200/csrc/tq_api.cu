@@ -41,8 +41,9 @@ int check_cache(const tq_kv_cache* c) {
     return TQ_ERR_SHAPE;
   if (!aligned16(c->blocks) || (reinterpret_cast<uintptr_t>(c->seq_lens) & 3u)) return TQ_ERR_ALIGN;
   if (c->page_table) {
-    if (c->page_tokens < 16 || (c->page_tokens % 16) != 0 || c->max_pages < 1 || c->num_pages < 1 ||
-        static_cast<long long>(c->page_tokens) * c->max_pages != c->S_cap)
+    if (c->page_tokens < 16 || (c->page_tokens & (c->page_tokens - 1)) != 0 || c->max_pages < 1 || c->num_pages < 1 ||
+        static_cast<long long>(c->page_tokens) * c->max_pages != c->S_cap ||
+        static_cast<long long>(c->num_pages) * c->H_kv * (c->page_tokens / 16) > 0x7fffffffLL)
       return TQ_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(c->page_table) & 3u) return TQ_ERR_ALIGN;
   }

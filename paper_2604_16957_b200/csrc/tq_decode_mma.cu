@@ -376,20 +376,25 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // copies it into ring slot n mod NST.  Contiguous cache: it starts at head_blocks + block * STAGE.  Paged:
   // page `pg` (the table entry, fetched ahead) holds [H_kv][page_tokens / 16] blocks.
   const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
-  const int bpp = PAGED ? cache.page_tokens >> 4 : 1;
-  auto page_of = [&](int n) -> int {
-    return cache.page_table[static_cast<long long>(b) * cache.max_pages + (blk0 + team + n * NTEAM) / bpp];
+  // page_tokens is a power of two, so block j sits in table entry j >> pshift at offset j & (bpp - 1).
+  const int pshift = PAGED ? 31 - __clz(cache.page_tokens >> 4) : 0;
+  auto table_entry = [&](int n) -> int {
+    return cache.page_table[static_cast<long long>(b) * cache.max_pages + ((blk0 + team + n * NTEAM) >> pshift)];
   };
   auto issue = [&](int n, int pg) {
     if (sub == 0 && lane == 0) {
       const int slot = n & (Cf::NST - 1), blk = blk0 + team + n * NTEAM;
-      const uint8_t* src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
+      const uint8_t* src;
       if (PAGED) {
-        if (pg < 0 || pg >= cache.num_pages) {
+        if (static_cast<uint32_t>(pg) >= static_cast<uint32_t>(cache.num_pages)) {
           if (status) atomicOr(status, TQ_STATUS_BAD_PAGE);
           pg = 0;
         }
-        src = cache.blocks + ((static_cast<size_t>(pg) * cache.H_kv + kvh) * bpp + blk % bpp) * Cf::STAGE;
+        // block index in the pool (fits 32 bits: the pool is checked to hold fewer than 2^31 blocks)
+        const uint32_t idx = ((static_cast<uint32_t>(pg) * cache.H_kv + kvh) << pshift) + (blk & ((1 << pshift) - 1));
+        src = cache.blocks + static_cast<size_t>(idx) * Cf::STAGE;
+      } else {
+        src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
       }
       const uint32_t bar = bars + 8 * slot;
       mbar_expect_tx(bar, Cf::STAGE);
@@ -400,8 +405,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // start streaming: the first stages are in flight while q is turned into fragments
   int pg_next = 0;  // paged: table entry of the next block to be issued
   {
-    int pre = 0;
-    if (PAGED && lane < Cf::NST && lane < nblk) pre = page_of(lane);  // the first entries, fetched side by side
+    int pre = 0;  // the first NST entries, fetched side by side
+    if (PAGED && lane < Cf::NST && lane < nblk) pre = table_entry(lane);
 #pragma unroll
     for (int s = 0; s < Cf::NST - 1; ++s) {
       const int pg = PAGED ? __shfl_sync(0xffffffffu, pre, s) : 0;
@@ -413,7 +418,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   auto refill = [&](int n) {
     if (n < nblk) {
       issue(n, pg_next);
-      if (PAGED && n + 1 < nblk) pg_next = page_of(n + 1);
+      if (PAGED && n + 1 < nblk) pg_next = table_entry(n + 1);
     }
   };
 
@@ -461,17 +466,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const int rem_last = t1 - (blk0 + team + (nblk - 1) * NTEAM) * kBlk;  // tokens in this team's last block
   int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;          // this team's blocks k < nfull are full
   int nhead = 0;                                                        // ... and blocks k < nhead are masked
-  int lo0 = 0, hi0 = 0, lo1 = 0, hi1 = 0;                               // token ranges of this thread's two columns
   if (GEN) {
-    const int s0 = min((v0 + 2 * tid4) / G, S_q - 1), s1 = min((v0 + 2 * tid4 + 1) / G, S_q - 1);
-    hi0 = query_hi(len, S_q, s0); lo0 = window_begin(hi0, window);
-    hi1 = query_hi(len, S_q, s1); lo1 = window_begin(hi1, window);
     const int full_end = min(t1, query_hi(len, S_q, 0)) >> 4;                   // blocks below it end inside every range
     const int full_begin = (query_lo(len, S_q, S_q - 1, window) + kBlk - 1) >> 4;  // blocks from it on begin inside
     const int first_blk = blk0 + team;
     nfull = full_end > first_blk ? min(nblk, (full_end - first_blk + NTEAM - 1) / NTEAM) : 0;
     nhead = full_begin > first_blk ? min(nblk, (full_begin - first_blk + NTEAM - 1) / NTEAM) : 0;
   }
+  const unsigned nplain = nfull > nhead ? nfull - nhead : 0;  // general form: blocks nhead <= k < nhead + nplain are full
   // per-lane byte offsets inside a stage: ldmatrix row addresses of the code, scale and zero fragments of
   // this warp's channel groups sub * NGW .. (see block_scores / block_softmax_pv)
   WarpCtx<D> cx;
@@ -503,12 +505,21 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     }
     const uint32_t st_s = ring_s + (k & (Cf::NST - 1)) * Cf::STAGE;
     const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
-    const bool plain = k < nfull && !(GEN && k < nhead);
+    const bool plain = GEN ? static_cast<unsigned>(k - nhead) < nplain : k < nfull;
     auto mask_of_block = [&]() {
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
       if (GEN) {
+        // token ranges of this thread's two columns, worked out here (masked blocks are rare) rather than
+        // kept in registers across the loop
+        const int n = checked_len(cache.seq_lens, blockIdx.z, cache.S_cap, nullptr);
+        int a, e;  // this split's token range, as at the top of the kernel
+        split_range(query_lo(n, S_q, 0, window), n, C, blockIdx.x, a, e);
+        const int col = (blockIdx.y % tiles) * 8 + 2 * (threadIdx.x & 3);
+        const int s0 = min(col / G, S_q - 1), s1 = min((col + 1) / G, S_q - 1);
+        const int hi0 = query_hi(n, S_q, s0), hi1 = query_hi(n, S_q, s1);
         const int first = (blk0 + team + k * NTEAM) * kBlk;  // first token of this block
-        mk = RowMask{t1 - first, lo0 - first, min(hi0, t1) - first, lo1 - first, min(hi1, t1) - first};
+        mk = RowMask{e - first, window_begin(hi0, window) - first, min(hi0, e) - first,
+                     window_begin(hi1, window) - first, min(hi1, e) - first};
       }
       return mk;
     };

@@ -145,7 +145,7 @@ class PagedKVCache:
     `page_table` [B][max_pages] int32 names the pool page of every page_tokens-token stretch of a sequence."""
 
     def __init__(self, B, H_kv, page_tokens, max_pages, num_pages, d, device="cuda"):
-        assert page_tokens % 16 == 0 and d in (64, 128, 256, 512)
+        assert page_tokens >= 16 and page_tokens & (page_tokens - 1) == 0 and d in (64, 128, 256, 512)
         self.B, self.H_kv, self.d = B, H_kv, d
         self.page_tokens, self.max_pages, self.num_pages = page_tokens, max_pages, num_pages
         self.S_cap = page_tokens * max_pages

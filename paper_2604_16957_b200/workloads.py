@@ -18,17 +18,27 @@ import torch
 from . import tq
 
 L2_BYTES = 126 << 20
+IDENTITY_PAGES = False  # --identity-pages: page i of a paged cache is pool page i (default: a random assignment)
 
 
-def _fill(B, H_kv, S_cap, d, n_caches, seed, outliers, sigma=1.0, lens=None):
-    """n_caches quantised caches filled to S_cap tokens; lens (if given) then overrides the lengths."""
+def _fill(B, H_kv, S_cap, d, n_caches, seed, outliers, sigma=1.0, lens=None, page_tokens=0):
+    """n_caches quantised caches filled to S_cap tokens; lens (if given) then overrides the lengths.
+    page_tokens > 0: paged caches, each with a seeded random page assignment."""
     gen = torch.Generator(device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     caches = []
     chunk = max(1, min(S_cap, (256 << 20) // (B * H_kv * d * 4)))  // 16 * 16 or 16
     for i in range(n_caches):
         gen.manual_seed(seed + i)
-        cache = tq.KVCache(B, H_kv, S_cap, d)
+        if page_tokens:
+            mp = S_cap // page_tokens
+            cache = tq.PagedKVCache(B, H_kv, page_tokens, mp, B * mp, d)
+            perm = torch.randperm(B * mp, generator=torch.Generator().manual_seed(seed + i)).int()
+            if IDENTITY_PAGES:
+                perm = torch.arange(B * mp, dtype=torch.int32)
+            cache.page_table.copy_(perm.view(B, mp))
+        else:
+            cache = tq.KVCache(B, H_kv, S_cap, d)
         ch = torch.randperm(d, generator=torch.Generator().manual_seed(seed))[:4].cuda()
         for t0 in range(0, S_cap, chunk):
             T = min(chunk, S_cap - t0)
@@ -78,13 +88,15 @@ def _emit(name, us, alg_bytes, **kw):
 
 
 def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, sigma=1.0, window=0, S_q=1, lens=None,
-                    with_append=False, compare=False, splits=0):
+                    with_append=False, compare=False, splits=0, page_tokens=0):
     """Times decode + combine (optionally preceded by a T = S_q append) over rotating caches."""
     per_tok = 2 * (d // 2 + d // 8)
     S_cap = (S + 15) // 16 * 16 + (64 if with_append else 0)
+    if page_tokens:
+        S_cap = -(-S_cap // page_tokens) * page_tokens
     cache_bytes = B * H_kv * S_cap * per_tok
     n = _n_caches(cache_bytes)
-    caches = _fill(B, H_kv, S_cap, d, n, 31, outliers, sigma, lens if lens is not None else [S] * B)
+    caches = _fill(B, H_kv, S_cap, d, n, 31, outliers, sigma, lens if lens is not None else [S] * B, page_tokens)
     base_lens = torch.as_tensor(lens if lens is not None else [S] * B, dtype=torch.int32).cuda()
     span = window or S
     C = splits or tq.tq_auto_splits(B, H_kv, H_q * S_q, d, span)
@@ -127,7 +139,7 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
 
         extra["dequant_then_attend_us"] = round(_time(enqueue_cmp, max(2, steps // 4), 1) / n * 1e6, 1)
     _emit(name, us, alg, B=B, H_q=H_q, H_kv=H_kv, d=d, S=S if lens is None else "ragged", S_q=S_q, window=window,
-          num_splits=C, caches_rotated=n, includes="append+decode+combine" if with_append else "decode+combine", **extra)
+          num_splits=C, caches_rotated=n, page_tokens=page_tokens, includes="append+decode+combine" if with_append else "decode+combine", **extra)
 
 
 def bulk_quantize_workload(steps, warmup):
@@ -170,6 +182,15 @@ WORKLOADS = {
     "ragged_b16": lambda a: decode_workload("ragged batch B=16, lengths U{4096..65536}", 16, 64, 8, 128, 65536,
                                             128 ** -0.5, a.steps, a.warmup, True, lens=ragged_lengths(),
                                             with_append=True, compare=a.splits == 0, splits=a.splits),
+    "ragged_b16_paged": lambda a: decode_workload("ragged batch B=16, lengths U{4096..65536}, 256-token pages", 16, 64, 8,
+                                                  128, 65536, 128 ** -0.5, a.steps, a.warmup, True,
+                                                  lens=ragged_lengths(), with_append=True, splits=a.splits,
+                                                  page_tokens=256),
+    "llama_32k_paged": lambda a: decode_workload("llama shape, 32K context, 64-token pages", 1, 64, 8, 128, 32768,
+                                                 128 ** -0.5, a.steps, a.warmup, True, page_tokens=64),
+    "ragged_b16_general": lambda a: decode_workload("ragged batch B=16, general kernel (window 2^30)", 16, 64, 8, 128, 65536,
+                                                    128 ** -0.5, a.steps, a.warmup, True, lens=ragged_lengths(),
+                                                    with_append=True, splits=a.splits or 10, window=1 << 30),
     "batch16_32k": lambda a: decode_workload("batch B=16, equal lengths 32K", 16, 64, 8, 128, 32768, 128 ** -0.5, a.steps,
                                              a.warmup, True, with_append=True, splits=a.splits),
     "bulk_quantize": lambda a: bulk_quantize_workload(a.steps, a.warmup),
@@ -182,7 +203,10 @@ def main():
     ap.add_argument("--splits", type=int, default=0, help="sequence splits for the batch workloads (0 = library default)")
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--identity-pages", action="store_true", help="paged workloads: pool page i holds page i")
     args = ap.parse_args()
+    global IDENTITY_PAGES
+    IDENTITY_PAGES = args.identity_pages
     assert torch.cuda.is_available(), "needs a CUDA device (there is no CPU path)"
     for name, fn in WORKLOADS.items():
         if args.only in (None, name):
