@@ -6,8 +6,8 @@ cosine 0.998 for int4 K with full-precision V and 0.994 for full-precision K wit
 Runs tq_sdpa_mixed_precision_attend four times on the same seeded inputs -- K and V each either the int4
 cache or the unquantised fp16 values -- and prints, per variant, the mean and minimum over heads of the
 cosine similarity between its output and the all-fp16 output.  Inputs: the Llama-shaped generator of the
-parity tests (N(0,1), four K channels x10 per KV head) and a second set with peaked attention (q scaled
-x4), where few tokens dominate the softmax.  Needs a CUDA device.
+parity tests -- plain N(0,1); with four K channels x10 per KV head; and the latter with peaked attention
+(q scaled x4), where few tokens dominate the softmax.  Needs a CUDA device.
 """
 import argparse
 import json
@@ -24,8 +24,8 @@ def cosines(a, b):
     return ((a * b).sum(-1) / (a.norm(dim=-1) * b.norm(dim=-1))).flatten()
 
 
-def run(context, seed, q_gain):
-    sh = I.Shape("llama", 1, 64, 8, 128, 128 ** -0.5, k_outlier_channels=4)
+def run(context, seed, q_gain, outliers):
+    sh = I.Shape("llama", 1, 64, 8, 128, 128 ** -0.5, k_outlier_channels=outliers)
     k, v = I.make_kv(sh, context, seed)
     q = (I.make_q(sh, seed).astype(np.float32) * q_gain).astype(np.float16)
     kd, vd, qd = (torch.from_numpy(np.ascontiguousarray(x)).cuda() for x in (k, v, q))
@@ -45,7 +45,7 @@ def run(context, seed, q_gain):
     ref = outs["fp16 K, fp16 V"]
     for name, out in outs.items():
         c = cosines(out, ref)
-        print(json.dumps({"context": context, "q_gain": q_gain, "variant": name, "cosine_mean": round(float(c.mean()), 5),
+        print(json.dumps({"context": context, "k_outlier_channels": outliers, "q_gain": q_gain, "variant": name, "cosine_mean": round(float(c.mean()), 5),
                           "cosine_min": round(float(c.min()), 5)}), flush=True)
 
 
@@ -55,8 +55,8 @@ def main():
     ap.add_argument("--seed", type=int, default=11)
     args = ap.parse_args()
     assert torch.cuda.is_available(), "needs a CUDA device (there is no CPU path)"
-    for gain in (1.0, 4.0):
-        run(args.context, args.seed, gain)
+    for outliers, gain in ((0, 1.0), (4, 1.0), (4, 4.0)):
+        run(args.context, args.seed, gain, outliers)
 
 
 if __name__ == "__main__":

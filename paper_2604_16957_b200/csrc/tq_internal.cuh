@@ -78,6 +78,16 @@ __device__ inline long long cache_block_index(const tq_kv_cache& c, int b, int k
   }
   return (static_cast<long long>(p) * c.H_kv + kvh) * bpp + (j - i * bpp);
 }
+// The same from bh = b * H_kv + kvh (what the quantiser has at hand); the contiguous case stays three instructions.
+__device__ inline uint8_t* cache_block_bh(const tq_kv_cache& c, long long bh, int b, int tok, int32_t* status, bool& ok) {
+  if (c.page_table == nullptr) {
+    ok = true;
+    return c.blocks + (bh * (c.S_cap >> 4) + (tok >> 4)) * block_bytes(c.d);
+  }
+  const long long idx = cache_block_index(c, b, static_cast<int>(bh - static_cast<long long>(b) * c.H_kv), tok >> 4, ok);
+  if (!ok && status) atomicOr(status, TQ_STATUS_BAD_PAGE);
+  return c.blocks + idx * block_bytes(c.d);
+}
 __device__ inline uint8_t* cache_block(const tq_kv_cache& c, int b, int kvh, int tok, int32_t* status, bool& ok) {
   const long long idx = cache_block_index(c, b, kvh, tok >> 4, ok);
   if (!ok && status) atomicOr(status, TQ_STATUS_BAD_PAGE);

@@ -111,7 +111,7 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
     const int t = static_cast<int>(row_in - bh * T);
     const int tok = len + t;
     bool ok;
-    uint8_t* blk = cache_block(c, b, static_cast<int>(bh - static_cast<long long>(b) * c.H_kv), tok, status, ok);
+    uint8_t* blk = cache_block_bh(c, bh, b, tok, status, ok);
     if (!ok) return;  // a page outside the pool: nothing is written
     *reinterpret_cast<uint32_t*>(blk + code_offset(d, which, tok & 15, cc * 4)) = word;
     if ((cc & 3) == 0) {
@@ -127,8 +127,11 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
 // grid: (blocks touched per sequence, B * H_kv, {K, V}); 2 * d threads (one per 8 elements).
 // seq_lens is read only here and bumped by bump_lens_kernel afterwards, so that no block can observe a
 // length that another block of the same launch has already advanced.
-__global__ void __launch_bounds__(1024) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
-                                                             int T, int32_t* status) {
+// THREADS = the largest block this instantiation is launched with (1024 only for d = 512, so that the
+// common head dimensions keep the register budget of a 512-thread block).
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
+                                                                int T, int32_t* status) {
   __shared__ __align__(16) __half sm_meta[2][16][16];  // [scale | zero][group][token], up to d = 512
   pdl_wait();
   pdl_launch_dependents();
@@ -150,8 +153,7 @@ __global__ void __launch_bounds__(1024) quantize_bulk_kernel(tq_kv_cache c, cons
   __half s, z;
   quantize_chunk(raw, active, word, s, z);
   bool page_ok;
-  uint8_t* blk = cache_block(c, b, static_cast<int>(bh - static_cast<long long>(b) * c.H_kv), 16 * j,
-                             threadIdx.x == 0 ? status : nullptr, page_ok);
+  uint8_t* blk = cache_block_bh(c, bh, b, 16 * j, threadIdx.x == 0 ? status : nullptr, page_ok);
   if (!page_ok) return;  // a page outside the pool: nothing is written (uniform over the block)
   if (active) *reinterpret_cast<uint32_t*>(blk + code_offset(d, which, t, cc * 4)) = word;
   const bool whole = tok_lo == 16 * j && tok_hi == 16 * j + 16;
@@ -222,7 +224,9 @@ cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, co
     return launch_kernel(quantize_step_kernel, dim3(c.B), dim3(256), 0, st, c, k_new, v_new, T, status);
   } else {
     dim3 grid(static_cast<unsigned>((T + 15) / 16 + 1), static_cast<unsigned>(c.B * c.H_kv), 2);
-    const cudaError_t e = launch_kernel(quantize_bulk_kernel, grid, dim3(2 * c.d), 0, st, c, k_new, v_new, T, status);
+    const cudaError_t e =
+        c.d > 256 ? launch_kernel(quantize_bulk_kernel<1024>, grid, dim3(2 * c.d), 0, st, c, k_new, v_new, T, status)
+                  : launch_kernel(quantize_bulk_kernel<512>, grid, dim3(2 * c.d), 0, st, c, k_new, v_new, T, status);
     if (e != cudaSuccess) return e;
     return launch_kernel(bump_lens_kernel, dim3((c.B + 127) / 128), dim3(128), 0, st, c, T, status);
   }
