@@ -155,7 +155,6 @@ __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_c
 
 template <int D>
 struct WarpCtx {
-  uint8_t* ring;
   uint32_t kaddr[Cfg<D>::NGW / 2];  // ldmatrix row address (offset in a stage) this lane supplies, per K load
   uint32_t vaddr[Cfg<D>::NGW / 2];  // same for the V loads
   uint32_t ksz_lane, vsz_lane;
@@ -302,6 +301,21 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
     mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1 & kMaskHi, y2 & kMaskLo, y2 & kMaskHi, b0, b1);
   }
+}
+
+// Row mask of a block that holds an end of some column's token range (general form).  Masked blocks are
+// rare, so this is a real call: whatever it needs is recomputed from the launch arguments instead of
+// being kept in registers across the block loop.  `col` = the thread's first score column in the KV head,
+// `first` = the block's first token.
+__device__ __noinline__ RowMask general_row_mask(const int32_t* seq_lens, int b, int S_cap, int S_q, int window, int C,
+                                                 int c, int G, int col, int first) {
+  const int n = checked_len(seq_lens, b, S_cap, nullptr);
+  int a, e;  // this split's token range, as at the top of the kernel
+  split_range(query_lo(n, S_q, 0, window), n, C, c, a, e);
+  const int s0 = min(col / G, S_q - 1), s1 = min((col + 1) / G, S_q - 1);
+  const int hi0 = query_hi(n, S_q, s0), hi1 = query_hi(n, S_q, s1);
+  return RowMask{e - first, window_begin(hi0, window) - first, min(hi0, e) - first, window_begin(hi1, window) - first,
+                 min(hi1, e) - first};
 }
 
 // Bounded wait on an mbarrier phase; false if the copy did not complete within the limit.
@@ -477,7 +491,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // per-lane byte offsets inside a stage: ldmatrix row addresses of the code, scale and zero fragments of
   // this warp's channel groups sub * NGW .. (see block_scores / block_softmax_pv)
   WarpCtx<D> cx;
-  cx.ring = ring; cx.cs = cs; cx.gid = gid;
+  cx.cs = cs; cx.gid = gid;
   cx.ksz_lane = 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32 + sub * NGW * 32;
   cx.vsz_lane = 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
 #pragma unroll
@@ -509,17 +523,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     auto mask_of_block = [&]() {
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
       if (GEN) {
-        // token ranges of this thread's two columns, worked out here (masked blocks are rare) rather than
-        // kept in registers across the loop
-        const int n = checked_len(cache.seq_lens, blockIdx.z, cache.S_cap, nullptr);
-        int a, e;  // this split's token range, as at the top of the kernel
-        split_range(query_lo(n, S_q, 0, window), n, C, blockIdx.x, a, e);
-        const int col = (blockIdx.y % tiles) * 8 + 2 * (threadIdx.x & 3);
-        const int s0 = min(col / G, S_q - 1), s1 = min((col + 1) / G, S_q - 1);
-        const int hi0 = query_hi(n, S_q, s0), hi1 = query_hi(n, S_q, s1);
-        const int first = (blk0 + team + k * NTEAM) * kBlk;  // first token of this block
-        mk = RowMask{e - first, window_begin(hi0, window) - first, min(hi0, e) - first,
-                     window_begin(hi1, window) - first, min(hi1, e) - first};
+        mk = general_row_mask(cache.seq_lens, blockIdx.z, cache.S_cap, S_q, window, C, blockIdx.x, H_q / cache.H_kv,
+                              (blockIdx.y % tiles) * 8 + 2 * (threadIdx.x & 3), (blk0 + team + k * NTEAM) * kBlk);
       }
       return mk;
     };

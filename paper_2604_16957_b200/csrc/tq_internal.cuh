@@ -58,11 +58,6 @@ __host__ __device__ inline int meta_offset(int d, int which, int is_zero, int g,
   const int ng = d >> 5;
   return 16 * d + (2 * which + is_zero) * (ng * 32) + (g * 16 + t) * 2;
 }
-// first byte of the block that holds token tok of (sequence * H_kv + head) bh
-__host__ __device__ inline long long block_base(long long bh, int S_cap, int d, int tok) {
-  return (bh * (S_cap >> 4) + (tok >> 4)) * static_cast<long long>(block_bytes(d));
-}
-
 // Index (in units of blocks) of the block that holds logical 16-token block j of (sequence b, KV head kvh),
 // contiguous or paged (see tq.h).  ok = false (paged only) when the page-table entry is outside the pool;
 // the index returned then refers to page 0.
