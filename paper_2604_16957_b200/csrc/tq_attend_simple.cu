@@ -76,7 +76,8 @@ struct SrcMixed {
 };
 
 // grid: (C, H_kv * head_tiles, B); block: kWarps warps.
-template <int D, typename Src>
+// GEN = sliding window and / or several query tokens: per-pair token ranges are checked inside the token loop.
+template <int D, typename Src, bool GEN>
 __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, const int32_t* seq_lens, int H_kv,
                                                                     int S_cap, const __half* q, int H_q, int S_q,
                                                                     float attn_scale, int window, int C, float* o_part,
@@ -123,7 +124,7 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
     src.load(true, row0 + i, lane, vx);
 #pragma unroll
     for (int h = 0; h < kHeadTile; ++h) {
-      if (i < lo[h] || i >= hi[h]) continue;
+      if (GEN && (i < lo[h] || i >= hi[h])) continue;
       float dot = 0.f;
 #pragma unroll
       for (int e = 0; e < EPL; ++e) dot = fmaf(qr[h][e], kx[e], dot);
@@ -183,8 +184,12 @@ cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q,
   const int GV = (H_q / c.H_kv) * S_q;
   const int tiles = (GV + kHeadTile - 1) / kHeadTile;
   dim3 grid(C, c.H_kv * tiles, c.B);
-  attend_simple_kernel<D, Src><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, S_q, attn_scale,
-                                                             window, C, o_part, m_part, l_part, status);
+  if (S_q > 1 || window > 0)
+    attend_simple_kernel<D, Src, true><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, S_q,
+                                                                     attn_scale, window, C, o_part, m_part, l_part, status);
+  else
+    attend_simple_kernel<D, Src, false><<<grid, kWarps * 32, 0, st>>>(src, c.seq_lens, c.H_kv, c.S_cap, q, H_q, 1,
+                                                                      attn_scale, 0, C, o_part, m_part, l_part, status);
   return cudaGetLastError();
 }
 
