@@ -15,22 +15,52 @@ namespace tq {
 namespace {
 
 
-// Redo the flagged elements with the defining arithmetic (true division).  Kept out of line so that the
-// common path carries no division code.
-__device__ __noinline__ uint32_t exact_codes(const float (&x)[8], float sf, float zf, uint32_t word, uint32_t unsure) {
-  for (int i = 0; i < 8; ++i) {
-    if (unsure & (1u << i)) {
-      const float u = fminf(fmaxf(__fadd_rn(__fdiv_rn(x[i], sf), zf), 0.0f), 15.0f);
-      const uint32_t q = __float_as_uint(u + 12582912.0f) & 0xFu;
-      word = (word & ~(0xFu << (4 * i))) | (q << (4 * i));
-    }
+struct QuantOut {
+  uint32_t word;  // eight codes, element i in bits 4i .. 4i+3
+  __half s, z;    // stored scale and zero of the group
+};
+
+// The defining arithmetic, step by step (true divisions, explicit roundings): what every result must be equal
+// to, bit for bit.  Out of line: the fast path below hands over whenever it cannot prove its own result.
+__device__ __noinline__ QuantOut quantize_exact(const float (&x)[8], float mn, float mx) {
+  QuantOut out;
+  out.word = 0u;
+  const float s32 = __fdiv_rn(__fsub_rn(mx, mn), 15.0f);
+  const __half s16 = __float2half_rn(s32);
+  if ((__half_as_ushort(s16) & 0x7FFFu) == 0) {  // scale rounds to zero: constant (or nearly constant) group
+    out.s = __ushort_as_half(0x3C00u);            // 1.0
+    out.z = __float2half_rn(__fsub_rn(0.0f, mn));
+    return out;
   }
-  return word;
+  const float sf = __half2float(s16);
+  float z32 = __fdiv_rn(__fsub_rn(0.0f, mn), sf);
+  z32 = fminf(fmaxf(z32, -65504.0f), 65504.0f);
+  const __half z16 = __float2half_rn(z32);
+  const float zf = __half2float(z16);
+  for (int i = 0; i < 8; ++i) {
+    const float u = fminf(fmaxf(__fadd_rn(__fdiv_rn(x[i], sf), zf), 0.0f), 15.0f);  // fmaxf also turns NaN into 0
+    out.word |= (__float_as_uint(u + 12582912.0f) & 0xFu) << (4 * i);             // rint, ties to even
+  }
+  out.s = s16;
+  out.z = z16;
+  return out;
 }
 
 // Quantise the 8 elements held by this thread (quad = one group).  All 32 lanes must call.
-__device__ __forceinline__ void quantize_chunk(const uint4 raw, bool active, uint32_t& word, __half& s_out,
-                                               __half& z_out) {
+//
+// Defining arithmetic: s = fp16((max - min) / 15), z = fp16(clamp((0 - min) / s)), u = fl(fl(x / s) + z),
+// q = clamp(rint(u), 0, 15), every operation rounded to nearest even in binary32.  A division, a round, two
+// clamps and a conversion per element would make this kernel many times slower than the memory system, so
+// the common case does less and proves that it changed nothing:
+//   ua = fma(x, 1/s, z) with the correctly rounded reciprocal differs from u by at most
+//        (|x/s| + |u|) * 2^-23 <= tol (a per-group bound, with a 4x margin);
+//   ua is monotone in x, so all eight lie between fma(min, 1/s, z) and fma(max, 1/s, z): if those are inside
+//        (-0.49, 15.49) no clamp can act;
+//   r = (ua + 1.5 * 2^23) - 1.5 * 2^23 is rint(ua), ties to even; if no ua is within tol of a rounding
+//        boundary k + 1/2, rint(u) = rint(ua) for all eight.
+// Whenever one of the conditions fails (a NaN anywhere fails them too: degenerate groups, overflowing zeros,
+// non-finite inputs) the thread takes quantize_exact.  The result is bit-identical to the defining arithmetic.
+__device__ __forceinline__ void quantize_chunk(const uint4 raw, uint32_t& word, __half& s_out, __half& z_out) {
   const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
   float x[8];
 #pragma unroll
@@ -39,55 +69,42 @@ __device__ __forceinline__ void quantize_chunk(const uint4 raw, bool active, uin
     x[2 * i] = f.x;
     x[2 * i + 1] = f.y;
   }
-  float mn = x[0], mx = x[0];
-#pragma unroll
-  for (int i = 1; i < 8; ++i) {
-    mn = fminf(mn, x[i]);
-    mx = fmaxf(mx, x[i]);
-  }
+  float mn = fminf(fminf(fminf(x[0], x[1]), fminf(x[2], x[3])), fminf(fminf(x[4], x[5]), fminf(x[6], x[7])));
+  float mx = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
 #pragma unroll
   for (int off = 1; off <= 2; off <<= 1) {
     mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
   }
-  (void)active;
-  const float range = __fsub_rn(mx, mn);
-  const float s32 = __fdiv_rn(range, 15.0f);
-  __half s16 = __float2half_rn(s32);
-  word = 0u;
-  if ((__half_as_ushort(s16) & 0x7FFFu) == 0) {  // scale rounds to zero: constant (or nearly constant) group
-    s_out = __ushort_as_half(0x3C00u);            // 1.0
-    z_out = __float2half_rn(__fsub_rn(0.0f, mn));
-    return;
-  }
+  const __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(mx, mn), 15.0f));
   const float sf = __half2float(s16);
-  float z32 = __fdiv_rn(__fsub_rn(0.0f, mn), sf);
-  z32 = fminf(fmaxf(z32, -65504.0f), 65504.0f);
-  const __half z16 = __float2half_rn(z32);
+  const __half z16 = __float2half_rn(__fdiv_rn(__fsub_rn(0.0f, mn), sf));  // no clamp here: an overflow fails the checks
   const float zf = __half2float(z16);
-  // Codes.  The defining arithmetic is u = fl(fl(x / s) + z) with a true division, q = clamp(rint(u), 0, 15)
-  // = rint(clamp(u, 0, 15)) (rint is monotone).  A true division, a round and a float-to-int conversion per
-  // element make this kernel bound by the special-function pipe, so the common case avoids all three:
-  //   ua = fl(x * (1/s) + z) with the correctly rounded reciprocal differs from u by at most
-  //        (|x/s| + |u|) * 2^-23 <= tol (a per-group bound, with a 4x margin);
-  //   y = clamp(ua) + 1.5 * 2^23 rounds to nearest-even in the addition and leaves the code in the low
-  //        mantissa bits.
-  // Only when clamp(ua) lies within tol of a rounding boundary k + 1/2 could the two disagree, and exactly
-  // those elements are redone with the division.  The result is bit-identical to the defining arithmetic.
   const float rs = __frcp_rn(sf);
   const float tol = (2.0f * fmaxf(fabsf(mn), fabsf(mx)) * rs + fabsf(zf) + 17.0f) * 4.76837158203125e-7f;  // 2^-21
   constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
-  uint32_t unsure = 0;  // elements whose fast result sits within tol of a rounding boundary
+  float r[8];          // the codes as floats
+  float far = 0.0f;    // largest |ua - rint(ua)| over the 8 elements (at most 1/2)
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const float u = fminf(fmaxf(fmaf(x[i], rs, zf), 0.0f), 15.0f);  // fmaxf also turns NaN into 0
-    const float y = u + kMagic;
-    if (fabsf(fabsf(u - (y - kMagic)) - 0.5f) <= tol) unsure |= 1u << i;
-    word |= (__float_as_uint(y) & 0xFu) << (4 * i);
+    const float u = fmaf(x[i], rs, zf);
+    r[i] = (u + kMagic) - kMagic;
+    far = fmaxf(far, fabsf(u - r[i]));
   }
-  if (unsure) word = exact_codes(x, sf, zf, word, unsure);  // rare
+  // four codes are a 16-bit integer that fp32 holds exactly: Horner with fused multiply-adds, then the
+  // integer is read off the low mantissa bits of (value + 2^23)
+  const float lo = fmaf(fmaf(fmaf(r[3], 16.0f, r[2]), 16.0f, r[1]), 16.0f, r[0]);
+  const float hi = fmaf(fmaf(fmaf(r[7], 16.0f, r[6]), 16.0f, r[5]), 16.0f, r[4]);
+  word = __byte_perm(__float_as_uint(lo + 8388608.0f), __float_as_uint(hi + 8388608.0f), 0x5410);
   s_out = s16;
   z_out = z16;
+  const bool proven = fmaf(mn, rs, zf) > -0.49f && fmaf(mx, rs, zf) < 15.49f && 0.5f - far > tol;
+  if (!proven) {  // rare
+    const QuantOut e = quantize_exact(x, mn, mx);
+    word = e.word;
+    s_out = e.s;
+    z_out = e.z;
+  }
 }
 
 // chunk index -> (b, h, t, c) of a [B][H_kv][T][d] tensor and the destination row in the cache
@@ -105,7 +122,7 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
   }
   uint32_t word;
   __half s, z;
-  quantize_chunk(raw, in_range, word, s, z);
+  quantize_chunk(raw, word, s, z);
   if (in_range) {
     const long long bh = row_in / T;
     const int t = static_cast<int>(row_in - bh * T);
@@ -121,59 +138,77 @@ __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half
   }
 }
 
-// Bulk variant: one thread block per destination cache block (16 tokens of one KV head, K or V), so the
-// codes leave as one contiguous kilobyte and the block's scales and zeros, gathered in shared memory,
-// as 16-byte vectors (written one by one they were four times as many memory transactions as the codes).
-// grid: (blocks touched per sequence, B * H_kv, {K, V}); 2 * d threads (one per 8 elements).
+// Bulk variant: a thread block of 2 * D threads (one per 8 elements) walks over kBulkBlocks consecutive
+// destination cache blocks (16 tokens of one KV head, K or V each), so the codes of a block leave as one
+// contiguous kilobyte and its scales and zeros, gathered in shared memory, as 16-byte vectors (written one by
+// one they were four times as many memory transactions as the codes).  The head dimension is a template
+// parameter: every offset inside a block is a compile-time constant per thread.
+// grid: (ceil(blocks touched per sequence / kBulkBlocks), B * H_kv, {K, V}).
 // seq_lens is read only here and bumped by bump_lens_kernel afterwards, so that no block can observe a
 // length that another block of the same launch has already advanced.
-// THREADS = the largest block this instantiation is launched with (1024 only for d = 512, so that the
-// common head dimensions keep the register budget of a 512-thread block).
-template <int THREADS>
-__global__ void __launch_bounds__(THREADS) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
-                                                                int T, int32_t* status) {
-  __shared__ __align__(16) __half sm_meta[2][16][16];  // [scale | zero][group][token], up to d = 512
+#ifndef TQ_BULK_BLOCKS
+#define TQ_BULK_BLOCKS 8
+#endif
+constexpr int kBulkBlocks = TQ_BULK_BLOCKS;
+
+template <int D>
+__global__ void __launch_bounds__(2 * D) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
+                                                              int T, int32_t* status) {
+  constexpr int CPR = D / 8, NG = D / 32;
+  __shared__ __align__(16) __half sm_meta[2][2][NG][16];  // [buffer][scale | zero][group][token]
   pdl_wait();
   pdl_launch_dependents();
-  const int d = c.d, cpr = d >> 3, ng = d >> 5;
   const long long bh = blockIdx.y;
   const int b = static_cast<int>(bh / c.H_kv);
   const int len = c.seq_lens[b];
   if (len < 0 || len + T > c.S_cap) return;  // flagged by bump_lens_kernel
   const int which = blockIdx.z;
-  const int j = (len >> 4) + blockIdx.x;                       // destination block
-  const int tok_lo = max(16 * j, len), tok_hi = min(16 * j + 16, len + T);
-  if (tok_lo >= tok_hi) return;
-  const int t = threadIdx.x / cpr, cc = threadIdx.x - t * cpr;  // token in the block, 8-element chunk in the row
-  const int tok = 16 * j + t;
-  const bool active = tok >= tok_lo && tok < tok_hi;
-  uint4 raw = make_uint4(0, 0, 0, 0);
-  if (active) raw = *reinterpret_cast<const uint4*>((which ? v_new : k_new) + (bh * T + (tok - len)) * d + cc * 8);
-  uint32_t word;
-  __half s, z;
-  quantize_chunk(raw, active, word, s, z);
-  bool page_ok;
-  uint8_t* blk = cache_block_bh(c, bh, b, 16 * j, threadIdx.x == 0 ? status : nullptr, page_ok);
-  if (!page_ok) return;  // a page outside the pool: nothing is written (uniform over the block)
-  if (active) *reinterpret_cast<uint32_t*>(blk + code_offset(d, which, t, cc * 4)) = word;
-  const bool whole = tok_lo == 16 * j && tok_hi == 16 * j + 16;
-  if ((cc & 3) == 0) {
-    if (whole) {
-      sm_meta[0][cc >> 2][t] = s;
-      sm_meta[1][cc >> 2][t] = z;
-    } else if (active) {  // a block only partly covered by this append: write the few values directly
-      *reinterpret_cast<__half*>(blk + meta_offset(d, which, 0, cc >> 2, t)) = s;
-      *reinterpret_cast<__half*>(blk + meta_offset(d, which, 1, cc >> 2, t)) = z;
+  const int t = threadIdx.x / CPR, cc = threadIdx.x % CPR;  // token in the block, 8-element chunk in the row
+  const int code_off = code_offset(D, which, t, cc * 4);
+  const __half* const src = which ? v_new : k_new;
+  const long long row_base = bh * T - len;  // row of token `tok` in the input is row_base + tok
+  const int j0 = (len >> 4) + blockIdx.x * kBulkBlocks;
+  auto fetch = [&](int j) {
+    const int tok = 16 * j + t;
+    return (tok >= len && tok < len + T) ? *reinterpret_cast<const uint4*>(src + (row_base + tok) * D + cc * 8)
+                                         : make_uint4(0, 0, 0, 0);
+  };
+  uint4 raw = fetch(j0);
+#pragma unroll 1
+  for (int jj = 0; jj < kBulkBlocks; ++jj) {
+    const int j = j0 + jj;                                    // destination block
+    const int tok_lo = max(16 * j, len), tok_hi = min(16 * j + 16, len + T);
+    if (tok_lo >= tok_hi) return;                             // past the end (uniform over the block)
+    const uint4 cur = raw;
+    if (jj + 1 < kBulkBlocks) raw = fetch(j + 1);             // next block's elements are in flight during the arithmetic
+    const int tok = 16 * j + t;
+    const bool active = tok >= tok_lo && tok < tok_hi;
+    uint32_t word;
+    __half s, z;
+    quantize_chunk(cur, word, s, z);
+    bool page_ok;
+    uint8_t* blk = cache_block_bh(c, bh, b, 16 * j, threadIdx.x == 0 ? status : nullptr, page_ok);
+    if (!page_ok) continue;  // a page outside the pool: nothing is written (uniform over the block)
+    if (active) *reinterpret_cast<uint32_t*>(blk + code_off) = word;
+    const bool whole = tok_lo == 16 * j && tok_hi == 16 * j + 16;
+    if ((cc & 3) == 0) {
+      if (whole) {
+        sm_meta[jj & 1][0][cc >> 2][t] = s;
+        sm_meta[jj & 1][1][cc >> 2][t] = z;
+      } else if (active) {  // a block only partly covered by this append: write the few values directly
+        *reinterpret_cast<__half*>(blk + meta_offset(D, which, 0, cc >> 2, t)) = s;
+        *reinterpret_cast<__half*>(blk + meta_offset(D, which, 1, cc >> 2, t)) = z;
+      }
     }
-  }
-  if (!whole) return;  // uniform over the block
-  __syncthreads();
-  // scales [ng][16] then zeros [ng][16] are adjacent in the cache block: 2 * ng * 32 bytes
-  const int vecs = ng * 2;  // 16-byte vectors per array
-  if (threadIdx.x < 2 * vecs) {
-    const int arr = threadIdx.x / vecs, v = threadIdx.x - arr * vecs;
-    const uint4 val = reinterpret_cast<const uint4*>(&sm_meta[arr][0][0])[v];
-    reinterpret_cast<uint4*>(blk + meta_offset(d, which, arr, 0, 0))[v] = val;
+    if (!whole) continue;  // uniform over the block
+    __syncthreads();       // one barrier per block: the two buffers alternate
+    // scales [NG][16] then zeros [NG][16] are adjacent in the cache block: 2 * NG * 32 bytes
+    constexpr int kVecs = NG * 2;  // 16-byte vectors per array
+    if (threadIdx.x < 2 * kVecs) {
+      const int arr = threadIdx.x / kVecs, v = threadIdx.x % kVecs;
+      const uint4 val = reinterpret_cast<const uint4*>(&sm_meta[jj & 1][arr][0][0])[v];
+      reinterpret_cast<uint4*>(blk + meta_offset(D, which, arr, 0, 0))[v] = val;
+    }
   }
 }
 
@@ -223,10 +258,15 @@ cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, co
   if (2 * per_seq <= 8192) {
     return launch_kernel(quantize_step_kernel, dim3(c.B), dim3(256), 0, st, c, k_new, v_new, T, status);
   } else {
-    dim3 grid(static_cast<unsigned>((T + 15) / 16 + 1), static_cast<unsigned>(c.B * c.H_kv), 2);
-    const cudaError_t e =
-        c.d > 256 ? launch_kernel(quantize_bulk_kernel<1024>, grid, dim3(2 * c.d), 0, st, c, k_new, v_new, T, status)
-                  : launch_kernel(quantize_bulk_kernel<512>, grid, dim3(2 * c.d), 0, st, c, k_new, v_new, T, status);
+    const int touched = (T + 15) / 16 + 1;  // destination blocks a sequence's new tokens can reach
+    dim3 grid(static_cast<unsigned>((touched + kBulkBlocks - 1) / kBulkBlocks), static_cast<unsigned>(c.B * c.H_kv), 2);
+    cudaError_t e;
+    switch (c.d) {
+      case 64: e = launch_kernel(quantize_bulk_kernel<64>, grid, dim3(128), 0, st, c, k_new, v_new, T, status); break;
+      case 128: e = launch_kernel(quantize_bulk_kernel<128>, grid, dim3(256), 0, st, c, k_new, v_new, T, status); break;
+      case 256: e = launch_kernel(quantize_bulk_kernel<256>, grid, dim3(512), 0, st, c, k_new, v_new, T, status); break;
+      default: e = launch_kernel(quantize_bulk_kernel<512>, grid, dim3(1024), 0, st, c, k_new, v_new, T, status); break;
+    }
     if (e != cudaSuccess) return e;
     return launch_kernel(bump_lens_kernel, dim3((c.B + 127) / 128), dim3(128), 0, st, c, T, status);
   }
