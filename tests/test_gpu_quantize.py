@@ -47,6 +47,11 @@ def test_adversarial_groups_bit_exact(gpu, oracle):
     rows.append(big)                                                                  # full fp16 range
     sub = (rng.integers(0, 1024, (16, 128)).astype(np.uint16)).view(np.float16)       # subnormal inputs
     rows.append(sub)
+    # a few thousand groups over many magnitudes and offsets (offset / spread up to ~1e4: the zero-point leaves
+    # the range in which the kernel's shortcut is provably exact and the step-by-step arithmetic takes over)
+    spread = 10.0 ** rng.uniform(-4, 3, (2048, 1))
+    offset = spread * rng.choice([0.0, 1.0, -1.0, 30.0, -30.0, 600.0, -600.0, 1e4], (2048, 1))
+    rows.append(np.clip(rng.standard_normal((2048, 128)) * spread + offset, -65504, 65504).astype(np.float16))
     x = np.concatenate(rows, 0)
     n = x.shape[0]
     shape = I.Shape("adv", 1, 1, 1, 128, 1.0)
