@@ -155,7 +155,7 @@ template <int D>
 __global__ void __launch_bounds__(2 * D) quantize_bulk_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
                                                               int T, int32_t* status) {
   constexpr int CPR = D / 8, NG = D / 32;
-  __shared__ __align__(16) __half sm_meta[2][2][NG][16];  // [buffer][scale | zero][group][token]
+  __shared__ __align__(16) __half sm_meta[kBulkBlocks][2][NG][16];  // [block][scale | zero][group][token]
   pdl_wait();
   pdl_launch_dependents();
   const long long bh = blockIdx.y;
@@ -173,6 +173,35 @@ __global__ void __launch_bounds__(2 * D) quantize_bulk_kernel(tq_kv_cache c, con
     return (tok >= len && tok < len + T) ? *reinterpret_cast<const uint4*>(src + (row_base + tok) * D + cc * 8)
                                          : make_uint4(0, 0, 0, 0);
   };
+  // Interior of the append (every block of this thread block lies entirely inside the new tokens, contiguous
+  // cache): no per-thread conditions, and the scales and zeros of all its blocks leave after ONE barrier.
+  if (16 * j0 >= len && 16 * (j0 + kBulkBlocks) <= len + T && c.page_table == nullptr) {
+    const __half* in = src + (row_base + 16 * j0 + t) * D + cc * 8;
+    uint8_t* const blk0 = c.blocks + (bh * (c.S_cap >> 4) + j0) * block_bytes(D);
+    uint4 nxt = *reinterpret_cast<const uint4*>(in);
+#pragma unroll 2
+    for (int jj = 0; jj < kBulkBlocks; ++jj) {
+      const uint4 cur = nxt;
+      in += 16 * D;
+      if (jj + 1 < kBulkBlocks) nxt = *reinterpret_cast<const uint4*>(in);
+      uint32_t word;
+      __half s, z;
+      quantize_chunk(cur, word, s, z);
+      *reinterpret_cast<uint32_t*>(blk0 + jj * block_bytes(D) + code_off) = word;
+      if ((cc & 3) == 0) {
+        sm_meta[jj][0][cc >> 2][t] = s;
+        sm_meta[jj][1][cc >> 2][t] = z;
+      }
+    }
+    __syncthreads();
+    constexpr int kVecsPerBlock = 2 * NG * 2;  // 16-byte vectors of one block's scales + zeros (adjacent in the cache)
+    for (int i = threadIdx.x; i < kBulkBlocks * kVecsPerBlock; i += 2 * D) {
+      const int jj = i / kVecsPerBlock, v = i % kVecsPerBlock;
+      const uint4 val = reinterpret_cast<const uint4*>(&sm_meta[jj][0][0][0])[v];
+      reinterpret_cast<uint4*>(blk0 + jj * block_bytes(D) + meta_offset(D, which, 0, 0, 0))[v] = val;
+    }
+    return;
+  }
   uint4 raw = fetch(j0);
 #pragma unroll 1
   for (int jj = 0; jj < kBulkBlocks; ++jj) {
@@ -193,20 +222,20 @@ __global__ void __launch_bounds__(2 * D) quantize_bulk_kernel(tq_kv_cache c, con
     const bool whole = tok_lo == 16 * j && tok_hi == 16 * j + 16;
     if ((cc & 3) == 0) {
       if (whole) {
-        sm_meta[jj & 1][0][cc >> 2][t] = s;
-        sm_meta[jj & 1][1][cc >> 2][t] = z;
+        sm_meta[jj][0][cc >> 2][t] = s;
+        sm_meta[jj][1][cc >> 2][t] = z;
       } else if (active) {  // a block only partly covered by this append: write the few values directly
         *reinterpret_cast<__half*>(blk + meta_offset(D, which, 0, cc >> 2, t)) = s;
         *reinterpret_cast<__half*>(blk + meta_offset(D, which, 1, cc >> 2, t)) = z;
       }
     }
     if (!whole) continue;  // uniform over the block
-    __syncthreads();       // one barrier per block: the two buffers alternate
+    __syncthreads();       // one barrier per block: each block has its own buffer
     // scales [NG][16] then zeros [NG][16] are adjacent in the cache block: 2 * NG * 32 bytes
     constexpr int kVecs = NG * 2;  // 16-byte vectors per array
     if (threadIdx.x < 2 * kVecs) {
       const int arr = threadIdx.x / kVecs, v = threadIdx.x % kVecs;
-      const uint4 val = reinterpret_cast<const uint4*>(&sm_meta[jj & 1][arr][0][0])[v];
+      const uint4 val = reinterpret_cast<const uint4*>(&sm_meta[jj][arr][0][0])[v];
       reinterpret_cast<uint4*>(blk + meta_offset(D, which, arr, 0, 0))[v] = val;
     }
   }
