@@ -87,3 +87,29 @@ def test_argument_validation_without_gpu(lib):
     assert need >= 2 * 2 * 64 * 128 * 4
     assert tq._lib.tq_sdpa_dequant_then_attend(C.byref(cs), fake, 8, 1.0, fake, need - 1, 1, fake, 1, None,
                                                None) == tq.TQ_ERR_WORKSPACE
+    # the secondary entry points validate the same way
+    assert tq._lib.tq_sdpa_int4_decode_window(C.byref(cs), fake, 8, 1.0, -1, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_int4_decode_multi(C.byref(cs), fake, 8, 0, 1.0, 0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_int4_decode_multi(C.byref(cs), fake, 8, 65, 1.0, 0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_mixed_precision_attend(C.byref(cs), fake + 2, None, fake, 8, 1.0, 1, fake, fake, fake, None,
+                                                  None) == tq.TQ_ERR_ALIGN
+    assert tq._lib.tq_sdpa_int4_attend_static(None, fake, 8, 1.0, fake, 1, None, None) == tq.TQ_ERR_NULL
+    # paged caches: page size a power of two >= 16, capacity = pages * page size, table aligned
+    ok_paged = dict(blocks=fake, seq_lens=fake, B=1, H_kv=2, S_cap=128, d=128, page_table=fake, page_tokens=32,
+                    max_pages=4, num_pages=9)
+    for bad in (dict(page_tokens=48), dict(page_tokens=8), dict(max_pages=3), dict(num_pages=0), dict(S_cap=96)):
+        cs = tq.tq_kv_cache(**{**ok_paged, **bad})
+        assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 8, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE, bad
+    cs = tq.tq_kv_cache(**{**ok_paged, "page_table": fake + 2})
+    assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 1, None, None) == tq.TQ_ERR_ALIGN
+    # split ranges under a window tile exactly the window
+    for length, window, Cn in ((3000, 1024, 5), (1029, 1024, 3), (7, 1024, 2), (100, 1, 4), (0, 5, 2)):
+        prev = max(0, length - window)
+        for c in range(Cn):
+            t0, t1 = tq.tq_split_range_window(length, window, Cn, c)
+            assert t0 == prev and t1 >= t0
+            prev = t1
+        assert prev == length
+    # split policy: one wave for few heads, several for a batch, never shorter than the stated minimum
+    assert tq.tq_auto_splits(16, 8, 64, 128, 65536) >= 4
+    assert tq.tq_auto_splits(16, 8, 64, 128, 2048) == 1
