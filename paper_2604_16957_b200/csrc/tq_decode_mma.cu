@@ -82,7 +82,7 @@ struct Cfg {
   static constexpr int XCH_TEAM = DS > 1 ? 2 * DS * 32 * 16 + 2 * DS * 4 : 0;
   static constexpr int SMEM = XCH + NTEAM * XCH_TEAM;
   static_assert(STAGE == TQ_BLOCK_BYTES(D), "a stage is one cache block");
-  static_assert(kWarps % DS == 0 && XCH % 16 == 0, "teams tile the block");
+  static_assert(kWarps % DS == 0 && XCH % 16 == 0 && SMEM % 8 == 0, "teams tile the block");
   __host__ __device__ static constexpr int swz(int tok) { return (tok >> SWZ_SHIFT) & (NG - 1); }
 };
 
@@ -333,7 +333,7 @@ __device__ __forceinline__ bool wait_stage(uint32_t bar, uint32_t parity) {
 // is the (S_q - 1 - s)-th newest cached token and attends causally: tokens [lo_s, hi_s) with
 // hi_s = len - (S_q - 1 - s), lo_s = max(0, hi_s - window).  The plain instantiation carries none of this
 // arithmetic into the block loop.  MODE: 0 plain, 1 general, 2 general over a paged cache (tq.h): the block
-// addresses then come from the page table, each entry fetched one block ahead of its use.
+// addresses then come from the page table through a per-thread-block table of page addresses.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, int S_q, float attn_scale, int window,
@@ -384,32 +384,37 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     for (int s = 0; s < Cf::NST; ++s) mbar_init(bars + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  if (DS > 1) __syncthreads();  // the team's other warps wait on these barriers too
-  else __syncwarp();
   // The team's n-th block is block blk0 + team + n * NTEAM of this (sequence, KV head); one lane of the team
-  // copies it into ring slot n mod NST.  Contiguous cache: it starts at head_blocks + block * STAGE.  Paged:
-  // page `pg` (the table entry, fetched ahead) holds [H_kv][page_tokens / 16] blocks.
+  // copies it into ring slot n mod NST.  Contiguous cache: it starts at head_blocks + block * STAGE.
+  // Paged: page_tokens is a power of two, so block j sits in table entry j >> pshift at offset j & (bpp - 1);
+  // the thread block first turns the table entries of its split into addresses of this KV head's part of each
+  // page (checked against the pool once), kept in shared memory behind everything else, so that issuing a copy
+  // costs a shift, a shared-memory load and a multiply-add.
   const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
-  // page_tokens is a power of two, so block j sits in table entry j >> pshift at offset j & (bpp - 1).
   const int pshift = PAGED ? 31 - __clz(cache.page_tokens >> 4) : 0;
-  auto table_entry = [&](int n) -> int {
-    return cache.page_table[static_cast<long long>(b) * cache.max_pages + ((blk0 + team + n * NTEAM) >> pshift)];
-  };
-  auto issue = [&](int n, int pg) {
+  const int page0 = blk0 >> pshift;
+  const uint8_t** const page_ptr = reinterpret_cast<const uint8_t**>(smem + Cf::SMEM);
+  if (PAGED) {
+    const int npages = blk1 > blk0 ? ((blk1 - 1) >> pshift) - page0 + 1 : 0;
+    for (int i = threadIdx.x; i < npages; i += kThreads) {
+      int pg = cache.page_table[static_cast<long long>(b) * cache.max_pages + page0 + i];
+      if (static_cast<uint32_t>(pg) >= static_cast<uint32_t>(cache.num_pages)) {
+        if (status) atomicOr(status, TQ_STATUS_BAD_PAGE);
+        pg = 0;
+      }
+      // block index in the pool (fits 32 bits: the pool is checked to hold fewer than 2^31 blocks)
+      const uint32_t idx = (static_cast<uint32_t>(pg) * cache.H_kv + kvh) << pshift;
+      page_ptr[i] = cache.blocks + static_cast<size_t>(idx) * Cf::STAGE;
+    }
+  }
+  if (DS > 1 || PAGED) __syncthreads();  // a team's warps wait on the same barriers; everybody reads the page addresses
+  else __syncwarp();
+  auto issue = [&](int n) {
     if (sub == 0 && lane == 0) {
       const int slot = n & (Cf::NST - 1), blk = blk0 + team + n * NTEAM;
       const uint8_t* src;
-      if (PAGED) {
-        if (static_cast<uint32_t>(pg) >= static_cast<uint32_t>(cache.num_pages)) {
-          if (status) atomicOr(status, TQ_STATUS_BAD_PAGE);
-          pg = 0;
-        }
-        // block index in the pool (fits 32 bits: the pool is checked to hold fewer than 2^31 blocks)
-        const uint32_t idx = ((static_cast<uint32_t>(pg) * cache.H_kv + kvh) << pshift) + (blk & ((1 << pshift) - 1));
-        src = cache.blocks + static_cast<size_t>(idx) * Cf::STAGE;
-      } else {
-        src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
-      }
+      if (PAGED) src = page_ptr[(blk >> pshift) - page0] + static_cast<size_t>(blk & ((1 << pshift) - 1)) * Cf::STAGE;
+      else src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
       const uint32_t bar = bars + 8 * slot;
       mbar_expect_tx(bar, Cf::STAGE);
       bulk_g2s(ring_s + slot * Cf::STAGE, src, Cf::STAGE, bar);
@@ -417,23 +422,12 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   };
 
   // start streaming: the first stages are in flight while q is turned into fragments
-  int pg_next = 0;  // paged: table entry of the next block to be issued
-  {
-    int pre = 0;  // the first NST entries, fetched side by side
-    if (PAGED && lane < Cf::NST && lane < nblk) pre = table_entry(lane);
 #pragma unroll
-    for (int s = 0; s < Cf::NST - 1; ++s) {
-      const int pg = PAGED ? __shfl_sync(0xffffffffu, pre, s) : 0;
-      if (s < nblk) issue(s, pg);
-    }
-    if (PAGED) pg_next = __shfl_sync(0xffffffffu, pre, Cf::NST - 1);
-  }
-  // issue the team's n-th block (if it has one) and fetch the table entry of the one after it
+  for (int s = 0; s < Cf::NST - 1; ++s)
+    if (s < nblk) issue(s);
+  // issue the team's n-th block, if it has one
   auto refill = [&](int n) {
-    if (n < nblk) {
-      issue(n, pg_next);
-      if (PAGED && n + 1 < nblk) pg_next = table_entry(n + 1);
-    }
+    if (n < nblk) issue(n);
   };
 
   // ---- q as MMA B fragments: column n = gid is column v0 + gid of the tile; k slots follow the nibble order.
@@ -652,13 +646,21 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 template <int D, int MODE>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
                    float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                Cfg<D>::SMEM);
+  size_t smem = Cfg<D>::SMEM;
+  if (MODE == 2) {
+    // room for the page addresses of the longest split: its blocks, rounded out to whole pages
+    const long long span = (window > 0 && window < c.S_cap) ? static_cast<long long>(window) + S_q + 15 : c.S_cap;
+    const long long blocks = (span + 15) / 16 + 1, per_split = (blocks + C - 1) / C + 1;
+    smem += 8 * static_cast<size_t>(per_split / (c.page_tokens / 16) + 2);
+    if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;  // tiny pages and too few splits for this capacity
+  }
+  const cudaError_t attr =
+      cudaFuncSetAttribute(decode_mma_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (attr != cudaSuccess) return attr;
   const int GV = (H_q / c.H_kv) * S_q;
   dim3 grid(C, c.H_kv * ((GV + 7) / 8), c.B);
-  return launch_kernel(decode_mma_kernel<D, MODE>, grid, dim3(kThreads), Cfg<D>::SMEM, st, c, q, H_q, S_q, attn_scale,
-                       window, C, o_part, m_part, l_part, status);
+  return launch_kernel(decode_mma_kernel<D, MODE>, grid, dim3(kThreads), smem, st, c, q, H_q, S_q, attn_scale, window, C,
+                       o_part, m_part, l_part, status);
 }
 
 template <int D>
