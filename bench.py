@@ -137,11 +137,13 @@ def run_reference(args, rank):
     if rank != 0:
         return
     # one cache build, then warmup + steps timed repetitions on it
-    per, secs, threads = oracle_sample_us_per_layer(args.context, repeats=args.warmup + args.steps)
+    # (a step is one full layer, all 64 query heads, so the oracle's thread pool is used as in the GPU arm's
+    # cpu_baseline; 80 layers per step would take minutes per step)
+    per, secs, threads = oracle_sample_us_per_layer(args.context, repeats=args.warmup + args.steps, kv_heads=H_KV)
     timed = per[args.warmup:]
     value = sum(timed) / len(timed)
-    sample = (f"1 of {H_KV} KV heads ({H_Q // H_KV} of {H_Q} query heads) of one {args.context}-token layer per step, "
-              f"fp64 oracle, time scaled x{H_KV} to a full layer")
+    sample = (f"one full {args.context}-token layer (all {H_Q} query heads, {H_KV} KV heads) per step instead of "
+              f"{args.layers}, fp64 oracle on the oracle-quantised cache")
     line = {"impl": "reference", "metric": "int4 decode-attn us/layer @128K (Llama-70B shape)", "value": value,
             "unit": "us/layer", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": value * args.layers / 1e3, "higher_is_better": False, "scaling": "weak",
