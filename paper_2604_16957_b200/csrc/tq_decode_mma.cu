@@ -1,18 +1,17 @@
 // Fused int4 decode attention, phase 1 (Sec. 3.1 Algorithm 1 per split, Sec. 3.2), for sm_100a.
 //
-// One thread block handles one (sequence, KV head, tile of up to 8 query heads, split); with several query
-// tokens per sequence the tile holds (query token, head) pairs.  The
-// query heads that share the KV head are packed into the N = 8 dimension of
-// mma.sync.m16n8k16, so every byte of the cache is read from HBM once per head tile.
-// The path is HBM-bound.  The cache is stored in 16-token blocks that are already in the shared-
-// memory layout this kernel wants (tq.h), so a stage is filled by ONE bulk asynchronous copy
-// (cp.async.bulk, the TMA unit) of a contiguous 2560-byte block (d = 128) issued by one lane and
-// completing on the stage's mbarrier.  Each warp owns a ring of 4 stages and its tokens end to
-// end, so the main loop has no block-wide barrier.  (Head dimensions 256 and 512 are split over teams
-// of 2 and 4 warps that share a ring and exchange their partial scores once per token block.)  Measured on the 128K Llama-shaped layer, the
-// copies alone take 27.9 us with bulk copies against 30.2 us with 16-byte cp.async.  The tensor
-// cores only take the G-packed q.K^T and P.V contractions off the CUDA cores, which could not
-// keep up with the memory system otherwise.
+// One thread block handles one (sequence, KV head, tile of up to 8 query heads, split); with several
+// query tokens per sequence the tile holds (query token, head) pairs.  The query heads that share the
+// KV head are packed into the N = 8 dimension of mma.sync.m16n8k16, so every byte of the cache is read
+// from HBM once per head tile.  The path is HBM-bound.  The cache is stored in 16-token blocks that are
+// already in the shared-memory layout this kernel wants (tq.h), so a stage is filled by ONE bulk
+// asynchronous copy (cp.async.bulk, the TMA unit) of a contiguous 2560-byte block (d = 128) issued by
+// one lane and completing on the stage's mbarrier.  Each warp owns a ring of 4 stages and its tokens
+// end to end, so the main loop has no block-wide barrier.  (Head dimensions 256 and 512 are split over
+// teams of 2 and 4 warps that share a ring and exchange their partial scores once per token block.)
+// Measured on the 128K Llama-shaped layer, the copies alone take 27.9 us with bulk copies against
+// 30.2 us with 16-byte cp.async.  The tensor cores only take the G-packed q.K^T and P.V contractions
+// off the CUDA cores, which could not keep up with the memory system otherwise.
 //
 // Dequantisation in registers (the paper's dequant4, and its Eq. 4 idea of folding the nibble
 // position into the other operand):
@@ -35,8 +34,8 @@
 //   K codes [16][D/2] | V codes [16][D/2] | K scale [D/32][16] | K zero | V scale | V zero
 // The 16-byte chunks of the code rows are XOR-swizzled with the token index, which makes the
 // fragment loads conflict free (a padded layout was measured too: it costs 3-4x the shared-memory
-// wavefronts on the way in).  Fragments come from ldmatrix, whose 8x8 b16 "matrix" is here 8 tokens x one 16-byte
-// chunk (32 codes of one group):
+// wavefronts on the way in).  Fragments come from ldmatrix, whose 8x8 b16 "matrix" is here 8 tokens x
+// one 16-byte chunk (32 codes of one group):
 //   K: plain ldmatrix  -> lane (gid, tid4) holds word tid4 of token gid: 8 codes of one token,
 //      the A operand rows of the score MMA;
 //   V: ldmatrix.trans  -> lane (gid, tid4) holds 16-bit lane gid of tokens 2*tid4 and 2*tid4+1
