@@ -11,7 +11,7 @@
  *     memory; the library allocates nothing, keeps no state between calls and never
  *     synchronises.  Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
  *     default stream) and is ordered by it.
- *   - All device pointers must be 16-byte aligned.
+ *   - All device pointers must be 16-byte aligned (m_part, l_part, seq_lens, page_table and status: 4-byte).
  *   - Every entry point returns a tq_result.  Errors that the host can see (null pointer, bad
  *     shape, bad alignment, workspace too small) are returned before anything is launched.
  *   - Conditions only the device can see (a full cache, an empty sequence) OR bits into the
@@ -150,7 +150,9 @@ void tq_split_range(int32_t len, int32_t C, int32_t c, int32_t* t0 /* host */, i
  *   num_splits : C >= 1, or 0 for tq_auto_splits(B, H_kv, H_q, d, S_cap).
  * All seq_lens[b] cached tokens are attended (no mask).  Requirements: H_q a multiple of H_kv,
  * H_q / H_kv <= 64, C <= TQ_MAX_SPLITS.
- * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_CUDA.  Status: TQ_STATUS_EMPTY_SEQ, TQ_STATUS_BAD_LEN.
+ * Errors: TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_CUDA.  Status: TQ_STATUS_EMPTY_SEQ, TQ_STATUS_BAD_LEN,
+ * TQ_STATUS_TIMEOUT (a bulk copy did not complete within the bound: that call's partials are not valid), and
+ * TQ_STATUS_BAD_PAGE with a paged cache.
  */
 int tq_sdpa_int4_decode(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
                         int32_t num_splits, float* o_part, float* m_part, float* l_part, int32_t* status,
