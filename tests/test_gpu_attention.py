@@ -498,3 +498,58 @@ def test_paged_cache_bad_page_is_flagged_not_followed(gpu, oracle):
     assert int(status.item()) & 16
     changed = (dev.blocks != before).flatten(1).any(dim=1).cpu().numpy()
     assert changed.sum() == 1 and changed[int(dev.page_table[1, 3])]  # only sequence 1's page was written
+
+
+def test_decode_step_replays_as_a_cuda_graph(gpu, oracle):
+    """The whole step (append, decode, combine) is captured once and replayed: lengths live in device memory,
+    so every replay appends at the next position and attends one token more; each replay matches the oracle
+    and the eager calls bit for bit."""
+    tq, torch = gpu
+    sh = I.Shape("x", 2, 16, 2, 128, 128 ** -0.5, k_outlier_channels=4)
+    lens = [500, 90]
+    host, dev = _both(gpu, oracle, sh, 500, 97, S_cap=512, lens=lens)
+    eager = tq.KVCache(sh.B, sh.H_kv, 512, sh.d)
+    eager.blocks.copy_(dev.blocks)
+    eager.seq_lens.copy_(dev.seq_lens)
+    C = 3
+    o, m, l = tq.alloc_partials(sh.B, sh.H_q, sh.d, C)
+    out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    k_in = torch.empty((sh.B, sh.H_kv, 1, sh.d), dtype=torch.float16, device="cuda")
+    v_in = torch.empty_like(k_in)
+    q_in = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float16, device="cuda")
+
+    def step(cache):
+        tq.tq_kv_quantize_append(cache, k_in, v_in, status)
+        tq.tq_sdpa_int4_decode(cache, q_in, sh.alpha, C, o, m, l, status)
+        tq.tq_sdpa_int4_combine(o, m, l, out)
+
+    k1, v1 = I.make_kv(sh, 1, 97, stream=1)
+    k_in.copy_(torch.from_numpy(k1)); v_in.copy_(torch.from_numpy(v1)); q_in.copy_(torch.from_numpy(I.make_q(sh, 97)))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(eager)                       # warm-up outside the capture (sets function attributes), on the eager copy
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    host.append(k1, v1)
+    eager_out = [out.clone()]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step(dev)
+    for i in range(3):
+        kn, vn = I.make_kv(sh, 1, 97, stream=1 + i)
+        qn = I.make_q(sh, 97, stream=i)
+        k_in.copy_(torch.from_numpy(kn)); v_in.copy_(torch.from_numpy(vn)); q_in.copy_(torch.from_numpy(qn))
+        if i > 0:
+            host.append(kn, vn)
+            step(eager)
+            torch.cuda.synchronize()
+            eager_out.append(out.clone())
+        g.replay()
+        torch.cuda.synchronize()
+        assert dev.seq_lens.tolist() == [lens[0] + i + 1, lens[1] + i + 1]
+        assert_attention_close(out.cpu().numpy(), oracle.attention(host, qn, sh.alpha), f"graph replay {i}")
+        assert torch.equal(out, eager_out[i])
+    assert int(status.item()) == 0
+    assert_cache_bits_equal(dev, host)
