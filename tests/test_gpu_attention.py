@@ -553,3 +553,38 @@ def test_decode_step_replays_as_a_cuda_graph(gpu, oracle):
         assert torch.equal(out, eager_out[i])
     assert int(status.item()) == 0
     assert_cache_bits_equal(dev, host)
+
+
+def test_offsets_beyond_4_gib(gpu, oracle):
+    """A 4M-token cache (5.4 GB) whose only tokens sit at its very end: bulk append, single-token append and
+    windowed decode address blocks more than 2^32 bytes into the buffer."""
+    tq, torch = gpu
+    sh = I.Shape("x", 1, 64, 8, 128, 128 ** -0.5, k_outlier_channels=4)
+    S_cap = 1 << 22
+    start = S_cap - 208
+    dev = tq.KVCache(sh.B, sh.H_kv, S_cap, sh.d)
+    assert dev.blocks.numel() > (1 << 32)
+    dev.seq_lens.fill_(start)
+    k, v = I.make_kv(sh, 150, 103)
+    k1, v1 = I.make_kv(sh, 1, 103, stream=1)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tq.tq_kv_quantize_append(dev, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
+    tq.tq_kv_quantize_append(dev, torch.from_numpy(k1).cuda(), torch.from_numpy(v1).cuda(), status)
+    host = oracle.Cache(sh.B, sh.H_kv, 160, sh.d)
+    host.append(k, v)
+    host.append(k1, v1)
+    q = I.make_q(sh, 103)
+    for window, C in ((120, 1), (151, 3), (40, 0)):
+        o, m, l = tq.alloc_partials(sh.B, sh.H_q, sh.d, C or tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q, sh.d, window))
+        out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+        tq.tq_sdpa_int4_decode_window(dev, torch.from_numpy(q).cuda(), sh.alpha, window, C, o, m, l, status)
+        tq.tq_sdpa_int4_combine(o, m, l, out)
+        torch.cuda.synchronize()
+        assert_attention_close(out.cpu().numpy(), oracle.attention_window(host, q, sh.alpha, window), f"4GiB w={window}")
+    assert int(status.item()) == 0 and dev.seq_lens.tolist() == [start + 151]
+    # the rows written are the oracle's, bit for bit (read back through the offset helpers)
+    blocks = dev.blocks[0, :, (start >> 4):].cpu()
+    tail = tq.KVCache(1, sh.H_kv, blocks.shape[1] * 16, sh.d, device="cpu")
+    tail.blocks.copy_(blocks.unsqueeze(0))
+    for d_arr, h_arr in zip(tail.arrays_token_major(), host.arrays()):
+        assert np.array_equal(d_arr[0, :, :151].numpy().view(np.uint8), h_arr[0, :, :151].view(np.uint8))
