@@ -45,7 +45,7 @@ def test_config1_tiny_then_append_one_token(gpu, oracle):
     tq.tq_kv_quantize_append(dev, torch.from_numpy(k1).cuda(), torch.from_numpy(v1).cuda())
     assert_cache_bits_equal(dev, host)
     q1 = I.make_q(sh, 1, stream=1)
-    for C in (0, 1, 3, 17):
+    for C in (0, 1, 3, 17, 256):  # up to the largest split count: nearly all splits are empty
         out, _, _ = fused_attention(tq, torch, dev, q1, sh.alpha, num_splits=C)
         assert_attention_close(out, oracle.attention(host, q1, sh.alpha), f"tiny/257 C={C}")
 
@@ -588,3 +588,20 @@ def test_offsets_beyond_4_gib(gpu, oracle):
     tail.blocks.copy_(blocks.unsqueeze(0))
     for d_arr, h_arr in zip(tail.arrays_token_major(), host.arrays()):
         assert np.array_equal(d_arr[0, :, :151].numpy().view(np.uint8), h_arr[0, :, :151].view(np.uint8))
+
+
+def test_many_sequences_and_the_widest_gqa(gpu, oracle):
+    """B = 96 short sequences (grid z) and 64 query heads on one KV head (eight head tiles)."""
+    tq, torch = gpu
+    sh = I.Shape("x", 96, 2, 1, 64, 0.125)
+    lens = [1 + (7 * i) % 80 for i in range(96)]
+    host, dev = _both(gpu, oracle, sh, 80, 111, lens=lens, fill_byte=0xFF)
+    q = I.make_q(sh, 111)
+    out, _, _ = fused_attention(tq, torch, dev, q, sh.alpha)
+    assert_attention_close(out, oracle.attention(host, q, sh.alpha), "B=96")
+    sh = I.Shape("x", 1, 64, 1, 128, 128 ** -0.5)
+    host, dev = _both(gpu, oracle, sh, 1000, 112, fill_byte=0xFF)
+    q = I.make_q(sh, 112)
+    for C in (0, 2):
+        out, _, _ = fused_attention(tq, torch, dev, q, sh.alpha, num_splits=C)
+        assert_attention_close(out, oracle.attention(host, q, sh.alpha), f"G=64 C={C}")
