@@ -328,7 +328,7 @@ def main():
             "breakdown_us_per_layer": {"append+decode+combine": us_per_layer, "decode+combine": t_attn / K / L * 1e6,
                                        "decode": decode_us, "append": t_append / K / L * 1e6},
             "hbm_gbs_whole_step": alg_bytes / (us_per_layer * 1e-6) / 1e9, "num_splits": C,
-            "paper_context": PAPER_CONTEXT}
+            "paper_context": PAPER_CONTEXT, "device": device_info(torch, dev)}
     if world > 1:
         line["config"]["replicas"] = "independent replicas, no collective (the path does not shard in this build)"
 
@@ -343,6 +343,14 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def device_info(torch, dev):
+    """What the budgets assume about the GPU, as the driver reports it."""
+    p = torch.cuda.get_device_properties(dev)
+    return {"name": p.name, "sms": p.multi_processor_count, "l2_bytes": getattr(p, "L2_cache_size", None),
+            "smem_per_sm_bytes": getattr(p, "shared_memory_per_multiprocessor", None),
+            "hbm_bytes": p.total_memory}
 
 
 def ncu_traffic_bytes():
