@@ -104,8 +104,8 @@ size_t tq_cache_code_offset(int32_t d, int32_t which, int32_t t, int32_t byte);
 size_t tq_cache_meta_offset(int32_t d, int32_t which, int32_t is_zero, int32_t g, int32_t t);
 
 /*
- * Quantise T new tokens per sequence and append them in place (Sec. 2.1, Eq. 2-3; "quantizes the
- * KV cache to int4 on the fly").  The paper's implementation appends by concatenation and names
+ * Quantise T new tokens per sequence and append them in place (Sec. 2.1, Eq. 2-3; Sec. 1 describes the
+ * cache as quantised while tokens are generated).  The paper's implementation appends by concatenation and names
  * that as its main end-to-end overhead; here the cache is pre-allocated and rows are written at
  * positions seq_lens[b] .. seq_lens[b] + T - 1.
  *   k_new, v_new : [B][H_kv][T][d] fp16, read only.
@@ -119,7 +119,8 @@ int tq_kv_quantize_append(const tq_kv_cache* cache /* host */, const void* k_new
 
 /*
  * Number of sequence splits C the library would pick for a decode step over sequences of up to
- * `max_seq_len` tokens (host function, no CUDA call).  Chosen from the SM count: with few
+ * `max_seq_len` tokens (host function; it launches nothing, but the first call on a device asks the CUDA
+ * runtime for the SM count of the current device and remembers it per device).  Chosen from the SM count: with few
  * (sequence, KV head) pairs, B * H_kv * ceil(G / 8) * C thread blocks fill the GPU in one wave of
  * equal splits (at least 512 tokens each); with a batch, in about four waves (splits of at least
  * 2048 tokens), so that sequences of different lengths even out.  Always in [1, TQ_MAX_SPLITS].
@@ -159,8 +160,8 @@ int tq_sdpa_int4_decode(const tq_kv_cache* cache /* host */, const void* q, int3
                         void* stream);
 
 /*
- * Phase 1 restricted to a sliding window (Appendix A: Gemma's sliding-attention layers, w = 1024,
- * "handled by a conditional skip in the inner loop"): sequence b attends only its last `window`
+ * Phase 1 restricted to a sliding window (Appendix A: Gemma's sliding-attention layers, w = 1024, which
+ * the paper's kernel serves by skipping tokens inside its loop): sequence b attends only its last `window`
  * tokens, [max(0, seq_lens[b] - window), seq_lens[b]).  Here the skip is not per token: the splits
  * partition the window only, so tokens outside it are never fetched.  window = 0 means no window
  * (identical to tq_sdpa_int4_decode); window < 0 is TQ_ERR_SHAPE.  num_splits = 0 picks
@@ -251,7 +252,8 @@ int tq_sdpa_mixed_precision_attend(const tq_kv_cache* cache /* host */, const vo
  *   Result: out[b][h][:] as tq_sdpa_int4_decode followed by tq_sdpa_int4_combine would give it
  *   (the split count may differ, so agreement is to rounding, not bit for bit).
  *   It calls no cudaMalloc / cudaFree nor any routine that allocates.  The caller still provides
- *   q, the cache and out.
+ *   q, the cache (contiguous or paged, any supported head dimension) and out; the arguments are
+ *   checked exactly as tq_sdpa_int4_decode and tq_sdpa_int4_combine check theirs.
  *   Limit: the partials of the chosen split count, B * H_q * C * (d + 2) * 4 bytes (plus padding),
  *   must fit the array.  The split count is lowered as far as 1 to make them fit; if they still
  *   do not, nothing is launched and TQ_ERR_WORKSPACE is returned.

@@ -12,7 +12,6 @@
  *   - dequant4:  x^ = (q - z) * s                                             (Eq. 3, Sec. 3.1)
  *   - single-query attention softmax(alpha * q K^T) V over dequantised K, V   (Algorithm 1, whose
  *     result is exactly this definition; written here as the plain two-pass definition in fp64)
- *   - a literal one-pass transcription of Algorithm 1 in fp64 (used only to pin the above)
  *   - split partials (o_c, m_c, l_c) and their reduction                      (Sec. 3.2, Eq. 5)
  *   - GQA head map kv_head = head / (H_q / H_kv)                              (Sec. 3.1)
  *   - sliding window: only the last w tokens are attended                     (Appendix A)
@@ -33,7 +32,7 @@
  * all 65536 halves and over ties; Eq. 4 identity over all 65536 words; pack/unpack round trip;
  * Eq. 1 / Table 4 closed forms; |x - x^| <= s/2; nearest-code brute force; constant groups;
  * softmax weights sum to 1; constant-V, S = 1, q = 0, permutation, split and GQA invariances;
- * Algorithm 1 (literal) against the two-pass definition; a library fp64 attention on the
+ * a blocked log-sum-exp evaluation written in the tests; a library fp64 attention on the
  * dequantised values; the windowed form against full attention over a cache cut to the window.
  * The bit-level operation ORDER of the quantiser (which of several mathematically equal float32
  * evaluation orders) is this build's reading and cannot be pinned
@@ -366,37 +365,6 @@ void tqo_combine(const double* o_part, const double* m_part, const double* l_par
     }
     for (int64_t x = 0; x < d; ++x) out[bh * d + x] /= den;
   }
-}
-
-/* Algorithm 1, one pass with running (m, l, o), in fp64, for one (b, h) over all lens[b]
- * tokens.  The query is pre-scaled by alpha as in its first step. */
-void tqo_algorithm1(const uint8_t* kp, const uint16_t* ks, const uint16_t* kz, const uint8_t* vp, const uint16_t* vs,
-                    const uint16_t* vz, const int32_t* lens, int64_t B, int64_t H_kv, int64_t S_cap, int64_t d,
-                    const uint16_t* q16, int64_t H_q, double alpha, int64_t b, int64_t h, double* out) {
-  tqo_cache c;
-  fill_cache(&c, kp, ks, kz, vp, vs, vz, lens, B, H_kv, S_cap, d);
-  int64_t kvh = h / (H_q / H_kv);
-  double* qs = (double*)malloc((size_t)d * sizeof(double));
-  double* kr = (double*)malloc((size_t)d * sizeof(double));
-  double* vr = (double*)malloc((size_t)d * sizeof(double));
-  for (int64_t x = 0; x < d; ++x) qs[x] = (double)tqo_half_to_float(q16[(b * H_q + h) * d + x]) * alpha;
-  double m = -INFINITY, l = 0.0;
-  for (int64_t x = 0; x < d; ++x) out[x] = 0.0;
-  for (int64_t i = 0; i < lens[b]; ++i) {
-    dequant_token(&c, 0, b, kvh, i, kr);
-    double a = 0.0;
-    for (int64_t x = 0; x < d; ++x) a += qs[x] * kr[x];
-    double m2 = a > m ? a : m;
-    double corr = exp(m - m2); /* exp(-inf) = 0 on the first token */
-    double p = exp(a - m2);
-    l = l * corr + p;
-    dequant_token(&c, 1, b, kvh, i, vr);
-    for (int64_t x = 0; x < d; ++x) out[x] = out[x] * corr + p * vr[x];
-    m = m2;
-  }
-  if (l > 0.0)
-    for (int64_t x = 0; x < d; ++x) out[x] /= l;
-  free(qs); free(kr); free(vr);
 }
 
 int tqo_num_threads(void) {

@@ -232,10 +232,3 @@ def combine(o_part, m_part, l_part) -> np.ndarray:
     out = np.zeros((B, H_q, d), np.float64)
     lib().tqo_combine(_p(o_part), _p(m_part), _p(l_part), _i64(B), _i64(H_q), _i64(Cn), _i64(d), _p(out))
     return out
-
-
-def algorithm1(cache: Cache, q, alpha, b, h) -> np.ndarray:
-    q = np.ascontiguousarray(q, dtype=np.float16)
-    out = np.zeros((cache.d,), np.float64)
-    lib().tqo_algorithm1(*cache._cargs(), _p(q), _i64(q.shape[1]), C.c_double(alpha), _i64(b), _i64(h), _p(out))
-    return out

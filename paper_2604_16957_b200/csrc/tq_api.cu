@@ -1,4 +1,5 @@
 // extern "C" entry points of libtq: argument validation and dispatch.  See include/tq.h.
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 
@@ -9,16 +10,27 @@ namespace tq {
 static thread_local int g_last_cuda_error = 0;
 
 int device_sm_count() {
-  static const int sms = [] {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        n <= 0) {
-      (void)cudaGetLastError();
-      n = 148;  // B200
-    }
-    return n;
-  }();
-  return sms;
+  // one attribute query per device and process; 148 (B200) when no device can be asked
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> cached[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
+TestHooks& test_hooks() {
+  static TestHooks h;
+  return h;
 }
 
 bool pdl_enabled() {
@@ -30,8 +42,8 @@ bool pdl_enabled() {
 }
 
 namespace {
-
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+}  // namespace
 
 int check_cache(const tq_kv_cache* c) {
   if (!c) return TQ_ERR_NULL;
@@ -55,18 +67,21 @@ int check_heads(const tq_kv_cache* c, int H_q) {
   return TQ_OK;
 }
 
+int check_decode_grid(const tq_kv_cache* c, int H_q, int S_q) {
+  const long long tiles = (static_cast<long long>(H_q / c->H_kv) * S_q + 7) / 8;
+  return static_cast<long long>(c->H_kv) * tiles > 65535 ? TQ_ERR_SHAPE : TQ_OK;
+}
+
 int finish(cudaError_t e) {
   if (e == cudaSuccess) return TQ_OK;
+  (void)cudaGetLastError();  // clear the sticky-free launch error so that it is reported once, here
   g_last_cuda_error = static_cast<int>(e);
   return TQ_ERR_CUDA;
 }
 
-size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+namespace {
 
-bool use_simple_decode() {
-  const char* e = std::getenv("TQ_DECODE_IMPL");
-  return e && std::strcmp(e, "simple") == 0;
-}
+size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 }  // namespace
 }  // namespace tq
@@ -144,13 +159,12 @@ int tq_sdpa_int4_decode_multi(const tq_kv_cache* cache, const void* q, int32_t H
       (reinterpret_cast<uintptr_t>(l_part) & 3u) || (reinterpret_cast<uintptr_t>(status) & 3u))
     return TQ_ERR_ALIGN;
   if (window < 0 || S_q < 1 || S_q > TQ_MAX_QUERY_TOKENS) return TQ_ERR_SHAPE;
-  if (static_cast<long long>(cache->H_kv) * ((static_cast<long long>(H_q / cache->H_kv) * S_q + 7) / 8) > 65535)
-    return TQ_ERR_SHAPE;
+  if (int r = check_decode_grid(cache, H_q, S_q)) return r;
   const int span = (window > 0 && window < cache->S_cap) ? window : cache->S_cap;  // most tokens a sequence attends
   const int C = num_splits ? num_splits : tq_auto_splits(cache->B, cache->H_kv, H_q * S_q, cache->d, span);
   auto st = static_cast<cudaStream_t>(stream);
   auto qh = static_cast<const __half*>(q);
-  if (use_simple_decode())
+  if (test_hooks().decode_impl.load(std::memory_order_relaxed) == 1)
     return finish(launch_decode_simple(*cache, qh, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st));
   return finish(launch_decode_mma(*cache, qh, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st));
 }
@@ -254,6 +268,17 @@ const char* tq_result_string(int r) {
 
 int tq_last_cuda_error(void) { return g_last_cuda_error; }
 
-const char* tq_version(void) { return "libtq 0.1 (sm_100a)"; }
+const char* tq_version(void) { return "libtq 0.2 (sm_100a)"; }
+
+// Test hook (tq_internal.cuh); deliberately absent from tq.h.
+int tq_internal_test_hook(int key, int value) {
+  TestHooks& h = test_hooks();
+  switch (key) {
+    case 0: h.decode_impl.store(value, std::memory_order_relaxed); return 0;
+    case 1: h.spin_limit.store(value, std::memory_order_relaxed); return 0;
+    case 2: h.fault_block.store(value, std::memory_order_relaxed); return 0;
+    default: return -1;
+  }
+}
 
 }  // extern "C"

@@ -4,7 +4,7 @@
 //    stream, one lane per D/32 consecutive channels, warp-shuffle dot products, fp32 online
 //    softmax.  Src selects where a K/V row comes from:
 //      SrcInt4  -- the packed cache, dequantised in registers (a plain reference variant of the
-//                  fused kernel, selected with TQ_DECODE_IMPL=simple; the tensor-core kernel in
+//                  fused kernel, selected by the test hook of tq_internal.cuh; the tensor-core kernel in
 //                  tq_decode_mma.cu is the production path)
 //      SrcF32 / SrcF16 -- a materialised [B][H_kv][S_cap][D] matrix: the attention half of the
 //                  dequantize-then-attend comparison path (Sec. 3.1 first paragraph, Table 2).

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "tq.h"
 
 namespace tq {
@@ -143,6 +145,22 @@ cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, 
 cudaError_t launch_attend_mixed(const tq_kv_cache& c, const __half* k_fp16, const __half* v_fp16, const __half* q, int H_q,
                                 float attn_scale, int C, float* o_part, float* m_part, float* l_part, int32_t* status,
                                 cudaStream_t st);
-int device_sm_count();
+// Knobs for the library's own tests, set through tq_internal_test_hook (exported from the shared object for
+// the test suite but not declared in tq.h: not part of the ABI).  Read with relaxed loads on the call path.
+struct TestHooks {
+  std::atomic<int> decode_impl{0};   // key 0: 0 = tensor-core kernel, 1 = the scalar Algorithm-1 kernel of tq_attend_simple.cu
+  std::atomic<int> spin_limit{0};    // key 1: > 0 = poll limit of the decode kernel's stage waits (instrumented instantiation)
+  std::atomic<int> fault_block{-1};  // key 2: >= 0 = the copy of this 16-token block announces 16 bytes that never arrive
+};
+TestHooks& test_hooks();
+extern "C" int tq_internal_test_hook(int key, int value);
+
+int device_sm_count();  // SM count of the current device (looked up once per device)
+
+// Host-side argument checks shared by every entry point (tq_api.cu).  Each returns a tq_result.
+int check_cache(const tq_kv_cache* c);                       // pointers, sizes, alignment, paging fields
+int check_heads(const tq_kv_cache* c, int H_q);              // GQA shape
+int check_decode_grid(const tq_kv_cache* c, int H_q, int S_q);  // blockIdx.y limit of the decode kernel
+int finish(cudaError_t e);                                   // records a CUDA error for tq_last_cuda_error()
 
 }  // namespace tq

@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(2 * D, 1536 / (2 * D)) quantize_bulk_kernel(tq
   const long long bh = blockIdx.y;
   const int b = static_cast<int>(bh / c.H_kv);
   const int len = c.seq_lens[b];
-  if (len < 0 || len + T > c.S_cap) return;  // flagged by bump_lens_kernel
+  if (len < 0 || len > c.S_cap - T) return;  // flagged by bump_lens_kernel
   const int which = blockIdx.z;
   const int t = threadIdx.x / CPR, cc = threadIdx.x % CPR;  // token in the block, 8-element chunk in the row
   const int code_off = code_offset(D, which, t, cc * 4);
@@ -248,7 +248,7 @@ __global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= c.B) return;
   const int len = c.seq_lens[b];
-  if (len < 0 || len + T > c.S_cap) {
+  if (len < 0 || len > c.S_cap - T) {
     if (status) atomicOr(status, TQ_STATUS_CACHE_FULL);
     return;
   }
@@ -263,7 +263,7 @@ __global__ void __launch_bounds__(256) quantize_step_kernel(tq_kv_cache c, const
   pdl_launch_dependents();
   const int b = blockIdx.x;
   const int len = c.seq_lens[b];
-  if (len < 0 || len + T > c.S_cap) {
+  if (len < 0 || len > c.S_cap - T) {
     if (status && threadIdx.x == 0) atomicOr(status, TQ_STATUS_CACHE_FULL);
     return;
   }

@@ -47,17 +47,17 @@ using namespace tq;
 
 extern "C" int tq_sdpa_int4_attend_static(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale,
                                           void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
-  // same host-side checks as tq_sdpa_int4_decode / tq_sdpa_int4_combine, before anything is launched
-  if (!cache || !q || !out) return TQ_ERR_NULL;
-  if (!cache->blocks || !cache->seq_lens) return TQ_ERR_NULL;
+  // the host-side checks of tq_sdpa_int4_decode and tq_sdpa_int4_combine (contiguous and paged caches,
+  // every head dimension), before anything is launched
+  if (int r = check_cache(cache)) return r;
+  if (!q || !out) return TQ_ERR_NULL;
+  if (int r = check_heads(cache, H_q)) return r;
+  if (int r = check_decode_grid(cache, H_q, 1)) return r;
+  if (static_cast<long long>(cache->B) * H_q > 0x7fffffffLL) return TQ_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u) ||
+      (reinterpret_cast<uintptr_t>(status) & 3u))
+    return TQ_ERR_ALIGN;
   const int d = cache->d;
-  if (!(d == 64 || d == 128 || d == 256) || cache->B < 1 || cache->B > 65535 || cache->H_kv < 1 || cache->S_cap < 16 ||
-      (cache->S_cap % 16) != 0 || H_q < 1 || (H_q % cache->H_kv) != 0 || H_q / cache->H_kv > 64)
-    return TQ_ERR_SHAPE;
-  const void* ptrs[] = {cache->blocks, q, out};
-  for (const void* p : ptrs)
-    if (reinterpret_cast<uintptr_t>(p) & 15u) return TQ_ERR_ALIGN;
-  if ((reinterpret_cast<uintptr_t>(cache->seq_lens) & 3u) || (reinterpret_cast<uintptr_t>(status) & 3u)) return TQ_ERR_ALIGN;
 
   // largest split count, not above the library's usual choice, whose partials fit the fixed scratch
   int C = tq_auto_splits(cache->B, cache->H_kv, H_q, d, cache->S_cap);
@@ -65,11 +65,7 @@ extern "C" int tq_sdpa_int4_attend_static(const tq_kv_cache* cache, const void* 
   if (partial_bytes(cache->B, H_q, d, C) > TQ_STATIC_SCRATCH_BYTES) return TQ_ERR_WORKSPACE;  // B * H_q * d too large
 
   void* base = nullptr;
-  cudaError_t e = scratch_address(&base);
-  if (e != cudaSuccess) {
-    (void)cudaGetLastError();
-    return TQ_ERR_CUDA;
-  }
+  if (int r = finish(scratch_address(&base))) return r;
   const size_t n = static_cast<size_t>(cache->B) * H_q * C;
   char* p = static_cast<char*>(base);
   float* o_part = reinterpret_cast<float*>(p);
@@ -78,8 +74,8 @@ extern "C" int tq_sdpa_int4_attend_static(const tq_kv_cache* cache, const void* 
   auto st = static_cast<cudaStream_t>(stream);
   // Every partial of every (sequence, head, split) is written by phase 1, empty splits included, so
   // nothing in the scratch has to be cleared between calls.
-  e = launch_decode_mma(*cache, static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
-  if (e != cudaSuccess) return TQ_ERR_CUDA;
-  e = launch_combine(o_part, m_part, l_part, cache->B, H_q, d, C, out, out_is_fp32 != 0, st);
-  return e == cudaSuccess ? TQ_OK : TQ_ERR_CUDA;
+  if (int r = finish(launch_decode_mma(*cache, static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, o_part, m_part,
+                                       l_part, status, st)))
+    return r;
+  return finish(launch_combine(o_part, m_part, l_part, cache->B, H_q, d, C, out, out_is_fp32 != 0, st));
 }

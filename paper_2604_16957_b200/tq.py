@@ -19,7 +19,7 @@ if not os.path.exists(LIB_PATH):
 _lib = C.CDLL(LIB_PATH)
 
 TQ_OK, TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_WORKSPACE, TQ_ERR_CUDA = range(6)
-TQ_STATUS_CACHE_FULL, TQ_STATUS_EMPTY_SEQ, TQ_STATUS_BAD_LEN = 1, 2, 4
+TQ_STATUS_CACHE_FULL, TQ_STATUS_EMPTY_SEQ, TQ_STATUS_BAD_LEN, TQ_STATUS_TIMEOUT, TQ_STATUS_BAD_PAGE = 1, 2, 4, 8, 16
 TQ_GROUP, TQ_SPLIT_QUANTUM, TQ_MAX_SPLITS = 32, 16, 256
 TQ_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -79,6 +79,16 @@ _lib.tq_result_string.argtypes = [C.c_int]
 _lib.tq_result_string.restype = C.c_char_p
 _lib.tq_last_cuda_error.restype = C.c_int
 _lib.tq_version.restype = C.c_char_p
+# knob of the library's own tests (exported by the shared object, not declared in tq.h, not part of the ABI)
+_lib.tq_internal_test_hook.argtypes = [C.c_int, C.c_int]
+_lib.tq_internal_test_hook.restype = C.c_int
+HOOK_DECODE_IMPL, HOOK_SPIN_LIMIT, HOOK_FAULT_BLOCK = 0, 1, 2
+
+
+def _test_hook(key, value):
+    """Set a test knob of the library (see TestHooks in csrc/tq_internal.cuh); used only by tests/."""
+    if _lib.tq_internal_test_hook(int(key), int(value)) != 0:
+        raise ValueError(f"unknown test hook {key}")
 
 
 class TqError(RuntimeError):

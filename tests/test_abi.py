@@ -29,6 +29,9 @@ def test_every_declared_symbol_is_exported(lib):
         assert hasattr(lib, n), n
     from paper_2604_16957_b200 import tq
     assert sorted(tq.SYMBOLS) == names
+    assert {"TQ_STATUS_TIMEOUT", "TQ_STATUS_BAD_PAGE"} <= set(dir(tq)) and tq.TQ_STATUS_TIMEOUT == 8
+    assert tq._lib.tq_internal_test_hook(99, 0) == -1   # the test knob is exported but is not in the header
+    assert "tq_internal_test_hook" not in names
 
 
 def test_host_side_helpers(lib):
@@ -94,14 +97,32 @@ def test_argument_validation_without_gpu(lib):
     assert tq._lib.tq_sdpa_mixed_precision_attend(C.byref(cs), fake + 2, None, fake, 8, 1.0, 1, fake, fake, fake, None,
                                                   None) == tq.TQ_ERR_ALIGN
     assert tq._lib.tq_sdpa_int4_attend_static(None, fake, 8, 1.0, fake, 1, None, None) == tq.TQ_ERR_NULL
+    # ... including the entry point with the built-in scratch: same shape, alignment and grid checks
+    assert tq._lib.tq_sdpa_int4_attend_static(C.byref(cs), fake, 7, 1.0, fake, 1, None, None) == tq.TQ_ERR_SHAPE
+    assert tq._lib.tq_sdpa_int4_attend_static(C.byref(cs), fake, 8, 1.0, None, 1, None, None) == tq.TQ_ERR_NULL
+    assert tq._lib.tq_sdpa_int4_attend_static(C.byref(cs), fake + 4, 8, 1.0, fake, 1, None, None) == tq.TQ_ERR_ALIGN
+    assert tq._lib.tq_sdpa_int4_attend_static(C.byref(cs), fake, 8, 1.0, fake, 1, fake + 2, None) == tq.TQ_ERR_ALIGN
+    for bad in (dict(d=100), dict(S_cap=60), dict(H_kv=5000), dict(B=70000), dict(blocks=fake + 8)):
+        bs = tq.tq_kv_cache(**{**dict(blocks=fake, seq_lens=fake, B=1, H_kv=2, S_cap=64, d=128), **bad})
+        r = tq._lib.tq_sdpa_int4_attend_static(C.byref(bs), fake, 2 * bs.H_kv, 1.0, fake, 1, None, None)
+        assert r == (tq.TQ_ERR_ALIGN if "blocks" in bad else tq.TQ_ERR_SHAPE), bad
+    big = tq.tq_kv_cache(fake, fake, 1, 4096, 64, 128)
+    # 4096 KV heads x 8 head tiles fit the grid, but the partials of one split exceed the built-in scratch;
+    # with 4 query tokens the 32 head tiles per KV head exceed the grid's y limit
+    assert tq._lib.tq_sdpa_int4_attend_static(C.byref(big), fake, 4096 * 64, 1.0, fake, 1, None, None) == tq.TQ_ERR_WORKSPACE
+    assert tq._lib.tq_sdpa_int4_decode_multi(C.byref(big), fake, 4096 * 64, 4, 1.0, 0, 1, fake, fake, fake, None,
+                                             None) == tq.TQ_ERR_SHAPE
     # paged caches: page size a power of two >= 16, capacity = pages * page size, table aligned
     ok_paged = dict(blocks=fake, seq_lens=fake, B=1, H_kv=2, S_cap=128, d=128, page_table=fake, page_tokens=32,
                     max_pages=4, num_pages=9)
     for bad in (dict(page_tokens=48), dict(page_tokens=8), dict(max_pages=3), dict(num_pages=0), dict(S_cap=96)):
         cs = tq.tq_kv_cache(**{**ok_paged, **bad})
         assert tq._lib.tq_sdpa_int4_decode(C.byref(cs), fake, 8, 1.0, 1, fake, fake, fake, None, None) == tq.TQ_ERR_SHAPE, bad
+        # a page size below 16 used to reach a host-side division by zero through this entry point
+        assert tq._lib.tq_sdpa_int4_attend_static(C.byref(cs), fake, 8, 1.0, fake, 1, None, None) == tq.TQ_ERR_SHAPE, bad
     cs = tq.tq_kv_cache(**{**ok_paged, "page_table": fake + 2})
     assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 1, None, None) == tq.TQ_ERR_ALIGN
+    assert tq._lib.tq_sdpa_int4_attend_static(C.byref(cs), fake, 8, 1.0, fake, 1, None, None) == tq.TQ_ERR_ALIGN
     # split ranges under a window tile exactly the window
     for length, window, Cn in ((3000, 1024, 5), (1029, 1024, 3), (7, 1024, 2), (100, 1, 4), (0, 5, 2)):
         prev = max(0, length - window)

@@ -179,11 +179,11 @@ def test_simple_reference_kernel_matches_oracle(gpu, oracle):
     sh = I.Shape("x", 2, 24, 2, 128, 128 ** -0.5)
     host, dev = _both(gpu, oracle, sh, 512, 15, lens=[512, 100])
     q = I.make_q(sh, 15)
-    os.environ["TQ_DECODE_IMPL"] = "simple"
+    tq._test_hook(tq.HOOK_DECODE_IMPL, 1)
     try:
         out, _, _ = fused_attention(tq, torch, dev, q, sh.alpha, num_splits=5)
     finally:
-        del os.environ["TQ_DECODE_IMPL"]
+        tq._test_hook(tq.HOOK_DECODE_IMPL, 0)
     assert_attention_close(out, oracle.attention(host, q, sh.alpha), "simple")
 
 
@@ -344,7 +344,7 @@ def test_multi_query_decode(gpu, oracle, d, H_q, H_kv, S_q, impl):
     q = np.ascontiguousarray(np.stack([I.make_q(sh, 61, stream=s) for s in range(S_q)], axis=1))
     qd = torch.from_numpy(q).cuda()
     if impl == "simple":
-        os.environ["TQ_DECODE_IMPL"] = "simple"
+        tq._test_hook(tq.HOOK_DECODE_IMPL, 1)
     try:
         for window, C in ((0, 0), (0, 3), (1024, 0), (20, 2), (1, 1)):
             ref = oracle.attention_multi(host, q, sh.alpha, window)
@@ -362,7 +362,7 @@ def test_multi_query_decode(gpu, oracle, d, H_q, H_kv, S_q, impl):
                     assert not got[2, s].any() and not ref[2, s].any()
             assert_attention_close(got.reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d), f"S_q {S_q} window {window} C {C}")
     finally:
-        os.environ.pop("TQ_DECODE_IMPL", None)
+        tq._test_hook(tq.HOOK_DECODE_IMPL, 0)
 
 
 @pytest.mark.parametrize("impl", ["mma", "simple"])
@@ -380,7 +380,7 @@ def test_head_dim_512(gpu, oracle, impl):
     assert_cache_bits_equal(dev, host)
     q = I.make_q(sh, 71)
     if impl == "simple":
-        os.environ["TQ_DECODE_IMPL"] = "simple"
+        tq._test_hook(tq.HOOK_DECODE_IMPL, 1)
     try:
         for C in (0, 1, 5):
             out, _, _ = fused_attention(tq, torch, dev, q, sh.alpha, num_splits=C)
@@ -395,7 +395,7 @@ def test_head_dim_512(gpu, oracle, impl):
             ref = oracle.attention_multi(host, q3, sh.alpha, window)
             assert_attention_close(out.cpu().numpy().reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d), f"d512 w={window}")
     finally:
-        os.environ.pop("TQ_DECODE_IMPL", None)
+        tq._test_hook(tq.HOOK_DECODE_IMPL, 0)
 
 
 def test_mixed_precision_attend_matches_oracle(gpu, oracle):

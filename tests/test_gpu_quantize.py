@@ -95,6 +95,25 @@ def test_decode_step_appends_and_overflow(gpu, oracle):
     assert host.lens.tolist() == [6, 23, 64, 46]
 
 
+def test_lengths_near_int_max_are_refused_not_wrapped(gpu):
+    """A caller-owned length close to INT_MAX must not wrap around in the capacity test: the sequence is
+    skipped and flagged, its length and every byte of the cache stay as they were (small and bulk paths)."""
+    tq, torch = gpu
+    shape = I.Shape("m", 2, 4, 2, 128, 0.1)
+    for T in (1, 3, 600):
+        dev = tq.KVCache(shape.B, shape.H_kv, 1024, shape.d)
+        dev.blocks.fill_(0xA5)
+        dev.seq_lens.copy_(torch.tensor([2 ** 31 - 1, 2 ** 31 - 2], dtype=torch.int32))
+        before = dev.blocks.clone()
+        k, v = I.make_kv(shape, T, 9)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        tq.tq_kv_quantize_append(dev, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
+        torch.cuda.synchronize()
+        assert int(status.item()) & tq.TQ_STATUS_CACHE_FULL
+        assert dev.seq_lens.cpu().tolist() == [2 ** 31 - 1, 2 ** 31 - 2]
+        assert torch.equal(dev.blocks, before)
+
+
 def test_bulk_path_with_ragged_lengths_and_overflow(gpu, oracle):
     tq, torch = gpu
     shape = I.Shape("r", 3, 8, 2, 128, 0.1)

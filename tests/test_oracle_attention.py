@@ -65,14 +65,30 @@ def test_brute_force_tiny_python_loops(oracle):
         assert np.abs(got[0, h] - np.array(out)).max() < 1e-13
 
 
-def test_algorithm1_one_pass_equals_two_pass_definition(oracle):
+def test_blocked_log_sum_exp_evaluation_equals_two_pass_definition(oracle):
+    """The same attention evaluated another way: tokens cut into uneven blocks, each block reduced to its
+    log-sum-exp and its softmax-weighted value mean, the blocks then merged by their log-sum-exps.  A
+    mistake in the oracle's maximum, exponent or normalisation shows up against this."""
     sh = I.Shape("t", 2, 4, 2, 64, 0.125)
-    cache = _cache(oracle, sh, 300, 8, lens=[300, 17])
+    lens = [300, 17]
+    cache = _cache(oracle, sh, 300, 8, lens=lens)
     q = I.make_q(sh, 8)
     full = oracle.attention(cache, q, sh.alpha)
+    kd, vd = _dequant(oracle, cache)
+    G = sh.H_q // sh.H_kv
     for b in range(2):
+        n = lens[b]
+        cuts = [0] + sorted(set(np.random.default_rng(b).integers(1, n, 6).tolist())) + [n]
         for h in range(4):
-            assert np.abs(oracle.algorithm1(cache, q, sh.alpha, b, h) - full[b, h]).max() < 1e-12
+            a = sh.alpha * (kd[b, h // G, :n] @ q[b, h].astype(np.float64))
+            lses, means = [], []
+            for i0, i1 in zip(cuts[:-1], cuts[1:]):
+                lse = np.logaddexp.reduce(a[i0:i1])
+                lses.append(lse)
+                means.append(np.exp(a[i0:i1] - lse) @ vd[b, h // G, i0:i1])
+            w = np.exp(np.array(lses) - np.logaddexp.reduce(lses))
+            assert abs(w.sum() - 1) < 1e-12
+            assert np.abs(w @ np.array(means) - full[b, h]).max() < 1e-12
 
 
 def test_constant_v_returns_v(oracle):
