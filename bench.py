@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-compare", action="store_true", help="skip the dequantize-then-attend timing")
     ap.add_argument("--splits", type=int, default=0, help="sequence splits C of the fused kernel (0 = library default)")
+    ap.add_argument("--no-parity", action="store_true", help="skip the oracle check of sampled layers of the timed state")
     return ap.parse_args()
 
 
@@ -62,7 +63,7 @@ class ClockSampler:
                0x80: "hw_power_brake", 0x2: "applications_clocks_setting", 0x100: "display_clock_setting"}
 
     def __init__(self, index):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.reasons, self.max_mhz, self.power_w, self.mem_mhz = [], set(), None, [], []
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -79,6 +80,11 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    self.power_w.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+                    self.mem_mhz.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_MEM)))
+                except Exception:
+                    pass
                 try:
                     mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
                 except Exception:
@@ -104,8 +110,13 @@ class ClockSampler:
     def summary(self):
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
-        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        out = {"sm_mhz": int(statistics.median(self.samples)), "sm_min_mhz": min(self.samples), "sm_max_mhz": self.max_mhz,
+               "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        if self.power_w:
+            out["power_w_median"] = round(statistics.median(self.power_w), 1)
+            out["power_w_max"] = round(max(self.power_w), 1)
+            out["mem_mhz"] = int(statistics.median(self.mem_mhz))
+        return out
 
 
 # ------------------------------------------------------------------ CPU oracle leg
@@ -146,7 +157,7 @@ def run_reference(args, rank):
               f"{args.layers}, fp64 oracle on the oracle-quantised cache")
     line = {"impl": "reference", "metric": "int4 decode-attn us/layer @128K (Llama-70B shape)", "value": value,
             "unit": "us/layer", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": value * args.layers / 1e3, "higher_is_better": False, "scaling": "weak",
+            "ms_per_step": value / 1e3, "layers_per_step": 1, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": config_dict(args),
             "cpu_baseline": {"value": value, "unit": "us/layer", "cores": threads, "kind": "oracle", "sample": sample},
@@ -208,21 +219,27 @@ def main():
     caches = []
     gen = torch.Generator(device=dev)
     ch_rng = torch.Generator().manual_seed(4242)
+    outlier_channels = [[torch.randperm(D, generator=ch_rng)[:4] for _ in range(H_KV)] for _ in range(L)]
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    for layer in range(L):
+
+    def layer_kv(layer):
+        """The seeded fp16 K, V that layer's cache was quantised from (regenerated for the parity check)."""
         gen.manual_seed(7000 + layer + 1000 * rank)
         k = torch.randn((1, H_KV, S, D), generator=gen, device=dev, dtype=torch.float32)
         for h in range(H_KV):
-            ch = torch.randperm(D, generator=ch_rng)[:4].to(dev)
-            k[0, h, :, ch] *= 10.0
+            k[0, h, :, outlier_channels[layer][h].to(dev)] *= 10.0
         k = k.to(torch.float16)
         v = torch.randn((1, H_KV, S, D), generator=gen, device=dev, dtype=torch.float32).to(torch.float16)
+        return k, v
+
+    for layer in range(L):
+        k, v = layer_kv(layer)
         cache = tq.KVCache(1, H_KV, S_cap, D, device=dev)
         tq.tq_kv_quantize_append(cache, k, v, status)
         caches.append(cache)
         del k, v
     torch.cuda.synchronize()
-    assert int(status.item()) == 0
+    assert int(status.item()) == 0, f"device status word set while filling the caches: {int(status.item())}"
 
     # per-layer step inputs (q, k_new, v_new) in one buffer, outputs in another
     per_layer_in = H_Q * D + 2 * H_KV * D
@@ -302,7 +319,16 @@ def main():
     t_e2e = time_graph(g_step, W, K, pre=lambda: inp.copy_(h_in, non_blocking=True),
                        post=lambda: (h_out.copy_(out, non_blocking=True), torch.cuda.current_stream().synchronize()))
     e2e_us = t_e2e / K / L * 1e6
-    assert int(status.item()) == 0, "device status word set during the benchmark"
+    assert int(status.item()) == 0, f"device status word set during the benchmark: {int(status.item())}"
+
+    # ---- what was timed is also what is right: one more replay of the timed graph from the initial lengths,
+    # then sampled layers of that very state against the CPU oracle (outside every timed region)
+    parity = None
+    if rank == 0 and not args.no_parity:
+        reset_lens()
+        g_step.replay()
+        torch.cuda.synchronize()
+        parity = check_sampled_layers(torch, caches, layer_kv, inp, out, S, S_cap, sorted({0, L // 2 - 1 if L > 1 else 0, L - 1}))
 
     if rank != 0:
         if world > 1:
@@ -329,6 +355,8 @@ def main():
                                        "decode": decode_us, "append": t_append / K / L * 1e6},
             "hbm_gbs_whole_step": alg_bytes / (us_per_layer * 1e-6) / 1e9, "num_splits": C,
             "paper_context": PAPER_CONTEXT, "device": device_info(torch, dev)}
+    if parity is not None:
+        line["parity"] = parity
     if world > 1:
         line["config"]["replicas"] = "independent replicas, no collective (the path does not shard in this build)"
 
@@ -343,6 +371,45 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def check_sampled_layers(torch, caches, layer_kv, inp, out, S, S_cap, layers):
+    """Oracle check of the state the benchmark timed.  For each sampled layer: the oracle quantises the same
+    seeded fp16 K, V (and the step's new token) on the host; the device cache must equal it bit for bit over
+    the S + 1 valid tokens; the step's output must match the oracle's fp64 attention over that cache within
+    max-abs 2e-3 (+ half an fp16 ulp, the output being fp16) and relative L2 1e-3 (+ 2^-11 for the fp16
+    rounding).  Raises if not."""
+    import numpy as np
+    from oracle import tq_oracle as O
+    res = {"layers": layers, "max_abs": 0.0, "rel_l2": 0.0, "cache_bits_equal": True,
+           "tolerance": {"max_abs": 2e-3, "rel_l2": 1e-3, "fp16_output_allowance": "half ulp / 2^-11"}}
+    for i in layers:
+        k, v = layer_kv(i)
+        host = O.Cache(1, H_KV, S_cap, D)
+        host.append(k.cpu().numpy(), v.cpu().numpy())
+        del k, v
+        row = inp[i].cpu().numpy()
+        q = row[:H_Q * D].reshape(1, H_Q, D)
+        host.append(row[H_Q * D:H_Q * D + H_KV * D].reshape(1, H_KV, 1, D), row[H_Q * D + H_KV * D:].reshape(1, H_KV, 1, D))
+        n = S + 1
+        assert int(caches[i].seq_lens.item()) == n == int(host.lens[0])
+        for d_arr, h_arr in zip(caches[i].arrays_token_major(), host.arrays()):
+            dv, hv = d_arr[:, :, :n].cpu().numpy(), h_arr[:, :, :n]
+            if dv.dtype == np.float16:
+                dv, hv = dv.view(np.uint16), hv.view(np.uint16)
+            if not np.array_equal(dv, hv):
+                res["cache_bits_equal"] = False
+        ref = O.attention(host, q, ALPHA)
+        got = out[i].float().cpu().numpy().astype(np.float64).reshape(ref.shape)
+        diff = np.abs(got - ref)
+        rel = float(np.sqrt((diff ** 2).sum() / max((ref ** 2).sum(), 1e-300)))
+        res["max_abs"] = max(res["max_abs"], float(diff.max()))
+        res["rel_l2"] = max(res["rel_l2"], rel)
+        ok = bool(np.all(diff <= 2e-3 + np.abs(ref) * 2.0 ** -11) and rel <= 1e-3 + 2.0 ** -11)
+        if not (ok and res["cache_bits_equal"]):
+            raise AssertionError(f"benchmark state fails the oracle check at layer {i}: {res}")
+        del host
+    return res
 
 
 def device_info(torch, dev):

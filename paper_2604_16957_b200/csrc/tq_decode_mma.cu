@@ -53,7 +53,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 4.0f;  // log2 units
 constexpr float kNoMax = -1.0e30f;         // running reference before any token was seen
-constexpr int kMaxSpins = 1 << 22;         // bound of every mbarrier wait
+constexpr long long kMaxWaitCycles = 1LL << 22;  // bound of every mbarrier wait: about 2 ms of SM clock
 constexpr uint32_t kMaskLo = 0x000F000Fu;  // nibbles 0 / 4 of a 32-bit word: n * 2^-24 as fp16
 constexpr uint32_t kMaskHi = 0x00F000F0u;  // nibbles 1 / 5: n * 2^-20 as fp16
 
@@ -142,6 +142,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// non-blocking probe of a phase
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // contiguous global -> shared copy (both 16-byte aligned, size a multiple of 16) completing on an mbarrier
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
@@ -154,12 +164,14 @@ __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_c
 
 template <int D>
 struct WarpCtx {
-  uint32_t kaddr[Cfg<D>::NGW / 2];  // ldmatrix row address (offset in a stage) this lane supplies, per K load
-  uint32_t vaddr[Cfg<D>::NGW / 2];  // same for the V loads
+  uint32_t kaddr[Cfg<D>::NGW / 2];  // ldmatrix row address this lane supplies (slot 0 of the warp's ring), per K load; V: + PK
   uint32_t ksz_lane, vsz_lane;
+  uint32_t kz_lane;            // row address of the scale / zero load that feeds the zero-point MMA of the scores
+  uint32_t fl_m, fl_h;         // half2 lane flags of that MMA's A operand: (0 | -1), (1 | 0) for tid4 < 2 | >= 2
   float cs;
   int gid;
 };
+template <int D> struct KZ { static constexpr bool on = Cfg<D>::DS == 1 && Cfg<D>::NGW == 4; };
 
 // Which tokens of a block count, as rows relative to the block's first token.  Rows >= zrow lie past the
 // end of the sequence and hold unspecified bytes; column j (j = 0, 1: the thread's two score columns, i.e.
@@ -171,8 +183,9 @@ struct RowMask {
 // First half of one 16-token block: this warp's share of the scores S[token][head] (over its DW channels;
 // they carry a factor 2^-24).  TAIL = a block in which some token does not count for some column.
 template <int D, bool TAIL>
-__device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_s, const RowMask& mk,
+__device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_off, const RowMask& mk,
                                              const uint32_t (&qf)[Cfg<D>::NGW][4], const float (&qs)[Cfg<D>::NGW][2],
+                                             const uint32_t (&qz)[2], const float (&cz)[2],
                                              const float (&zero4)[4], float (&sc)[4]) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW;
@@ -186,14 +199,46 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
     }
     __syncwarp();
   }
-  // matrix j = 4 * i + m of load i is (tokens 8 * (j / NGW) .., group j % NGW of this warp)
+  // matrix j = 4 * i + m of load i is (group j / 2 of this warp, tokens 8 * (j % 2) ..), as for V below
   uint32_t kw[NGW / 2][4], ksz[4];
 #pragma unroll
-  for (int i = 0; i < NGW / 2; ++i) ldmatrix_x4(kw[i], st_s + cx.kaddr[i]);
+  for (int i = 0; i < NGW / 2; ++i) ldmatrix_x4(kw[i], cx.kaddr[i] + st_off);
+  if constexpr (KZ<D>::on) {
+    // Zero-point term of the scores by one MMA: sum_g (s_g z_g) * qsum_g with the product s * z split
+    // exactly into an fp16 pair (hi = rn(s z), lo = s z - hi by a fused multiply-add) and qsum into
+    // hi + lo as well; k slots 0-3 hi x hi, 4-7 lo x hi, 8-11 hi x lo (lo x lo is below 2^-22 of the term).
+    // The transposing load hands lane (gid, tid4) the half2 (x[g][token], x[g+1][token]) of groups
+    // g = 2 * (tid4 & 1): scales of tokens gid, gid + 8, then zeros of the same.
+    uint32_t r[4];
+    ldmatrix_x4_trans(r, cx.kz_lane + st_off);
+    const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
+    const uint32_t a0 = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hmul2(pa, u32_as_h2(cx.fl_m))));
+    const uint32_t a1 = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hmul2(pb, u32_as_h2(cx.fl_m))));
+    const uint32_t a2 = h2_as_u32(__hmul2(pa, u32_as_h2(cx.fl_h))), a3 = h2_as_u32(__hmul2(pb, u32_as_h2(cx.fl_h)));
+    float accz[4];
+    mma16816_first(accz, a0, a1, a2, a3, qz[0], qz[1], zero4);
+    // scales of all four groups for tokens gid, gid + 8: matrices (g0 g1 | tokens 0-7), (g0 g1 | 8-15), (g2 g3 | ..)
+    ldmatrix_x4_trans(ksz, cx.ksz_lane + st_off);
+    sc[0] = accz[0] * cz[0]; sc[1] = accz[1] * cz[1]; sc[2] = accz[2] * cz[0]; sc[3] = accz[3] * cz[1];
+#pragma unroll
+    for (int g = 0; g < NGW; ++g) {
+      const uint32_t w0 = kw[g / 2][2 * (g % 2)];                // token gid
+      const uint32_t w8 = kw[g / 2][2 * (g % 2) + 1];            // token gid + 8
+      float acc[4];
+      mma16816_first(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1], zero4);
+      const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
+      mma16816(acc, y0 & kMaskLo, y8 & kMaskLo, y0 & kMaskHi, y8 & kMaskHi, qf[g][2], qf[g][3]);
+      const __half2 slo = u32_as_h2(ksz[2 * (g / 2)]), shi = u32_as_h2(ksz[2 * (g / 2) + 1]);
+      const float s_lo = (g & 1) ? __high2float(slo) : __low2float(slo);
+      const float s_hi = (g & 1) ? __high2float(shi) : __low2float(shi);
+      sc[0] = fmaf(s_lo, acc[0], sc[0]); sc[1] = fmaf(s_lo, acc[1], sc[1]);
+      sc[2] = fmaf(s_hi, acc[2], sc[2]); sc[3] = fmaf(s_hi, acc[3], sc[3]);
+    }
+  } else {
 #pragma unroll
   for (int g = 0; g < NGW; ++g) {
-    const uint32_t w0 = kw[g / 4][g % 4];                      // token gid
-    const uint32_t w8 = kw[(NGW + g) / 4][(NGW + g) % 4];      // token gid + 8
+    const uint32_t w0 = kw[g / 2][2 * (g % 2)];                // token gid
+    const uint32_t w8 = kw[g / 2][2 * (g % 2) + 1];            // token gid + 8
     float acc[4];
     mma16816_first(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1], zero4);
     const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
@@ -202,7 +247,7 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
     // matrices are (scale | tokens 0-7), (scale | 8-15), (zero | 0-7), (zero | 8-15), each with rows
     // alternating between the 16-byte chunks of groups g and g+1, so every lane receives element gid
     // of both chunks: half2 (x[g][token], x[g+1][token]).
-    if ((g & 1) == 0) ldmatrix_x4_trans(ksz, st_s + cx.ksz_lane + 32 * g);
+    if ((g & 1) == 0) ldmatrix_x4_trans(ksz, cx.ksz_lane + st_off + 32 * g);
     const float s_lo = (g & 1) ? __high2float(u32_as_h2(ksz[0])) : __low2float(u32_as_h2(ksz[0]));
     const float s_hi = (g & 1) ? __high2float(u32_as_h2(ksz[1])) : __low2float(u32_as_h2(ksz[1]));
     const float z_lo = (g & 1) ? __high2float(u32_as_h2(ksz[2])) : __low2float(u32_as_h2(ksz[2]));
@@ -216,11 +261,12 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
       sc[2] = fmaf(s_hi, t2, sc[2]); sc[3] = fmaf(s_hi, t3, sc[3]);
     }
   }
+  }
 }
 
 // Second half: online softmax on the complete scores, then P.V for this warp's DW output channels.
 template <int D, bool TAIL>
-__device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t st_s, const RowMask& mk,
+__device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t st_off, const RowMask& mk,
                                                  const float (&sc)[4], float (&oacc)[Cfg<D>::DW / 16][4],
                                                  float (&zacc)[Cfg<D>::NGW][4], float& m0, float& m1, float& l0,
                                                  float& l1) {
@@ -288,13 +334,13 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     // four result registers are, as they stand, the A operand of the zero-point MMA: rows 0-7 hold z_g
     // (c0, c1 accumulate sum_tok z_g * B_g), rows 8-15 hold the scales and produce values never read.
     uint32_t vsz[4];
-    ldmatrix_x4(vsz, st_s + cx.vsz_lane + 32 * g);
+    ldmatrix_x4(vsz, cx.vsz_lane + st_off + 32 * g);
     const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vsz[1])));
     const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vsz[3])));
     mma16816(zacc[g], vsz[0], vsz[1], vsz[2], vsz[3], b0, b1);
     // r1 = (tokens 2*tid4, 2*tid4+1), r2 = (tokens 2*tid4+8, +9): 16-bit lane gid of chunk g, i.e. codes of
     // channels 32g + 4*gid .. +3 of two tokens side by side
-    if ((g & 1) == 0) ldmatrix_x4_trans(vw, st_s + cx.vaddr[g / 2]);
+    if ((g & 1) == 0) ldmatrix_x4_trans(vw, cx.kaddr[g / 2] + st_off + Cfg<D>::PK);
     const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
     mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
     const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
@@ -318,12 +364,16 @@ __device__ __noinline__ RowMask general_row_mask(const int32_t* seq_lens, int b,
 }
 
 // Bounded wait on an mbarrier phase; false if the copy did not complete within the limit.
-__device__ __forceinline__ bool wait_stage(uint32_t bar, uint32_t parity) {
-  int spins = 0;
+__device__ __noinline__ bool wait_stage_slow(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (++spins > kMaxSpins) return false;
+    if (clock64() - t0 > kMaxWaitCycles) return false;
   }
   return true;
+}
+__device__ __forceinline__ bool wait_stage(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;  // the common case: the copy landed while the warp computed
+  return wait_stage_slow(bar, parity);
 }
 
 // GEN = the general form: a sliding window (Appendix A) and / or several query tokens per sequence
@@ -347,7 +397,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const int GV = GEN ? G * S_q : G;  // columns of this KV head
   const int tiles = (GV + 7) >> 3;
   const int c = blockIdx.x, kvh = blockIdx.y / tiles, tile = blockIdx.y - kvh * tiles, b = blockIdx.z;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gid = lane >> 2, tid4 = lane & 3;
+  // the warp index through a broadcast, so that the compiler keeps what derives from it (ring, barrier and
+  // block addresses) in uniform registers
+  const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0);
+  const int lane = threadIdx.x & 31, gid = lane >> 2, tid4 = lane & 3;
   const int team = warp / DS, sub = warp - team * DS;  // this warp works on channels [sub * DW, (sub + 1) * DW)
   const int v0 = tile * 8;                   // first column of this tile
   const int nh = min(8, GV - v0);            // columns in the tile; the rest of N = 8 is zero padding
@@ -408,9 +461,9 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   if (DS > 1 || PAGED) __syncthreads();  // a team's warps wait on the same barriers; everybody reads the page addresses
   else __syncwarp();
-  auto issue = [&](int n) {
+  auto issue_to = [&](int n, int slot) {
     if (sub == 0 && lane == 0) {
-      const int slot = n & (Cf::NST - 1), blk = blk0 + team + n * NTEAM;
+      const int blk = blk0 + team + n * NTEAM;
       const uint8_t* src;
       if (PAGED) src = page_ptr[(blk >> pshift) - page0] + static_cast<size_t>(blk & ((1 << pshift) - 1)) * Cf::STAGE;
       else src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
@@ -419,6 +472,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       bulk_g2s(ring_s + slot * Cf::STAGE, src, Cf::STAGE, bar);
     }
   };
+
+  auto issue = [&](int n) { issue_to(n, n & (Cf::NST - 1)); };
 
   // start streaming: the first stages are in flight while q is turned into fragments
 #pragma unroll
@@ -455,6 +510,43 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     qs[g][1] = __shfl_sync(0xffffffffu, sum, (2 * tid4 + 1) * 4);
   }
 
+  // B operand and per-column factor of the zero-point MMA of the scores (see block_scores)
+  uint32_t qz[2] = {0u, 0u};
+  float cz[2] = {0.f, 0.f};
+  if constexpr (KZ<D>::on) {
+    // head gid's row scaled by a power of two so that its largest magnitude lies in [1, 2): the group sums
+    // then fit fp16 pairs whatever the size of q
+    float mx = 0.f, sumg[NGW];
+#pragma unroll
+    for (int g = 0; g < NGW; ++g) {
+      const __half2* h2 = reinterpret_cast<const __half2*>(&qraw[g]);
+      float sum = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h2[i]);
+        sum += f.x + f.y;
+        mx = fmaxf(mx, fmaxf(fabsf(f.x), fabsf(f.y)));
+      }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      sumg[g] = sum;
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    int e = ((__float_as_int(mx) >> 23) & 0xff) - 127;  // floor(log2(max)); an all-zero row gives -127
+    e = max(-24, min(e, 15));
+    const float down = __int_as_float((127 - e) << 23);       // 2^-e
+    const float up24 = __int_as_float((127 + e - 24) << 23);  // 2^(e - 24): the code operands carry 2^-24
+    const float sa = -(tid4 & 1 ? sumg[2] : sumg[0]) * down, sb = -(tid4 & 1 ? sumg[3] : sumg[1]) * down;
+    const __half2 hi = __floats2half2_rn(sa, sb);
+    const float2 hf = __half22float2(hi);
+    const __half2 lo = __floats2half2_rn(sa - hf.x, sb - hf.y);
+    qz[0] = h2_as_u32(hi);
+    qz[1] = tid4 < 2 ? h2_as_u32(lo) : 0u;
+    cz[0] = __shfl_sync(0xffffffffu, up24, (2 * tid4) * 4);
+    cz[1] = __shfl_sync(0xffffffffu, up24, (2 * tid4 + 1) * 4);
+  }
+
   float oacc[Cf::DW / 16][4];  // [M tile][c0..c3]: rows = channels, cols = heads 2*tid4, 2*tid4+1
   float zacc[NGW][4];          // sum_tok B_g * z_g: [0], [1] are heads 2*tid4, 2*tid4+1; [2], [3] are not used
   float zero4[4];              // four registers holding 0, opaque to the compiler: the C operand of accumulator-less MMAs
@@ -485,23 +577,59 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // this warp's channel groups sub * NGW .. (see block_scores / block_softmax_pv)
   WarpCtx<D> cx;
   cx.cs = cs; cx.gid = gid;
-  cx.ksz_lane = 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32 + sub * NGW * 32;
-  cx.vsz_lane = 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
+  cx.ksz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32 + sub * NGW * 32;
+  if constexpr (KZ<D>::on) {
+    cx.ksz_lane = ring_s + 2 * Cf::PK + (2 * (lane >> 4) + (lane & 1)) * 32 + ((lane >> 3) & 1) * 16;
+    cx.kz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32;
+    cx.fl_m = tid4 < 2 ? 0u : 0xBC00BC00u;  // half2 (0, 0) | (-1, -1)
+    cx.fl_h = tid4 < 2 ? 0x3C003C00u : 0u;  // half2 (1, 1) | (0, 0)
+  } else {
+    cx.kz_lane = cx.fl_m = cx.fl_h = 0;
+  }
+  cx.vsz_lane = ring_s + 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
 #pragma unroll
   for (int i = 0; i < NGW / 2; ++i) {
     const int j = 4 * i + (lane >> 3);
-    const int ktok = (lane & 7) + 8 * (j / NGW), kgrp = sub * NGW + j % NGW;
-    cx.kaddr[i] = ktok * Cf::ROWB + ((kgrp ^ Cf::swz(ktok)) << 4);
-    const int vtok = (lane & 7) + 8 * (j % 2), vgrp = sub * NGW + j / 2;
-    cx.vaddr[i] = Cf::PK + vtok * Cf::ROWB + ((vgrp ^ Cf::swz(vtok)) << 4);
+    const int tok = (lane & 7) + 8 * (j % 2), grp = sub * NGW + j / 2;
+    cx.kaddr[i] = ring_s + tok * Cf::ROWB + ((grp ^ Cf::swz(tok)) << 4);
   }
   // score exchange of a team: [2 (parity of k)][DS][32 lanes] float4, then [2][DS] timeout flags
   float4* const xch = reinterpret_cast<float4*>(smem + Cf::XCH + team * Cf::XCH_TEAM);
   int* const xflag = reinterpret_cast<int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
 
   bool timed_out = false;
-#pragma unroll 2  // measured: 34.3 -> 33.3 us per 128K layer (loop overhead shared by two blocks)
-  for (int k = 0; k < nblk; ++k) {
+  int k = 0;
+  if constexpr (DS == 1 && !GEN) {
+    // Full blocks four at a time: ring slot, barrier and stage offsets are constants of each of the four
+    // copies of the block step, so the loop carries no slot arithmetic.
+    static_assert(Cf::NST == 4, "the unrolled loop walks a ring of four slots");
+    const RowMask all{kBlk, 0, kBlk, 0, kBlk};
+    uint32_t par = 0;
+    // The barrier of the next block is probed one block ahead (the probe's latency then hides behind a block
+    // of arithmetic); only a probe that came back negative is followed by the blocking wait.  No warp-wide
+    // synchronisation is needed before a slot is refilled: its last readers were the warp-collective loads
+    // of the previous block, whose results the MMAs issued since then have already consumed.
+    bool ready = k + 4 <= nfull ? mbar_test_wait(bars, 0) : false;
+    for (; k + 4 <= nfull && !timed_out; k += 4) {
+#pragma unroll
+      for (int S = 0; S < 4; ++S) {
+        if (!timed_out) {
+          if (!ready && !wait_stage(bars + 8 * S, par)) {
+            timed_out = true;
+          } else {
+            if (k + S + 3 < nblk) issue_to(k + S + 3, (S + 3) & 3);
+            ready = mbar_test_wait(bars + 8 * ((S + 1) & 3), S == 3 ? par ^ 1 : par);
+            float sc[4];
+            block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, cz, zero4, sc);
+            block_softmax_pv<D, false>(cx, S * Cf::STAGE, all, sc, oacc, zacc, m0, m1, l0, l1);
+          }
+        }
+      }
+      par ^= 1;
+    }
+  }
+#pragma unroll 1
+  for (; k < nblk && !timed_out; ++k) {
     // Wait for this block's bytes.  The wait is bounded: if the copy never completes (which would take
     // a bad pointer), the warp flags the status word and stops consuming.
     const bool arrived = wait_stage(bars + 8 * (k & (Cf::NST - 1)), (k / Cf::NST) & 1);
@@ -510,7 +638,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
       refill(k + Cf::NST - 1);
     }
-    const uint32_t st_s = ring_s + (k & (Cf::NST - 1)) * Cf::STAGE;
+    const uint32_t st_s = (k & (Cf::NST - 1)) * Cf::STAGE;
     const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
     const bool plain = GEN ? static_cast<unsigned>(k - nhead) < nplain : k < nfull;
     auto mask_of_block = [&]() {
@@ -525,17 +653,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     float sc[4];
     if (DS == 1) {
       if (plain) {
-        block_scores<D, false>(cx, st, st_s, all, qf, qs, zero4, sc);
+        block_scores<D, false>(cx, st, st_s, all, qf, qs, qz, cz, zero4, sc);
         block_softmax_pv<D, false>(cx, st_s, all, sc, oacc, zacc, m0, m1, l0, l1);
       } else {
         const RowMask mk = mask_of_block();
-        block_scores<D, true>(cx, st, st_s, mk, qf, qs, zero4, sc);
+        block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
         block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       }
     } else {
       const RowMask mk = plain ? all : mask_of_block();
-      if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, zero4, sc);
-      else block_scores<D, true>(cx, st, st_s, mk, qf, qs, zero4, sc);
+      if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
+      else block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
       // The warps of the team each hold the scores over their own channels: exchange and add them in a fixed
       // order, so that every warp of the team continues with bit-identical scores.  The barrier of
       // iteration k also tells that every warp is done with the slot of iteration k - 1, which is refilled
@@ -562,8 +690,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     // Copies of this team may still be in flight into its ring: give each a bounded time to land before
     // the block reuses the memory, then report.  The partial written below is not valid in that case.
     for (int s = 0; s < Cf::NST; ++s) {
-      int spins = 0;
-      while (!mbar_try_wait(bars + 8 * s, 0) && !mbar_try_wait(bars + 8 * s, 1) && ++spins < kMaxSpins) {}
+      const long long t0 = clock64();
+      while (!mbar_try_wait(bars + 8 * s, 0) && !mbar_try_wait(bars + 8 * s, 1) && clock64() - t0 < kMaxWaitCycles) {}
     }
     if (lane == 0 && status) atomicOr(status, TQ_STATUS_TIMEOUT);
   }
