@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-compare", action="store_true", help="skip the dequantize-then-attend timing")
     ap.add_argument("--splits", type=int, default=0, help="sequence splits C of the fused kernel (0 = library default)")
+    ap.add_argument("--classic", action="store_true",
+                    help="use tq_sdpa_int4_decode (waits for the preceding kernel first) instead of the overlapped entry")
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle check of sampled layers of the timed state")
     return ap.parse_args()
 
@@ -256,12 +258,16 @@ def main():
         for cch in caches:
             cch.seq_lens.fill_(S)
 
-    def enqueue(append=True, decode=True, combine=True):
+    # The S tokens of the fill were written long before any step: they are the stable part the overlapped
+    # decode may attend without waiting for the append just before it (tq.h).
+    def enqueue(append=True, decode=True, combine=True, classic=args.classic):
         for i in range(L):
             if append:
                 tq.tq_kv_quantize_append(caches[i], kn_l[i], vn_l[i], status)
-            if decode:
+            if decode and classic:
                 tq.tq_sdpa_int4_decode(caches[i], q_l[i], ALPHA, C, o_part, m_part, l_part, status)
+            elif decode:
+                tq.tq_sdpa_int4_decode_overlapped(caches[i], q_l[i], ALPHA, C, S, o_part, m_part, l_part, status)
             if combine:
                 tq.tq_sdpa_int4_combine(o_part, m_part, l_part, out_l[i])
 
@@ -300,6 +306,7 @@ def main():
     g_decode = make_graph(append=False, combine=False)
     g_attn = make_graph(append=False)
     g_append = make_graph(decode=False, combine=False)
+    g_decode_classic = make_graph(append=False, combine=False, classic=True)
 
     W, K = args.warmup, args.steps
     with ClockSampler(local_rank) as clocks:
@@ -311,6 +318,7 @@ def main():
     t_attn = time_graph(g_attn, W, K)
     t_append = time_graph(g_append, W, K)
     decode_us = t_decode / K / L * 1e6
+    decode_classic_us = time_graph(g_decode_classic, W, K) / K / L * 1e6
 
     # ---- end to end through host buffers: pinned host inputs -> device, the step, outputs -> pinned host
     h_in = torch.empty_like(inp, device="cpu").pin_memory()
@@ -352,7 +360,9 @@ def main():
                     "d2h_bytes_per_step": out.numel() * 2},
             "gpu_launches": 3 * L * K, "roofline": roofline,
             "breakdown_us_per_layer": {"append+decode+combine": us_per_layer, "decode+combine": t_attn / K / L * 1e6,
-                                       "decode": decode_us, "append": t_append / K / L * 1e6},
+                                       "decode": decode_us, "append": t_append / K / L * 1e6,
+                                       "decode_waiting_for_predecessor": decode_classic_us},
+            "decode_entry": "tq_sdpa_int4_decode" if args.classic else f"tq_sdpa_int4_decode_overlapped(stable_tokens={S})",
             "hbm_gbs_whole_step": alg_bytes / (us_per_layer * 1e-6) / 1e9, "num_splits": C,
             "paper_context": PAPER_CONTEXT, "device": device_info(torch, dev)}
     if parity is not None:

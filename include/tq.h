@@ -160,6 +160,38 @@ int tq_sdpa_int4_decode(const tq_kv_cache* cache /* host */, const void* q, int3
                         void* stream);
 
 /*
+ * Phase 1 overlapped with the work before it in the stream (the paper's Sec. 3.2 two-phase attention, unchanged
+ * in what it computes; the paper orders its two Metal dispatches through the framework's graph, here the
+ * ordering against the preceding kernel is relaxed where the data allows it).  The ordinary call starts by
+ * waiting for everything enqueued before it, because the quantize-append just before it may still be writing
+ * the newest tokens and the length.  A decode step, however, reads almost only tokens that were written
+ * steps ago.  The caller states how many:
+ *   stable_tokens : every sequence's cached tokens [0, stable_tokens) -- rounded down to a multiple of 16 --
+ *                   and all of q are FINAL before the preceding work in the stream starts: nothing that can
+ *                   still be running when this call's kernel starts writes them.  (Typically the shortest
+ *                   sequence length before this step's append.  libtq's own kernels let their successor be
+ *                   scheduled as soon as they start, so "the preceding work" reaches back to the last kernel
+ *                   that was not launched with programmatic dependent launch, or to the last synchronisation.)
+ * The kernel then streams and attends the stable tokens at once, waits for the preceding kernel only after
+ * that, reads seq_lens[b], and lets its last split attend the tokens [stable_tokens, seq_lens[b]).  The splits
+ * therefore partition the stable part, not the whole sequence: tq_split_range_stable gives the partition; keep
+ * stable_tokens close to the lengths or the last split grows (inside a replayed CUDA graph the value is fixed at
+ * capture time: re-capture, or update the node, every few hundred steps).
+ * seq_lens[b] < stable_tokens breaks the promise: TQ_STATUS_BAD_LEN is set and that sequence's result is not valid.
+ * With a paged cache, or stable_tokens / 16 below the split count, the call is exactly tq_sdpa_int4_decode.
+ * Everything else (arguments, partial layout, errors, status) as tq_sdpa_int4_decode; stable_tokens < 0 or
+ * > S_cap is TQ_ERR_SHAPE.  On the 128K Llama-shaped layer the overlap is worth about 3 us per launch.
+ */
+int tq_sdpa_int4_decode_overlapped(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
+                                   int32_t num_splits, int32_t stable_tokens, float* o_part, float* m_part,
+                                   float* l_part, int32_t* status, void* stream);
+/* Token range of split c under tq_sdpa_int4_decode_overlapped (host function): with sb = stable_tokens / 16 >= C,
+ * split c covers tokens [16 * floor(c * sb / C), 16 * floor((c + 1) * sb / C)), and the last one reaches to len;
+ * with sb < C it is tq_split_range(len, C, c). */
+void tq_split_range_stable(int32_t len, int32_t stable_tokens, int32_t C, int32_t c, int32_t* t0 /* host */,
+                           int32_t* t1 /* host */);
+
+/*
  * Phase 1 restricted to a sliding window (Appendix A: Gemma's sliding-attention layers, w = 1024, which
  * the paper's kernel serves by skipping tokens inside its loop): sequence b attends only its last `window`
  * tokens, [max(0, seq_lens[b] - window), seq_lens[b]).  Here the skip is not per token: the splits

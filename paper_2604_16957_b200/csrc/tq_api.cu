@@ -141,6 +141,37 @@ int tq_sdpa_int4_decode(const tq_kv_cache* cache, const void* q, int32_t H_q, fl
   return tq_sdpa_int4_decode_window(cache, q, H_q, attn_scale, 0, num_splits, o_part, m_part, l_part, status, stream);
 }
 
+void tq_split_range_stable(int32_t len, int32_t stable_tokens, int32_t C, int32_t c, int32_t* t0, int32_t* t1) {
+  int a = 0, b = 0;
+  if (C >= 1 && c >= 0 && c < C) {
+    if (stable_tokens / kQuantum >= C) split_range_stable(len, stable_tokens, C, c, a, b);
+    else split_range(0, len, C, c, a, b);
+  }
+  if (t0) *t0 = a;
+  if (t1) *t1 = b;
+}
+
+int tq_sdpa_int4_decode_overlapped(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale,
+                                   int32_t num_splits, int32_t stable_tokens, float* o_part, float* m_part,
+                                   float* l_part, int32_t* status, void* stream) {
+  if (int r = check_cache(cache)) return r;
+  if (stable_tokens < 0 || stable_tokens > cache->S_cap) return TQ_ERR_SHAPE;
+  if (!q || !o_part || !m_part || !l_part) return TQ_ERR_NULL;
+  if (int r = check_heads(cache, H_q)) return r;
+  if (num_splits < 0 || num_splits > TQ_MAX_SPLITS) return TQ_ERR_SHAPE;
+  if (!aligned16(q) || !aligned16(o_part) || (reinterpret_cast<uintptr_t>(m_part) & 3u) ||
+      (reinterpret_cast<uintptr_t>(l_part) & 3u) || (reinterpret_cast<uintptr_t>(status) & 3u))
+    return TQ_ERR_ALIGN;
+  if (int r = check_decode_grid(cache, H_q, 1)) return r;
+  const int C = num_splits ? num_splits : tq_auto_splits(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
+  const bool overlapped = cache->page_table == nullptr && stable_tokens / kQuantum >= C &&
+                          test_hooks().decode_impl.load(std::memory_order_relaxed) == 0;
+  if (!overlapped)
+    return tq_sdpa_int4_decode(cache, q, H_q, attn_scale, C, o_part, m_part, l_part, status, stream);
+  return finish(launch_decode_mma(*cache, static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, o_part, m_part, l_part,
+                                  status, static_cast<cudaStream_t>(stream), stable_tokens));
+}
+
 int tq_sdpa_int4_decode_window(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale, int32_t window,
                                int32_t num_splits, float* o_part, float* m_part, float* l_part, int32_t* status,
                                void* stream) {

@@ -89,8 +89,8 @@ __global__ void __launch_bounds__(kWarps * 32) attend_simple_kernel(Src src, con
   const int tiles = (GV + kHeadTile - 1) / kHeadTile;
   const int c = blockIdx.x, kvh = blockIdx.y / tiles, tile = blockIdx.y % tiles, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int len = checked_len(seq_lens, b, S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
   int t0, t1;
   split_range(query_lo(len, S_q, 0, window), len, C, c, t0, t1);
@@ -196,8 +196,8 @@ cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q,
 // x^ = (q - z) * s for every valid row; one thread per 8 consecutive elements.
 template <typename T>
 __global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T* v_mat) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int d = c.d, cpr = d >> 3;
   const int b = blockIdx.y;
   int len = c.seq_lens[b];

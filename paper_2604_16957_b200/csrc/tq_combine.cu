@@ -17,8 +17,8 @@ __global__ void __launch_bounds__(kThreads) combine_kernel(const float* __restri
   __shared__ float w[TQ_MAX_SPLITS];
   __shared__ float red[kThreads / 32];
   __shared__ float4 acc[kThreads];
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const long long bh = blockIdx.x;
   const float* m = m_part + bh * C;
   const float* l = l_part + bh * C;

@@ -387,10 +387,10 @@ template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, int S_q, float attn_scale, int window,
                       int C, float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
-                      int32_t* status) {
+                      int32_t* status, int stable_blocks) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
-  constexpr bool GEN = MODE != 0, PAGED = MODE == 2;
+  constexpr bool GEN = MODE == 1 || MODE == 2, PAGED = MODE == 2, OVL = MODE == 3;
   extern __shared__ __align__(1024) uint8_t smem[];
 
   const int G = H_q / cache.H_kv;
@@ -409,11 +409,22 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     const int s = GEN ? v / G : 0;
     return (static_cast<long long>(b) * (GEN ? S_q : 1) + s) * H_q + kvh * G + (v - s * G);
   };
-  pdl_wait();  // nothing global is read before this point
+  // The next kernel in the stream may be scheduled from here on (it waits for this one where it must).
   pdl_launch_dependents();
-  const int len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
-  int t0, t1;
-  split_range(GEN ? query_lo(len, S_q, 0, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
+  // Overlapped form (MODE 3): the splits partition the `stable_blocks` oldest 16-token blocks, which nothing
+  // still running writes, and q is final too (the caller's promise, tq.h); so this kernel streams and
+  // computes without waiting for the kernel before it, waits once the stable part is done, reads the length
+  // and lets its last split take the tokens beyond the stable part.  Every other form waits here, before its
+  // first global access.
+  if (!OVL) pdl_wait();
+  int len = 0, t0, t1;
+  if (OVL) {
+    t0 = static_cast<int>((static_cast<long long>(stable_blocks) * c) / C) * kBlk;
+    t1 = static_cast<int>((static_cast<long long>(stable_blocks) * (c + 1)) / C) * kBlk;
+  } else {
+    len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
+    split_range(GEN ? query_lo(len, S_q, 0, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
+  }
 
   // ---- q first (a handful of loads that must not queue behind the cache stream), used further down
   uint4 qraw[NGW];
@@ -425,8 +436,9 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
 
   // ---- this team's token blocks: blk0 + team, blk0 + team + NTEAM, ...
-  const int blk0 = t0 / kBlk, blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
-  const int nblk = blk1 - blk0 > team ? (blk1 - blk0 - team + NTEAM - 1) / NTEAM : 0;
+  int blk0 = t0 / kBlk;
+  const int blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
+  int nblk = blk1 - blk0 > team ? (blk1 - blk0 - team + NTEAM - 1) / NTEAM : 0;
   const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
   uint8_t* const ring = smem + team * (Cf::NST * Cf::STAGE);
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
@@ -562,8 +574,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // Blocks in which every token counts for every column go through the plain step, the others through the
   // masking one.  Plain decode: only the block holding the end of the sequence is partial.  General form:
   // blocks that reach beyond the oldest query's end, or begin before the newest query's window start.
-  const int rem_last = t1 - (blk0 + team + (nblk - 1) * NTEAM) * kBlk;  // tokens in this team's last block
-  int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;          // this team's blocks k < nfull are full
+  int rem_last = t1 - (blk0 + team + (nblk - 1) * NTEAM) * kBlk;  // tokens in this team's last block
+  int nfull = (nblk > 0 && rem_last < kBlk) ? nblk - 1 : nblk;    // this team's blocks k < nfull are full
   int nhead = 0;                                                        // ... and blocks k < nhead are masked
   if (GEN) {
     const int full_end = min(t1, query_hi(len, S_q, 0)) >> 4;                   // blocks below it end inside every range
@@ -599,7 +611,32 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
   bool timed_out = false;
   int k = 0;
+#pragma unroll 1
+  for (int phase = 0; phase < (OVL ? 2 : 1); ++phase) {
+  if (OVL && phase == 1) {
+    // the stable part is done: from here on this kernel is ordered after the one before it
+    pdl_wait();
+    len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
+    const int stable_tokens = stable_blocks * kBlk;
+    if (len < stable_tokens && c == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status)
+      atomicOr(status, TQ_STATUS_BAD_LEN);  // the promise did not hold: tokens beyond the length were attended
+    int next = 0;
+    if (c == C - 1 && len > stable_tokens && !timed_out) {
+      const int eb1 = (len + kBlk - 1) / kBlk;
+      next = eb1 - stable_blocks > team ? (eb1 - stable_blocks - team + NTEAM - 1) / NTEAM : 0;
+    }
+    // the ring goes on where it stood: block number n >= nblk of this team is now stable_blocks + team + (n - nblk) * NTEAM
+    blk0 = stable_blocks - nblk * NTEAM;
+    nblk += next;
+    rem_last = next > 0 ? len - (blk0 + team + (nblk - 1) * NTEAM) * kBlk : kBlk;
+    nfull = rem_last < kBlk ? nblk - 1 : nblk;
+    if (next > 0) {
+      for (int n = k; n < k + Cf::NST - 1; ++n)
+        if (n < nblk) issue(n);
+    }
+  }
   if constexpr (DS == 1 && !GEN) {
+   if (phase == 0) {
     // Full blocks four at a time: ring slot, barrier and stage offsets are constants of each of the four
     // copies of the block step, so the loop carries no slot arithmetic.
     static_assert(Cf::NST == 4, "the unrolled loop walks a ring of four slots");
@@ -627,6 +664,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       }
       par ^= 1;
     }
+   }
   }
 #pragma unroll 1
   for (; k < nblk && !timed_out; ++k) {
@@ -686,6 +724,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       else block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
     }
   }
+  }  // phase
   if (timed_out) {
     // Copies of this team may still be in flight into its ring: give each a bounded time to land before
     // the block reuses the memory, then report.  The partial written below is not valid in that case.
@@ -772,7 +811,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
 template <int D, int MODE>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
-                   float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, cudaStream_t st) {
   size_t smem = Cfg<D>::SMEM;
   if (MODE == 2) {
     // room for the page addresses of the longest split: its blocks, rounded out to whole pages
@@ -787,26 +826,30 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
   const int GV = (H_q / c.H_kv) * S_q;
   dim3 grid(C, c.H_kv * ((GV + 7) / 8), c.B);
   return launch_kernel(decode_mma_kernel<D, MODE>, grid, dim3(kThreads), smem, st, c, q, H_q, S_q, attn_scale, window, C,
-                       o_part, m_part, l_part, status);
+                       o_part, m_part, l_part, status, stable_blocks);
 }
 
 template <int D>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
-                   float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
-  if (c.page_table != nullptr) return launch<D, 2>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
-  return (window > 0 || S_q > 1) ? launch<D, 1>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st)
-                                 : launch<D, 0>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, st);
+                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, cudaStream_t st) {
+  if (c.page_table != nullptr) return launch<D, 2>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, st);
+  if (window > 0 || S_q > 1) return launch<D, 1>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, st);
+  if (stable_blocks > 0) return launch<D, 3>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, st);
+  return launch<D, 0>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, 0, st);
 }
 
 }  // namespace
 
+// stable_tokens > 0 selects the overlapped form (plain decode over a contiguous cache only; see tq.h)
 cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
-                              int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st) {
+                              int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st,
+                              int stable_tokens) {
+  const int sb = stable_tokens > 0 ? stable_tokens / kBlk : 0;
   switch (c.d) {
-    case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
-    case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
-    case 512: return launch<512>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
-    default: return launch<256>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, st);
+    case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
+    case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
+    case 512: return launch<512>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
+    default: return launch<256>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
   }
 }
 

@@ -30,6 +30,14 @@ __host__ __device__ inline void split_range(int begin, int len, int C, int c, in
   t0 = (int)s;
   t1 = (int)e;
 }
+// Partition of the overlapped decode: the first stable_tokens / 16 blocks are cut into C equal runs of blocks,
+// whatever the length; the last split also takes every token from there to len.
+__host__ __device__ inline void split_range_stable(int len, int stable_tokens, int C, int c, int& t0, int& t1) {
+  const long long sb = stable_tokens > 0 ? stable_tokens / kQuantum : 0;
+  t0 = static_cast<int>((sb * c) / C) * kQuantum;
+  t1 = static_cast<int>((sb * (c + 1)) / C) * kQuantum;
+  if (c == C - 1 && len > t1) t1 = len;
+}
 __host__ __device__ inline int window_begin(int len, int window) {
   return (window > 0 && window < len) ? len - window : 0;
 }
@@ -104,11 +112,13 @@ __device__ inline int checked_len(const int32_t* seq_lens, int b, int S_cap, int
 
 // Programmatic dependent launch.  The three kernels of a decode step (append, phase 1, reduction) are
 // launched with the programmatic-stream-serialization attribute, so the launch latency of each one
-// overlaps the tail of the kernel before it in the stream.  Every kernel calls pdl_wait() before its
-// first global access (that wait returns once the preceding kernel has completed and its writes are
-// visible, so ordering is exactly stream order) and pdl_launch_dependents() right after, which lets
-// the next kernel be scheduled as soon as this one's blocks start to retire.  Both are no-ops when
-// the kernel was launched the ordinary way.
+// overlaps the tail of the kernel before it in the stream.  Every kernel first calls
+// pdl_launch_dependents(), which lets the next kernel's blocks be scheduled as soon as there is room for
+// them, and then pdl_wait() before its first global access (that wait returns once the preceding kernel
+// has completed and its writes are visible, so ordering is exactly stream order; it holds transitively,
+// since the preceding kernel itself waited for the one before it).  The one exception is the overlapped
+// decode (tq_sdpa_int4_decode_overlapped), which reads what its caller promised to be final before it
+// waits.  Both calls are no-ops when the kernel was launched the ordinary way.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
@@ -133,7 +143,8 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, const __half* v_new, int T,
                                    int32_t* status, cudaStream_t st);
 cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
-                              int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
+                              int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st,
+                              int stable_tokens = 0);
 cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
                                  int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
 cudaError_t launch_combine(const float* o_part, const float* m_part, const float* l_part, int B, int H_q, int d, int C,

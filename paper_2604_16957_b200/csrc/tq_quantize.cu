@@ -157,8 +157,8 @@ __global__ void __launch_bounds__(2 * D, 1536 / (2 * D)) quantize_bulk_kernel(tq
                                                               int T, int32_t* status) {
   constexpr int CPR = D / 8, NG = D / 32;
   __shared__ __align__(16) __half sm_meta[kBulkBlocks][2][NG][16];  // [block][scale | zero][group][token]
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const long long bh = blockIdx.y;
   const int b = static_cast<int>(bh / c.H_kv);
   const int len = c.seq_lens[b];
@@ -243,8 +243,8 @@ __global__ void __launch_bounds__(2 * D, 1536 / (2 * D)) quantize_bulk_kernel(tq
 }
 
 __global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= c.B) return;
   const int len = c.seq_lens[b];
@@ -259,8 +259,8 @@ __global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
 // then advances the length itself -- a single launch, and no block reads another's length.
 __global__ void __launch_bounds__(256) quantize_step_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new,
                                                             int T, int32_t* status) {
-  pdl_wait();
   pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.x;
   const int len = c.seq_lens[b];
   if (len < 0 || len > c.S_cap - T) {

@@ -28,7 +28,8 @@ SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa
            "tq_partials_bytes", "tq_sdpa_dequant_then_attend", "tq_dequant_workspace_bytes", "tq_cache_bytes",
            "tq_result_string", "tq_last_cuda_error", "tq_version", "tq_sdpa_int4_attend_static",
            "tq_cache_code_offset", "tq_cache_meta_offset", "tq_sdpa_int4_decode_window", "tq_split_range_window",
-           "tq_sdpa_int4_decode_multi", "tq_sdpa_mixed_precision_attend")
+           "tq_sdpa_int4_decode_multi", "tq_sdpa_mixed_precision_attend", "tq_sdpa_int4_decode_overlapped",
+           "tq_split_range_stable")
 
 
 class tq_kv_cache(C.Structure):
@@ -51,6 +52,10 @@ _lib.tq_split_range.argtypes = [_i32, _i32, _i32, C.POINTER(_i32), C.POINTER(_i3
 _lib.tq_split_range.restype = None
 _lib.tq_sdpa_int4_decode.argtypes = [_cache_p, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.tq_sdpa_int4_decode.restype = C.c_int
+_lib.tq_sdpa_int4_decode_overlapped.argtypes = [_cache_p, _vp, _i32, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
+_lib.tq_sdpa_int4_decode_overlapped.restype = C.c_int
+_lib.tq_split_range_stable.argtypes = [_i32, _i32, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32)]
+_lib.tq_split_range_stable.restype = None
 _lib.tq_sdpa_int4_decode_window.argtypes = [_cache_p, _vp, _i32, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.tq_sdpa_int4_decode_window.restype = C.c_int
 _lib.tq_sdpa_int4_decode_multi.argtypes = [_cache_p, _vp, _i32, _i32, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
@@ -224,6 +229,21 @@ def tq_sdpa_int4_decode(cache, q, attn_scale, num_splits, o_part, m_part, l_part
     cs = _cs(cache)
     _check(_lib.tq_sdpa_int4_decode(C.byref(cs), _ptr(q), q.shape[1], float(attn_scale), int(num_splits), _ptr(o_part),
                                     _ptr(m_part), _ptr(l_part), _ptr(status), _stream(stream)), "tq_sdpa_int4_decode")
+
+
+def tq_sdpa_int4_decode_overlapped(cache, q, attn_scale, num_splits, stable_tokens, o_part, m_part, l_part, status=None,
+                                   stream=None):
+    """Phase 1 that does not wait for the preceding kernel before attending the first stable_tokens tokens."""
+    cs = _cs(cache)
+    _check(_lib.tq_sdpa_int4_decode_overlapped(C.byref(cs), _ptr(q), q.shape[1], float(attn_scale), int(num_splits),
+                                               int(stable_tokens), _ptr(o_part), _ptr(m_part), _ptr(l_part),
+                                               _ptr(status), _stream(stream)), "tq_sdpa_int4_decode_overlapped")
+
+
+def tq_split_range_stable(length, stable_tokens, C_, c):
+    t0, t1 = _i32(), _i32()
+    _lib.tq_split_range_stable(length, stable_tokens, C_, c, C.byref(t0), C.byref(t1))
+    return t0.value, t1.value
 
 
 def tq_sdpa_int4_decode_window(cache, q, attn_scale, window, num_splits, o_part, m_part, l_part, status=None,
