@@ -45,7 +45,7 @@ def parse_args():
     ap.add_argument("--no-compare", action="store_true", help="skip the dequantize-then-attend timing")
     ap.add_argument("--splits", type=int, default=0, help="sequence splits C of the fused kernel (0 = library default)")
     ap.add_argument("--classic", action="store_true",
-                    help="use tq_sdpa_int4_decode (waits for the preceding kernel first) instead of the overlapped entry")
+                    help="time the step as three calls (append, tq_sdpa_int4_decode, combine) instead of the fused step")
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle check of sampled layers of the timed state")
     return ap.parse_args()
 
@@ -171,7 +171,7 @@ def run_reference(args, rank):
 def config_dict(args):
     return {"workload": f"llama70b-shape long context: B=1, H_q={H_Q}, H_kv={H_KV}, d={D}, context={args.context}, "
                         f"{args.layers} layers resident, int4 KV group 32, attn_scale=1/sqrt(d), one decode step "
-                        f"layer by layer (quantize-append + fused int4 attention + split combine)",
+                        f"layer by layer (quantize-append + fused int4 attention + split combine per layer)",
             "context": args.context, "layers": args.layers, "H_q": H_Q, "H_kv": H_KV, "d": D,
             "l2": "inputs larger than L2: every layer's cache (168 MB at 128K) is a distinct buffer, 13.4 GB in all"}
 
@@ -214,7 +214,7 @@ def main():
     L, S = args.layers, args.context
     total_appends = 2 * (args.warmup + args.steps) + 8
     S_cap = (S + total_appends + 15) // 16 * 16
-    C = args.splits or tq.tq_auto_splits(1, H_KV, H_Q, D, S)
+    C = args.splits or (tq.tq_auto_splits if args.classic else tq.tq_auto_splits_step)(1, H_KV, H_Q, D, S)
 
     # ---- resident state: L quantised layer caches, filled from seeded device-side normals.
     # K gets 4 seeded outlier channels x10 per KV head, like the parity-test generator.
@@ -258,10 +258,16 @@ def main():
         for cch in caches:
             cch.seq_lens.fill_(S)
 
-    # The S tokens of the fill were written long before any step: they are the stable part the overlapped
-    # decode may attend without waiting for the append just before it (tq.h).
+    # The S tokens of the fill were written long before any step: they are the stable part that the fused
+    # step / the overlapped decode may attend without waiting for the kernel before it (tq.h).
+    ws = tq.alloc_step_workspace(1, H_KV, H_Q, D, C, device=dev)
+
     def enqueue(append=True, decode=True, combine=True, classic=args.classic):
+        fused = append and decode and combine and not classic
         for i in range(L):
+            if fused:   # one launch: quantize-append + fused int4 attention + split reduction
+                tq.tq_sdpa_int4_step(caches[i], kn_l[i], vn_l[i], q_l[i], ALPHA, C, S, ws, out_l[i], status)
+                continue
             if append:
                 tq.tq_kv_quantize_append(caches[i], kn_l[i], vn_l[i], status)
             if decode and classic:
@@ -307,6 +313,7 @@ def main():
     g_attn = make_graph(append=False)
     g_append = make_graph(decode=False, combine=False)
     g_decode_classic = make_graph(append=False, combine=False, classic=True)
+    g_three = make_graph(classic=True)
 
     W, K = args.warmup, args.steps
     with ClockSampler(local_rank) as clocks:
@@ -319,6 +326,7 @@ def main():
     t_append = time_graph(g_append, W, K)
     decode_us = t_decode / K / L * 1e6
     decode_classic_us = time_graph(g_decode_classic, W, K) / K / L * 1e6
+    three_us = time_graph(g_three, W, K) / K / L * 1e6
 
     # ---- end to end through host buffers: pinned host inputs -> device, the step, outputs -> pinned host
     h_in = torch.empty_like(inp, device="cpu").pin_memory()
@@ -346,10 +354,14 @@ def main():
     # ---- roofline of the dominant kernel (fused decode)
     peak, peak_src = measured_peak()
     alg_bytes = H_KV * S * BYTES_PER_TOKEN_HEAD
-    achieved = alg_bytes / (decode_us * 1e-6) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_mma_kernel<128>", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    # the timed step is one launch of the fused kernel per layer, so its per-layer time is that kernel's average
+    # launch-to-launch duration; with --classic the fused-attention kernel is timed in a graph of its own
+    kernel_us = decode_classic_us if args.classic else us_per_layer
+    achieved = alg_bytes / (kernel_us * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_mma_kernel<128, 0>" if args.classic else
+                "decode_mma_kernel<128, 3> (append + attention + reduction in one launch)", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src, "traffic": ncu_traffic_bytes() if S == CONTEXT else None,
-                "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": decode_us,
+                "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": kernel_us,
                 "frac_of_nominal_8TBs": achieved / HBM_NOMINAL_GBS}
 
     line = {"metric": "int4 decode-attn us/layer @128K (Llama-70B shape)", "value": job_us_per_layer(t_step, K, L, world),
@@ -358,11 +370,13 @@ def main():
             "data": "synthetic", "config": config_dict(args), "clocks": clocks.summary(),
             "e2e": {"value": e2e_us / world, "unit": "us/layer", "h2d_bytes_per_step": inp.numel() * 2,
                     "d2h_bytes_per_step": out.numel() * 2},
-            "gpu_launches": 3 * L * K, "roofline": roofline,
+            "gpu_launches": (3 if args.classic else 1) * L * K, "roofline": roofline,
             "breakdown_us_per_layer": {"append+decode+combine": us_per_layer, "decode+combine": t_attn / K / L * 1e6,
                                        "decode": decode_us, "append": t_append / K / L * 1e6,
-                                       "decode_waiting_for_predecessor": decode_classic_us},
-            "decode_entry": "tq_sdpa_int4_decode" if args.classic else f"tq_sdpa_int4_decode_overlapped(stable_tokens={S})",
+                                       "decode_waiting_for_predecessor": decode_classic_us,
+                                       "append+decode+combine as three calls": three_us},
+            "step_entry": ("tq_kv_quantize_append + tq_sdpa_int4_decode + tq_sdpa_int4_combine" if args.classic else
+                           f"tq_sdpa_int4_step(stable_tokens={S}): one launch per layer"),
             "hbm_gbs_whole_step": alg_bytes / (us_per_layer * 1e-6) / 1e9, "num_splits": C,
             "paper_context": PAPER_CONTEXT, "device": device_info(torch, dev)}
     if parity is not None:

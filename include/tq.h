@@ -179,6 +179,7 @@ int tq_sdpa_int4_decode(const tq_kv_cache* cache /* host */, const void* q, int3
  * capture time: re-capture, or update the node, every few hundred steps).
  * seq_lens[b] < stable_tokens breaks the promise: TQ_STATUS_BAD_LEN is set and that sequence's result is not valid.
  * With a paged cache, or stable_tokens / 16 below the split count, the call is exactly tq_sdpa_int4_decode.
+ * num_splits = 0 picks tq_auto_splits_step(B, H_kv, H_q, d, S_cap).
  * Everything else (arguments, partial layout, errors, status) as tq_sdpa_int4_decode; stable_tokens < 0 or
  * > S_cap is TQ_ERR_SHAPE.  On the 128K Llama-shaped layer the overlap is worth about 3 us per launch.
  */
@@ -190,6 +191,43 @@ int tq_sdpa_int4_decode_overlapped(const tq_kv_cache* cache /* host */, const vo
  * with sb < C it is tq_split_range(len, C, c). */
 void tq_split_range_stable(int32_t len, int32_t stable_tokens, int32_t C, int32_t c, int32_t* t0 /* host */,
                            int32_t* t1 /* host */);
+
+/*
+ * One decode step of one layer in a single launch: the quantize-append of the new token (Sec. 2.1), the fused
+ * int4 attention over the cache including it (Sec. 3.1, 3.2) and the reduction of Eq. 5.  The paper runs these as
+ * separate dispatches chained through its framework; here one kernel does all three, so a step costs one
+ * launch (what short contexts are made of) and consecutive layers' steps follow each other without the two
+ * hand-overs in between.  The result is that of tq_kv_quantize_append (T = 1), tq_sdpa_int4_decode_overlapped
+ * and tq_sdpa_int4_combine called in that order, up to the summation order of the reduction.
+ *   k_new, v_new : [B][H_kv][1][d] fp16, or both NULL for a step that appends nothing.  The row of KV head h is
+ *                  quantised by the thread block of that head's last split, written to the cache, and read
+ *                  back by the same block; seq_lens[b] is advanced by the last block of the sequence to have
+ *                  read the old value.  A full cache sets TQ_STATUS_CACHE_FULL and attends the old tokens only.
+ *   stable_tokens: as in tq_sdpa_int4_decode_overlapped (the promise covers q and the first stable_tokens cached
+ *                  tokens; k_new / v_new are read after the wait for the preceding kernel).  0 or a value below
+ *                  16 * C: nothing is read early and the splits partition the whole sequence.
+ *   workspace    : tq_step_workspace_bytes(...) bytes, 16-byte aligned: counters, then the split partials.
+ *                  ZERO the first tq_step_counter_bytes(B, H_kv) bytes once before the first use (cudaMemsetAsync);
+ *                  every launch leaves them zero again.  After a TQ_STATUS_TIMEOUT zero them again.  Launches that may
+ *                  overlap on the GPU (other streams) need workspaces of their own.
+ *   out          : [B][H_q][d] fp16 or fp32, written by the last thread block of each (sequence, KV head) to finish.
+ *   num_splits   : C >= 1, or 0 for tq_auto_splits_step(B, H_kv, H_q, d, S_cap).
+ * Restrictions: contiguous cache (page_table == NULL) and H_q / H_kv <= 8; otherwise TQ_ERR_SHAPE -- use the three
+ * calls.  Errors: TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_WORKSPACE, TQ_ERR_CUDA.  Status as the three calls.
+ */
+int tq_sdpa_int4_step(const tq_kv_cache* cache /* host */, const void* k_new, const void* v_new, const void* q,
+                      int32_t H_q, float attn_scale, int32_t num_splits, int32_t stable_tokens, void* workspace,
+                      size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream);
+size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t num_splits);
+/*
+ * Split count that tq_sdpa_int4_step and tq_sdpa_int4_decode_overlapped pick for num_splits = 0 (host function).
+ * Like tq_auto_splits, but when one wave of thread blocks fills the GPU it leaves one resident slot per
+ * (sequence, KV head) unused: launches of these entry points overlap their predecessor, and with every slot
+ * taken the blocks that finish a launch last (those that also reduce the partials) hold up the first blocks
+ * of the next one.  Measured on the 128K Llama-shaped step: 36.5 us per layer with 37 splits, 32.3 us with 36.
+ */
+int32_t tq_auto_splits_step(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len);
+size_t tq_step_counter_bytes(int32_t B, int32_t H_kv);
 
 /*
  * Phase 1 restricted to a sliding window (Appendix A: Gemma's sliding-attention layers, w = 1024, which

@@ -125,6 +125,15 @@ int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t 
   return static_cast<int32_t>(C);
 }
 
+int32_t tq_auto_splits_step(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len) {
+  const int32_t C = tq_auto_splits(B, H_kv, H_q, d, max_seq_len);
+  if (B < 1 || H_kv < 1 || H_q < H_kv) return C;
+  const long long base = static_cast<long long>(B) * H_kv * ((H_q / H_kv + 7) / 8);
+  const long long slots = 2LL * device_sm_count();
+  // one wave that takes every slot: leave one per (sequence, KV head) to the stragglers of the launch before
+  return (4 * base <= slots && C > 1 && C * base > slots - base) ? C - 1 : C;
+}
+
 void tq_split_range(int32_t len, int32_t C, int32_t c, int32_t* t0, int32_t* t1) {
   tq_split_range_window(len, 0, C, c, t0, t1);
 }
@@ -163,13 +172,48 @@ int tq_sdpa_int4_decode_overlapped(const tq_kv_cache* cache, const void* q, int3
       (reinterpret_cast<uintptr_t>(l_part) & 3u) || (reinterpret_cast<uintptr_t>(status) & 3u))
     return TQ_ERR_ALIGN;
   if (int r = check_decode_grid(cache, H_q, 1)) return r;
-  const int C = num_splits ? num_splits : tq_auto_splits(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
+  const int C = num_splits ? num_splits : tq_auto_splits_step(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
   const bool overlapped = cache->page_table == nullptr && stable_tokens / kQuantum >= C &&
                           test_hooks().decode_impl.load(std::memory_order_relaxed) == 0;
   if (!overlapped)
     return tq_sdpa_int4_decode(cache, q, H_q, attn_scale, C, o_part, m_part, l_part, status, stream);
   return finish(launch_decode_mma(*cache, static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, o_part, m_part, l_part,
                                   status, static_cast<cudaStream_t>(stream), stable_tokens));
+}
+
+size_t tq_step_counter_bytes(int32_t B, int32_t H_kv) {
+  if (B < 1 || H_kv < 1) return 0;
+  return align256((static_cast<size_t>(B) * H_kv + B) * sizeof(int32_t));
+}
+
+size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t num_splits) {
+  if (B < 1 || H_kv < 1 || H_q < 1 || d < 1 || num_splits < 1) return 0;
+  return tq_step_counter_bytes(B, H_kv) + tq_partials_bytes(B, H_q, d, num_splits);
+}
+
+int tq_sdpa_int4_step(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
+                      float attn_scale, int32_t num_splits, int32_t stable_tokens, void* workspace,
+                      size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
+  if (int r = check_cache(cache)) return r;
+  if (!q || !workspace || !out || ((k_new == nullptr) != (v_new == nullptr))) return TQ_ERR_NULL;
+  if (int r = check_heads(cache, H_q)) return r;
+  if (cache->page_table != nullptr || H_q / cache->H_kv > 8) return TQ_ERR_SHAPE;
+  if (stable_tokens < 0 || stable_tokens > cache->S_cap || num_splits < 0 || num_splits > TQ_MAX_SPLITS) return TQ_ERR_SHAPE;
+  if (!aligned16(q) || !aligned16(workspace) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new) ||
+      (reinterpret_cast<uintptr_t>(status) & 3u))
+    return TQ_ERR_ALIGN;
+  const int C = num_splits ? num_splits : tq_auto_splits_step(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
+  if (workspace_bytes < tq_step_workspace_bytes(cache->B, cache->H_kv, H_q, cache->d, C)) return TQ_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(workspace);
+  int32_t* counters = reinterpret_cast<int32_t*>(ws);
+  const size_t n = static_cast<size_t>(cache->B) * H_q * C;
+  float* o_part = reinterpret_cast<float*>(ws + tq_step_counter_bytes(cache->B, cache->H_kv));
+  float* m_part = reinterpret_cast<float*>(reinterpret_cast<char*>(o_part) + align256(n * cache->d * sizeof(float)));
+  float* l_part = reinterpret_cast<float*>(reinterpret_cast<char*>(m_part) + align256(n * sizeof(float)));
+  const int stable = stable_tokens / kQuantum >= C ? stable_tokens : 0;
+  return finish(launch_decode_step(*cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new),
+                                   static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, stable, o_part, m_part, l_part,
+                                   counters, out, out_is_fp32 != 0, status, static_cast<cudaStream_t>(stream)));
 }
 
 int tq_sdpa_int4_decode_window(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale, int32_t window,

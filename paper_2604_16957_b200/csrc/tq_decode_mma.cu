@@ -42,6 +42,7 @@
 //      side by side: the token-pair interleave the P.V MMA needs (k = tokens), done by the
 //      load itself, so V needs no byte permutes.
 #include "tq_internal.cuh"
+#include "tq_quantize_core.cuh"
 
 namespace tq {
 namespace {
@@ -376,6 +377,15 @@ __device__ __forceinline__ bool wait_stage(uint32_t bar, uint32_t parity) {
   return wait_stage_slow(bar, parity);
 }
 
+// What the fused decode step (tq_sdpa_int4_step) adds to phase 1; all null for the plain calls.
+struct StepArgs {
+  const __half* k_new;  // [B][H_kv][1][D]: quantised and appended by the last split of each KV head (null: no append)
+  const __half* v_new;
+  void* out;            // [B][H_q][D]: written by the last block to finish of each (sequence, KV head) (null: no reduction)
+  int out_fp32;
+  int32_t* counters;    // [B * H_kv] arrivals, then [B] length readers; zero between launches
+};
+
 // GEN = the general form: a sliding window (Appendix A) and / or several query tokens per sequence
 // (S_q > 1, the grid's S_q factor in Appendix A).  With S_q query tokens the "heads" of a KV head are its
 // G * S_q (query token, head) pairs, v = s * G + g, packed into MMA columns like plain heads; query token s
@@ -387,7 +397,7 @@ template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, int S_q, float attn_scale, int window,
                       int C, float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
-                      int32_t* status, int stable_blocks) {
+                      int32_t* status, int stable_blocks, StepArgs sa) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
   constexpr bool GEN = MODE == 1 || MODE == 2, PAGED = MODE == 2, OVL = MODE == 3;
@@ -416,13 +426,66 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // computes without waiting for the kernel before it, waits once the stable part is done, reads the length
   // and lets its last split take the tokens beyond the stable part.  Every other form waits here, before its
   // first global access.
-  if (!OVL) pdl_wait();
+  const bool ovl = OVL && stable_blocks > 0;
+  if (!ovl) pdl_wait();
+  const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
+  const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
+  // The length of this sequence; in the fused step also the place where the new token is quantised and
+  // written (by the block of the last split of this KV head, which is the only one to read that row: it
+  // issues its copies of the newest blocks after this) and where the length is advanced (by whichever block
+  // of the sequence is the last to have read the old one).  Every block of the grid calls it once, after the
+  // wait for the preceding kernel.
+  auto read_len = [&]() -> int {
+    int n = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
+    if (OVL && sa.k_new != nullptr) {
+      const int old = n;
+      if (old < cache.S_cap) n = old + 1;
+      else if (c == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status) atomicOr(status, TQ_STATUS_CACHE_FULL);
+      if (c == C - 1 && n > old) {  // one head tile per KV head in this form (checked on the host)
+        if (warp == 0) {
+          uint8_t* const blk = const_cast<uint8_t*>(head_blocks) + static_cast<size_t>(old >> 4) * Cf::STAGE;
+          constexpr int CPR = D / 8;  // 8-element chunks per row; K chunks first, then V
+#pragma unroll
+          for (int i0 = 0; i0 < 2 * CPR; i0 += 32) {
+            const int i = i0 + lane;
+            const bool on = i < 2 * CPR;
+            const int which = i >= CPR ? 1 : 0, cc = i - which * CPR;
+            uint4 raw = make_uint4(0, 0, 0, 0);
+            if (on) raw = *reinterpret_cast<const uint4*>((which ? sa.v_new : sa.k_new) + (static_cast<long long>(b) * cache.H_kv + kvh) * D + cc * 8);
+            uint32_t word;
+            __half sq, zq;
+            quantize_chunk(raw, word, sq, zq);
+            if (on) {
+              *reinterpret_cast<uint32_t*>(blk + code_offset(D, which, old & 15, cc * 4)) = word;
+              if ((cc & 3) == 0) {
+                *reinterpret_cast<__half*>(blk + meta_offset(D, which, 0, cc >> 2, old & 15)) = sq;
+                *reinterpret_cast<__half*>(blk + meta_offset(D, which, 1, cc >> 2, old & 15)) = zq;
+              }
+            }
+          }
+          // the row is fetched back by this block's bulk copies (asynchronous proxy): order them after the stores
+          __threadfence();
+          asm volatile("fence.proxy.async;\n" ::: "memory");
+        }
+        __syncthreads();
+      }
+      if (threadIdx.x == 0) {
+        const int readers = cache.H_kv * C;
+        int32_t* const cnt = sa.counters + static_cast<long long>(cache.B) * cache.H_kv + b;
+        if (atomicAdd(cnt, 1) == readers - 1) {  // every block of the sequence has read the old length
+          cache.seq_lens[b] = n;
+          *cnt = 0;
+        }
+      }
+    }
+    return n;
+  };
   int len = 0, t0, t1;
-  if (OVL) {
+  if (ovl) {
     t0 = static_cast<int>((static_cast<long long>(stable_blocks) * c) / C) * kBlk;
     t1 = static_cast<int>((static_cast<long long>(stable_blocks) * (c + 1)) / C) * kBlk;
   } else {
-    len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
+    len = OVL ? read_len() : checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
     split_range(GEN ? query_lo(len, S_q, 0, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
   }
 
@@ -439,7 +502,6 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   int blk0 = t0 / kBlk;
   const int blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
   int nblk = blk1 - blk0 > team ? (blk1 - blk0 - team + NTEAM - 1) / NTEAM : 0;
-  const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
   uint8_t* const ring = smem + team * (Cf::NST * Cf::STAGE);
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
   const uint32_t bars = static_cast<uint32_t>(__cvta_generic_to_shared(smem + Cf::BARS)) + team * (Cf::NST * 8);
@@ -454,7 +516,6 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // the thread block first turns the table entries of its split into addresses of this KV head's part of each
   // page (checked against the pool once), kept in shared memory behind everything else, so that issuing a copy
   // costs a shift, a shared-memory load and a multiply-add.
-  const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
   const int pshift = PAGED ? 31 - __clz(cache.page_tokens >> 4) : 0;
   const int page0 = blk0 >> pshift;
   const uint8_t** const page_ptr = reinterpret_cast<const uint8_t**>(smem + Cf::SMEM);
@@ -612,11 +673,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   bool timed_out = false;
   int k = 0;
 #pragma unroll 1
-  for (int phase = 0; phase < (OVL ? 2 : 1); ++phase) {
-  if (OVL && phase == 1) {
+  for (int phase = 0; phase < (ovl ? 2 : 1); ++phase) {
+  if (ovl && phase == 1) {
     // the stable part is done: from here on this kernel is ordered after the one before it
     pdl_wait();
-    len = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
+    len = read_len();
     const int stable_tokens = stable_blocks * kBlk;
     if (len < stable_tokens && c == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status)
       atomicOr(status, TQ_STATUS_BAD_LEN);  // the promise did not hold: tokens beyond the length were attended
@@ -807,11 +868,82 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       }
     }
   }
+
+  // ---------------- fused step: Eq. 5 by the last block of this (sequence, KV head) to get here
+  if (OVL && sa.out != nullptr) {
+    constexpr int kWts = (Cf::MERGE + 15) & ~15;  // behind the merge arrays, inside the ring's memory
+    static_assert(kWts + kWarps * TQ_MAX_SPLITS * 4 + 16 <= Cf::PIPE, "the weights fit the ring");
+    float* const wts = reinterpret_cast<float*>(smem + kWts) + warp * TQ_MAX_SPLITS;
+    int* const ticket = reinterpret_cast<int*>(smem + kWts + kWarps * TQ_MAX_SPLITS * 4);
+    __threadfence();  // this block's partial is visible before its arrival is
+    __syncthreads();
+    if (threadIdx.x == 0) *ticket = atomicAdd(sa.counters + static_cast<long long>(b) * cache.H_kv + kvh, 1);
+    __syncthreads();
+    if (*ticket == C - 1) {
+      __threadfence();
+      if (warp < nh) {  // one warp per query head; the partials of other blocks come from L2 (ld.cg)
+        const long long prow = q_row(v0 + warp) * C;
+        // weights: every lane fetches (m, l) of up to 8 splits at once, one round trip to L2
+        constexpr int kPer = TQ_MAX_SPLITS / 32;
+        float lv[kPer], mv[kPer];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int cc = lane + 32 * i;
+          lv[i] = cc < C ? __ldcg(l_part + prow + cc) : 0.f;
+          mv[i] = cc < C ? __ldcg(m_part + prow + cc) : -INFINITY;
+        }
+        float mg = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i)
+          if (lv[i] > 0.f) mg = fmaxf(mg, mv[i]);
+#pragma unroll
+        for (int off = 16; off; off >>= 1) mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, off));
+        float den = 0.f;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int cc = lane + 32 * i;
+          const float wc = lv[i] > 0.f ? lv[i] * __expf(mv[i] - mg) : 0.f;
+          if (cc < C) wts[cc] = wc;
+          den += wc;
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
+        __syncwarp();
+        const float inv = den > 0.f ? 1.f / den : 0.f;
+        const float4* const op = reinterpret_cast<const float4*>(o_part + prow * D);
+        for (int ch = lane; ch < D / 4; ch += 32) {
+          float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+          constexpr int kBatch = 16;  // partial outputs in flight per lane
+          for (int c0 = 0; c0 < C; c0 += kBatch) {
+            float4 v[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i)
+              v[i] = c0 + i < C ? __ldcg(op + static_cast<long long>(c0 + i) * (D / 4) + ch) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+              const float wc = c0 + i < C ? wts[c0 + i] : 0.f;
+              a.x = fmaf(wc, v[i].x, a.x); a.y = fmaf(wc, v[i].y, a.y); a.z = fmaf(wc, v[i].z, a.z); a.w = fmaf(wc, v[i].w, a.w);
+            }
+          }
+          a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
+          const long long orow = q_row(v0 + warp) * D;
+          if (sa.out_fp32) {
+            reinterpret_cast<float4*>(static_cast<float*>(sa.out) + orow)[ch] = a;
+          } else {
+            __half2 h[2] = {__floats2half2_rn(a.x, a.y), __floats2half2_rn(a.z, a.w)};
+            reinterpret_cast<uint2*>(static_cast<__half*>(sa.out) + orow)[ch] = *reinterpret_cast<uint2*>(h);
+          }
+        }
+      }
+      if (threadIdx.x == 0) sa.counters[static_cast<long long>(b) * cache.H_kv + kvh] = 0;  // ready for the next launch
+    }
+  }
 }
 
 template <int D, int MODE>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
-                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, cudaStream_t st) {
+                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
+                   cudaStream_t st) {
   size_t smem = Cfg<D>::SMEM;
   if (MODE == 2) {
     // room for the page addresses of the longest split: its blocks, rounded out to whole pages
@@ -826,30 +958,45 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
   const int GV = (H_q / c.H_kv) * S_q;
   dim3 grid(C, c.H_kv * ((GV + 7) / 8), c.B);
   return launch_kernel(decode_mma_kernel<D, MODE>, grid, dim3(kThreads), smem, st, c, q, H_q, S_q, attn_scale, window, C,
-                       o_part, m_part, l_part, status, stable_blocks);
+                       o_part, m_part, l_part, status, stable_blocks, sa);
 }
 
 template <int D>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
-                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, cudaStream_t st) {
-  if (c.page_table != nullptr) return launch<D, 2>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, st);
-  if (window > 0 || S_q > 1) return launch<D, 1>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, st);
-  if (stable_blocks > 0) return launch<D, 3>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, st);
-  return launch<D, 0>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, 0, st);
+                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
+                   bool step, cudaStream_t st) {
+  const StepArgs none = {nullptr, nullptr, nullptr, 0, nullptr};
+  if (step) return launch<D, 3>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
+  if (c.page_table != nullptr) return launch<D, 2>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, none, st);
+  if (window > 0 || S_q > 1) return launch<D, 1>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, none, st);
+  return launch<D, 0>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, 0, none, st);
 }
 
 }  // namespace
 
-// stable_tokens > 0 selects the overlapped form (plain decode over a contiguous cache only; see tq.h)
+// Plain decode; stable_tokens > 0 selects the overlapped form (contiguous cache, one query token, no window).
 cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
                               int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st,
                               int stable_tokens) {
+  return launch_decode_step(c, nullptr, nullptr, q, H_q, S_q, attn_scale, window, C, stable_tokens, o_part, m_part, l_part,
+                            nullptr, nullptr, false, status, st);
+}
+
+// The fused step (tq_sdpa_int4_step): k_new / v_new non-null appends one token, out non-null reduces in the
+// same launch (counters then points at B * H_kv + B zeroed ints).  Both null with stable_tokens > 0 is the
+// overlapped decode.
+cudaError_t launch_decode_step(const tq_kv_cache& c, const __half* k_new, const __half* v_new, const __half* q, int H_q,
+                               int S_q, float attn_scale, int window, int C, int stable_tokens, float* o_part,
+                               float* m_part, float* l_part, int32_t* counters, void* out, bool out_fp32,
+                               int32_t* status, cudaStream_t st) {
   const int sb = stable_tokens > 0 ? stable_tokens / kBlk : 0;
+  const StepArgs sa = {k_new, v_new, out, out_fp32 ? 1 : 0, counters};
+  const bool step = c.page_table == nullptr && window == 0 && S_q == 1 && (sb > 0 || k_new != nullptr || out != nullptr);
   switch (c.d) {
-    case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
-    case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
-    case 512: return launch<512>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
-    default: return launch<256>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, st);
+    case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);
+    case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);
+    case 512: return launch<512>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);
+    default: return launch<256>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);
   }
 }
 

@@ -10,102 +10,11 @@
 // is bit-identical on any machine that follows the same operation order:
 //   s = fp16((max - min) / 15);  z = fp16((0 - min) / s);  q = clamp(rint(x / s + z), 0, 15).
 #include "tq_internal.cuh"
+#include "tq_quantize_core.cuh"
 
 namespace tq {
 namespace {
 
-
-struct QuantOut {
-  uint32_t word;  // eight codes, element i in bits 4i .. 4i+3
-  __half s, z;    // stored scale and zero of the group
-};
-
-// The defining arithmetic, step by step (true divisions, explicit roundings): what every result must be equal
-// to, bit for bit.  Out of line: the fast path below hands over whenever it cannot prove its own result.
-__device__ __noinline__ QuantOut quantize_exact(const float (&x)[8], float mn, float mx) {
-  QuantOut out;
-  out.word = 0u;
-  const float s32 = __fdiv_rn(__fsub_rn(mx, mn), 15.0f);
-  const __half s16 = __float2half_rn(s32);
-  if ((__half_as_ushort(s16) & 0x7FFFu) == 0) {  // scale rounds to zero: constant (or nearly constant) group
-    out.s = __ushort_as_half(0x3C00u);            // 1.0
-    out.z = __float2half_rn(__fsub_rn(0.0f, mn));
-    return out;
-  }
-  const float sf = __half2float(s16);
-  float z32 = __fdiv_rn(__fsub_rn(0.0f, mn), sf);
-  z32 = fminf(fmaxf(z32, -65504.0f), 65504.0f);
-  const __half z16 = __float2half_rn(z32);
-  const float zf = __half2float(z16);
-  for (int i = 0; i < 8; ++i) {
-    const float u = fminf(fmaxf(__fadd_rn(__fdiv_rn(x[i], sf), zf), 0.0f), 15.0f);  // fmaxf also turns NaN into 0
-    out.word |= (__float_as_uint(u + 12582912.0f) & 0xFu) << (4 * i);             // rint, ties to even
-  }
-  out.s = s16;
-  out.z = z16;
-  return out;
-}
-
-// Quantise the 8 elements held by this thread (quad = one group).  All 32 lanes must call.
-//
-// Defining arithmetic: s = fp16((max - min) / 15), z = fp16(clamp((0 - min) / s)), u = fl(fl(x / s) + z),
-// q = clamp(rint(u), 0, 15), every operation rounded to nearest even in binary32.  A division, a round, two
-// clamps and a conversion per element would make this kernel many times slower than the memory system, so
-// the common case does less and proves that it changed nothing:
-//   ua = fma(x, 1/s, z) with the correctly rounded reciprocal differs from u by at most
-//        (|x/s| + |u|) * 2^-23 <= tol (a per-group bound, with a 4x margin);
-//   ua is monotone in x, so all eight lie between fma(min, 1/s, z) and fma(max, 1/s, z): if those are inside
-//        (-0.49, 15.49) no clamp can act;
-//   r = (ua + 1.5 * 2^23) - 1.5 * 2^23 is rint(ua), ties to even; if no ua is within tol of a rounding
-//        boundary k + 1/2, rint(u) = rint(ua) for all eight.
-// Whenever one of the conditions fails (a NaN anywhere fails them too: degenerate groups, overflowing zeros,
-// non-finite inputs) the thread takes quantize_exact.  The result is bit-identical to the defining arithmetic.
-__device__ __forceinline__ void quantize_chunk(const uint4 raw, uint32_t& word, __half& s_out, __half& z_out) {
-  const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-  float x[8];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 f = __half22float2(h2[i]);
-    x[2 * i] = f.x;
-    x[2 * i + 1] = f.y;
-  }
-  float mn = fminf(fminf(fminf(x[0], x[1]), fminf(x[2], x[3])), fminf(fminf(x[4], x[5]), fminf(x[6], x[7])));
-  float mx = fmaxf(fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), fmaxf(fmaxf(x[4], x[5]), fmaxf(x[6], x[7])));
-#pragma unroll
-  for (int off = 1; off <= 2; off <<= 1) {
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-  }
-  const __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(mx, mn), 15.0f));
-  const float sf = __half2float(s16);
-  const __half z16 = __float2half_rn(__fdiv_rn(__fsub_rn(0.0f, mn), sf));  // no clamp here: an overflow fails the checks
-  const float zf = __half2float(z16);
-  const float rs = __frcp_rn(sf);
-  const float tol = (2.0f * fmaxf(fabsf(mn), fabsf(mx)) * rs + fabsf(zf) + 17.0f) * 4.76837158203125e-7f;  // 2^-21
-  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
-  float r[8];          // the codes as floats
-  float far = 0.0f;    // largest |ua - rint(ua)| over the 8 elements (at most 1/2)
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const float u = fmaf(x[i], rs, zf);
-    r[i] = (u + kMagic) - kMagic;
-    far = fmaxf(far, fabsf(u - r[i]));
-  }
-  // four codes are a 16-bit integer that fp32 holds exactly: Horner with fused multiply-adds, then the
-  // integer is read off the low mantissa bits of (value + 2^23)
-  const float lo = fmaf(fmaf(fmaf(r[3], 16.0f, r[2]), 16.0f, r[1]), 16.0f, r[0]);
-  const float hi = fmaf(fmaf(fmaf(r[7], 16.0f, r[6]), 16.0f, r[5]), 16.0f, r[4]);
-  word = __byte_perm(__float_as_uint(lo + 8388608.0f), __float_as_uint(hi + 8388608.0f), 0x5410);
-  s_out = s16;
-  z_out = z16;
-  const bool proven = fmaf(mn, rs, zf) > -0.49f && fmaf(mx, rs, zf) < 15.49f && 0.5f - far > tol;
-  if (!proven) {  // rare
-    const QuantOut e = quantize_exact(x, mn, mx);
-    word = e.word;
-    s_out = e.s;
-    z_out = e.z;
-  }
-}
 
 // chunk index -> (b, h, t, c) of a [B][H_kv][T][d] tensor and the destination row in the cache
 __device__ __forceinline__ void process_chunk(const tq_kv_cache& c, const __half* src, int which, int T,

@@ -29,7 +29,7 @@ SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa
            "tq_result_string", "tq_last_cuda_error", "tq_version", "tq_sdpa_int4_attend_static",
            "tq_cache_code_offset", "tq_cache_meta_offset", "tq_sdpa_int4_decode_window", "tq_split_range_window",
            "tq_sdpa_int4_decode_multi", "tq_sdpa_mixed_precision_attend", "tq_sdpa_int4_decode_overlapped",
-           "tq_split_range_stable")
+           "tq_split_range_stable", "tq_sdpa_int4_step", "tq_step_workspace_bytes", "tq_step_counter_bytes", "tq_auto_splits_step")
 
 
 class tq_kv_cache(C.Structure):
@@ -48,6 +48,8 @@ _lib.tq_kv_quantize_append.argtypes = [_cache_p, _vp, _vp, _i32, _vp, _vp]
 _lib.tq_kv_quantize_append.restype = C.c_int
 _lib.tq_auto_splits.argtypes = [_i32] * 5
 _lib.tq_auto_splits.restype = _i32
+_lib.tq_auto_splits_step.argtypes = [_i32] * 5
+_lib.tq_auto_splits_step.restype = _i32
 _lib.tq_split_range.argtypes = [_i32, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.tq_split_range.restype = None
 _lib.tq_sdpa_int4_decode.argtypes = [_cache_p, _vp, _i32, _f32, _i32, _vp, _vp, _vp, _vp, _vp]
@@ -56,6 +58,12 @@ _lib.tq_sdpa_int4_decode_overlapped.argtypes = [_cache_p, _vp, _i32, _f32, _i32,
 _lib.tq_sdpa_int4_decode_overlapped.restype = C.c_int
 _lib.tq_split_range_stable.argtypes = [_i32, _i32, _i32, _i32, C.POINTER(_i32), C.POINTER(_i32)]
 _lib.tq_split_range_stable.restype = None
+_lib.tq_sdpa_int4_step.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _i32, _vp, _sz, _vp, _i32, _vp, _vp]
+_lib.tq_sdpa_int4_step.restype = C.c_int
+_lib.tq_step_workspace_bytes.argtypes = [_i32] * 5
+_lib.tq_step_workspace_bytes.restype = _sz
+_lib.tq_step_counter_bytes.argtypes = [_i32] * 2
+_lib.tq_step_counter_bytes.restype = _sz
 _lib.tq_sdpa_int4_decode_window.argtypes = [_cache_p, _vp, _i32, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
 _lib.tq_sdpa_int4_decode_window.restype = C.c_int
 _lib.tq_sdpa_int4_decode_multi.argtypes = [_cache_p, _vp, _i32, _i32, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
@@ -201,6 +209,10 @@ def tq_auto_splits(B, H_kv, H_q, d, max_seq_len):
     return int(_lib.tq_auto_splits(B, H_kv, H_q, d, max_seq_len))
 
 
+def tq_auto_splits_step(B, H_kv, H_q, d, max_seq_len):
+    return int(_lib.tq_auto_splits_step(B, H_kv, H_q, d, max_seq_len))
+
+
 def tq_split_range(length, C_, c):
     t0, t1 = _i32(), _i32()
     _lib.tq_split_range(length, C_, c, C.byref(t0), C.byref(t1))
@@ -238,6 +250,24 @@ def tq_sdpa_int4_decode_overlapped(cache, q, attn_scale, num_splits, stable_toke
     _check(_lib.tq_sdpa_int4_decode_overlapped(C.byref(cs), _ptr(q), q.shape[1], float(attn_scale), int(num_splits),
                                                int(stable_tokens), _ptr(o_part), _ptr(m_part), _ptr(l_part),
                                                _ptr(status), _stream(stream)), "tq_sdpa_int4_decode_overlapped")
+
+
+def alloc_step_workspace(B, H_kv, H_q, d, num_splits, device="cuda"):
+    """Zeroed workspace of tq_sdpa_int4_step (counters, then partials) as a uint8 tensor."""
+    return torch.zeros(int(_lib.tq_step_workspace_bytes(B, H_kv, H_q, d, num_splits)), dtype=torch.uint8, device=device)
+
+
+def tq_sdpa_int4_step(cache, k_new, v_new, q, attn_scale, num_splits, stable_tokens, workspace, out, status=None,
+                      stream=None):
+    """append (k_new, v_new: [B][H_kv][1][d] fp16 or None) + fused int4 attention + split reduction, one launch."""
+    assert q.is_contiguous() and q.dtype == torch.float16 and q.dim() == 3
+    assert out.is_contiguous() and out.shape == q.shape and out.dtype in (torch.float16, torch.float32)
+    for t in (k_new, v_new):
+        assert t is None or (t.is_contiguous() and t.dtype == torch.float16 and t.shape == (cache.B, cache.H_kv, 1, cache.d))
+    cs = _cs(cache)
+    _check(_lib.tq_sdpa_int4_step(C.byref(cs), _ptr(k_new), _ptr(v_new), _ptr(q), q.shape[1], float(attn_scale),
+                                  int(num_splits), int(stable_tokens), _ptr(workspace), workspace.numel(), _ptr(out),
+                                  int(out.dtype == torch.float32), _ptr(status), _stream(stream)), "tq_sdpa_int4_step")
 
 
 def tq_split_range_stable(length, stable_tokens, C_, c):

@@ -157,3 +157,133 @@ def test_back_to_back_steps_overlap_their_predecessors(gpu, oracle, use_graph):
         if i in (0, 1, 4, 5, 10, steps - 1):       # lengths 4107 + i + 1: the second sequence crosses 4112 = 257 * 16 at i = 4
             assert_attention_close(got[i], oracle.attention(host, qn[i], sh.alpha), f"step {i}")
     assert dev.seq_lens.cpu().tolist() == [lens[0] + steps, lens[1] + steps]
+
+
+# ------------------------------------------------------------------------------------------------ fused step
+def _step_setup(tq, torch, oracle, sh, S, S_cap, lens, seed):
+    k, v = I.make_kv(sh, S, seed)
+    host = oracle_cache(oracle, sh, k, v, S_cap, lens)
+    dev = device_cache(tq, torch, sh, k, v, S_cap, lens, fill_byte=0xFF)
+    return host, dev
+
+
+@pytest.mark.parametrize("d,H_q,H_kv", [(128, 16, 2), (64, 4, 1), (256, 4, 2), (512, 8, 1), (128, 64, 8)])
+def test_fused_step_matches_three_calls_and_oracle(gpu, oracle, d, H_q, H_kv):
+    """tq_sdpa_int4_step against the oracle: the appended rows bit for bit, the lengths, and the outputs, over
+    several steps, stable parts (none, exact, short), split counts, both output types; lengths pass a block
+    boundary, one sequence is one token short of its capacity at the start."""
+    from util import assert_cache_bits_equal
+    tq, torch = gpu
+    sh = I.Shape("x", 3, H_q, H_kv, d, d ** -0.5 if d < 256 else 1.0, sigma_qk=1.0 if d < 256 else 0.25,
+                 k_outlier_channels=4 if d == 128 else 0)
+    lens = [900, 13, 1039]
+    S_cap = 1040
+    host, dev = _step_setup(tq, torch, oracle, sh, 1039, S_cap, lens, 111)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for step, (C, stable, dt) in enumerate(((4, 0, torch.float32), (4, 0, torch.float32), (3, 896, torch.float32),
+                                            (1, 0, torch.float16), (7, 16, torch.float32), (37, 900, torch.float32))):
+        ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, C)
+        kn, vn = I.make_kv(sh, 1, 111, stream=1 + step)
+        qn = I.make_q(sh, 111, stream=step)
+        out = torch.full((sh.B, sh.H_q, sh.d), 7.0, dtype=dt, device="cuda")
+        st_stable = min(stable, 13 // 16 * 16) if stable else 0    # the promise must hold for every sequence
+        tq.tq_sdpa_int4_step(dev, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(qn).cuda(),
+                             sh.alpha, C, st_stable, ws, out, status)
+        torch.cuda.synchronize()
+        skipped = host.append(kn, vn)
+        full = int(status.item()) & tq.TQ_STATUS_CACHE_FULL
+        assert bool(full) == (skipped > 0) and int(status.item()) & ~tq.TQ_STATUS_CACHE_FULL == 0
+        status.zero_()
+        assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
+        assert_cache_bits_equal(dev, host)
+        assert not ws[:tq._lib.tq_step_counter_bytes(sh.B, sh.H_kv)].any()     # counters are left zero
+        ref = oracle.attention(host, qn, sh.alpha)
+        got = out.float().cpu().numpy()
+        if dt == torch.float32:
+            assert_attention_close(got, ref, f"step {step} C={C} stable={st_stable}")
+        else:
+            assert np.abs(got - ref).max() <= 2e-3 + np.abs(ref).max() * 2.0 ** -11
+    assert host.lens.tolist() == [906, 19, 1040]
+
+
+def test_fused_step_with_a_real_stable_part_and_no_append(gpu, oracle):
+    tq, torch = gpu
+    sh = I.Shape("x", 2, 64, 8, 128, 128 ** -0.5, k_outlier_channels=4)
+    lens = [5000, 4100]
+    host, dev = _step_setup(tq, torch, oracle, sh, 5000, 5008, lens, 112)
+    q = I.make_q(sh, 112)
+    ref = oracle.attention(host, q, sh.alpha)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for C, stable in ((9, 4096), (0, 4100), (16, 0)):
+        Cn = C or tq.tq_auto_splits_step(sh.B, sh.H_kv, sh.H_q, sh.d, 5008)
+        ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, Cn)
+        out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+        tq.tq_sdpa_int4_step(dev, None, None, torch.from_numpy(q).cuda(), sh.alpha, C, stable, ws, out, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0 and dev.seq_lens.cpu().tolist() == lens
+        assert_attention_close(out.cpu().numpy(), ref, f"no append C={C} stable={stable}")
+
+
+def test_fused_step_argument_checks(gpu):
+    tq, torch = gpu
+    dev = tq.KVCache(1, 2, 64, 128)
+    q = torch.zeros((1, 32, 128), dtype=torch.float16, device="cuda")       # 16 query heads per KV head
+    out = torch.zeros((1, 32, 128), dtype=torch.float32, device="cuda")
+    ws = tq.alloc_step_workspace(1, 2, 32, 128, 2)
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_sdpa_int4_step(dev, None, None, q, 1.0, 2, 0, ws, out)
+    assert e.value.code == tq.TQ_ERR_SHAPE
+    q, out = q[:, :16].contiguous(), out[:, :16].contiguous()
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_sdpa_int4_step(dev, None, None, q, 1.0, 2, 0, ws[:1024], out)
+    assert e.value.code == tq.TQ_ERR_WORKSPACE
+    paged = tq.PagedKVCache(1, 2, 32, 2, 3, 128)
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_sdpa_int4_step(paged, None, None, q, 1.0, 2, 0, ws, out)
+    assert e.value.code == tq.TQ_ERR_SHAPE
+
+
+@pytest.mark.parametrize("use_graph", [False, True])
+def test_fused_steps_back_to_back(gpu, oracle, use_graph):
+    """Twenty fused steps on one cache enqueued without synchronisation (each kernel overlaps the tail of the
+    one before it), eager and as a replayed CUDA graph: every output matches the oracle, the cache ends up
+    bit-identical to the oracle's."""
+    from util import assert_cache_bits_equal
+    tq, torch = gpu
+    sh = I.Shape("x", 2, 64, 8, 128, 128 ** -0.5, k_outlier_channels=4)
+    lens = [6000, 4107]
+    steps, C, stable = 20, 9, 4096
+    host, dev = _step_setup(tq, torch, oracle, sh, 6000, 6032, lens, 113)
+    kn = [I.make_kv(sh, 1, 113, stream=1 + i) for i in range(steps)]
+    qn = [I.make_q(sh, 113, stream=i) for i in range(steps)]
+    k_in = torch.stack([torch.from_numpy(a[0]) for a in kn]).cuda()
+    v_in = torch.stack([torch.from_numpy(a[1]) for a in kn]).cuda()
+    q_in = torch.stack([torch.from_numpy(a) for a in qn]).cuda()
+    outs = torch.zeros((steps, sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+    ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, C)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    def enqueue(cache):
+        for i in range(steps):
+            tq.tq_sdpa_int4_step(cache, k_in[i], v_in[i], q_in[i], sh.alpha, C, stable, ws, outs[i], status)
+
+    if use_graph:
+        warm = tq.KVCache(sh.B, sh.H_kv, 6032, sh.d)      # function attributes are set outside the capture
+        warm.blocks.copy_(dev.blocks); warm.seq_lens.copy_(dev.seq_lens)
+        tq.tq_sdpa_int4_step(warm, k_in[0], v_in[0], q_in[0], sh.alpha, C, stable, ws, outs[0], status)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            enqueue(dev)
+        g.replay()
+    else:
+        enqueue(dev)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = outs.cpu().numpy()
+    for i in range(steps):
+        host.append(*kn[i])
+        if i in (0, 1, 4, 5, 10, steps - 1):
+            assert_attention_close(got[i], oracle.attention(host, qn[i], sh.alpha), f"step {i}")
+    assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
+    assert_cache_bits_equal(dev, host)
