@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--splits", type=int, default=0, help="sequence splits C of the fused kernel (0 = library default)")
     ap.add_argument("--classic", action="store_true",
                     help="time the step as three calls (append, tq_sdpa_int4_decode, combine) instead of the fused step")
+    ap.add_argument("--lib", default=None,
+                    help="time another build of the library (a timing probe from `build.py --probe`); implies --no-parity")
     ap.add_argument("--no-parity", action="store_true", help="skip the oracle check of sampled layers of the timed state")
     return ap.parse_args()
 
@@ -202,6 +204,9 @@ def main():
         run_reference(args, rank)
         return
 
+    if args.lib:
+        os.environ["TQ_LIBRARY"] = os.path.abspath(args.lib)
+        args.no_parity = True
     import torch
     from paper_2604_16957_b200 import tq  # fails loudly if libtq.so is missing
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
@@ -378,7 +383,7 @@ def main():
             "step_entry": ("tq_kv_quantize_append + tq_sdpa_int4_decode + tq_sdpa_int4_combine" if args.classic else
                            f"tq_sdpa_int4_step(stable_tokens={S}): one launch per layer"),
             "hbm_gbs_whole_step": alg_bytes / (us_per_layer * 1e-6) / 1e9, "num_splits": C,
-            "paper_context": PAPER_CONTEXT, "device": device_info(torch, dev)}
+            "paper_context": PAPER_CONTEXT, "device": device_info(torch, dev), "library": tq.tq_version()}
     if parity is not None:
         line["parity"] = parity
     if world > 1:

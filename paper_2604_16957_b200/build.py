@@ -1,6 +1,11 @@
 """Build libtq.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
     python -m paper_2604_16957_b200.build [--force] [--verbose]
+    python -m paper_2604_16957_b200.build --probe copies|math    # timing-probe builds of the decode kernel
+
+The probe libraries (libtq_probe_copies.so, libtq_probe_math.so) are the same sources compiled with
+-DTQ_PROBE_COPIES_ONLY / -DTQ_PROBE_MATH_ONLY: the fused decode kernel with its arithmetic, or its copies,
+taken out.  They produce meaningless results and exist only to time (`bench.py --lib <path>`).
 """
 import glob
 import os
@@ -42,5 +47,17 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_probe(which: str) -> str:
+    """Timing-probe build of the library: which = "copies" or "math"."""
+    macro = {"copies": "TQ_PROBE_COPIES_ONLY", "math": "TQ_PROBE_MATH_ONLY"}[which]
+    out = os.path.join(HERE, f"libtq_probe_{which}.so")
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    subprocess.run([nvcc] + NVCC_FLAGS + ["-D" + macro, "-I", INCLUDE, "-I", CSRC, "-o", out] + sources(), check=True)
+    return out
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--probe" in sys.argv:
+        print(build_probe(sys.argv[sys.argv.index("--probe") + 1]))
+    else:
+        print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))

@@ -343,7 +343,15 @@ const char* tq_result_string(int r) {
 
 int tq_last_cuda_error(void) { return g_last_cuda_error; }
 
-const char* tq_version(void) { return "libtq 0.2 (sm_100a)"; }
+const char* tq_version(void) {
+#if defined(TQ_PROBE_COPIES_ONLY)
+  return "libtq 0.2 (sm_100a) TIMING PROBE: copies only, results are meaningless";
+#elif defined(TQ_PROBE_MATH_ONLY)
+  return "libtq 0.2 (sm_100a) TIMING PROBE: arithmetic only, results are meaningless";
+#else
+  return "libtq 0.2 (sm_100a)";
+#endif
+}
 
 // Test hook (tq_internal.cuh); deliberately absent from tq.h.
 int tq_internal_test_hook(int key, int value) {
