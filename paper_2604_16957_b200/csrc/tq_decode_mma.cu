@@ -47,6 +47,7 @@
 //   V: ldmatrix.trans  -> lane (gid, tid4) holds 16-bit lane gid of tokens 2*tid4 and 2*tid4+1
 //      side by side: the token-pair interleave the P.V MMA needs (k = tokens), done by the
 //      load itself, so V needs no byte permutes.
+#include "tq_async.cuh"
 #include "tq_internal.cuh"
 #include "tq_quantize_core.cuh"
 
@@ -60,7 +61,6 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 4.0f;  // log2 units
 constexpr float kNoMax = -1.0e30f;         // running reference before any token was seen
-constexpr long long kMaxWaitCycles = 1LL << 22;  // bound of every mbarrier wait: about 2 ms of SM clock
 constexpr uint32_t kMaskLo = 0x000F000Fu;  // nibbles 0 / 4 of a 32-bit word: n * 2^-24 as fp16
 constexpr uint32_t kMaskHi = 0x00F000F0u;  // nibbles 1 / 5: n * 2^-20 as fp16
 
@@ -131,39 +131,6 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
-}
-
-// ---- bulk-copy / mbarrier primitives.  Every wait on an mbarrier in this file is bounded.
-__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// non-blocking probe of a phase
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// contiguous global -> shared copy (both 16-byte aligned, size a multiple of 16) completing on an mbarrier
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
 }
 
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
@@ -368,19 +335,6 @@ __device__ __noinline__ RowMask general_row_mask(const int32_t* seq_lens, int b,
   const int hi0 = query_hi(n, S_q, s0), hi1 = query_hi(n, S_q, s1);
   return RowMask{e - first, window_begin(hi0, window) - first, min(hi0, e) - first, window_begin(hi1, window) - first,
                  min(hi1, e) - first};
-}
-
-// Bounded wait on an mbarrier phase; false if the copy did not complete within the limit.
-__device__ __noinline__ bool wait_stage_slow(uint32_t bar, uint32_t parity, long long limit) {
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > limit) return false;
-  }
-  return true;
-}
-__device__ __forceinline__ bool wait_stage(uint32_t bar, uint32_t parity, long long limit = kMaxWaitCycles) {
-  if (mbar_try_wait(bar, parity)) return true;  // the common case: the copy landed while the warp computed
-  return wait_stage_slow(bar, parity, limit);
 }
 
 // What the fused decode step (tq_sdpa_int4_step) adds to phase 1; all null for the plain calls.

@@ -101,4 +101,79 @@ __device__ __forceinline__ void quantize_chunk(const uint4 raw, uint32_t& word, 
   }
 }
 
+
+// The same quantiser for a thread that holds a whole group of 32 elements (the bulk kernel): minimum and
+// maximum are found on the packed halves, the per-group work (two divisions, a reciprocal, the bound) is paid
+// once per 32 elements instead of once per 8, and no shuffle is needed.  raw[j] holds elements 8j .. 8j+7.
+// Bit-identical to quantize_chunk run by a lane quad, by the same argument: the fast path proves its own
+// result or hands over to quantize_exact.
+__device__ __forceinline__ void quantize_group32(const uint4 (&raw)[4], uint32_t (&word)[4], __half& s_out, __half& z_out) {
+  const __half2* h2 = reinterpret_cast<const __half2*>(&raw[0]);
+  __half2 mn2 = h2[0], mx2 = h2[0];
+#pragma unroll
+  for (int i = 1; i < 16; ++i) {
+    mn2 = __hmin2(mn2, h2[i]);
+    mx2 = __hmax2(mx2, h2[i]);
+  }
+  const float mn = fminf(__low2float(mn2), __high2float(mn2));
+  const float mx = fmaxf(__low2float(mx2), __high2float(mx2));
+  const __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(mx, mn), 15.0f));
+  const float sf = __half2float(s16);
+  const __half z16 = __float2half_rn(__fdiv_rn(__fsub_rn(0.0f, mn), sf));  // no clamp here: an overflow fails the checks
+  const float zf = __half2float(z16);
+  const float rs = __frcp_rn(sf);
+  const float tol = (2.0f * fmaxf(fabsf(mn), fabsf(mx)) * rs + fabsf(zf) + 17.0f) * 4.76837158203125e-7f;  // 2^-21
+  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
+  float far = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    float r[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(h2[4 * j + i]);
+      const float u0 = fmaf(f.x, rs, zf), u1 = fmaf(f.y, rs, zf);
+      r[2 * i] = (u0 + kMagic) - kMagic;
+      r[2 * i + 1] = (u1 + kMagic) - kMagic;
+      far = fmaxf(far, fmaxf(fabsf(u0 - r[2 * i]), fabsf(u1 - r[2 * i + 1])));
+    }
+    const float lo = fmaf(fmaf(fmaf(r[3], 16.0f, r[2]), 16.0f, r[1]), 16.0f, r[0]);
+    const float hi = fmaf(fmaf(fmaf(r[7], 16.0f, r[6]), 16.0f, r[5]), 16.0f, r[4]);
+    word[j] = __byte_perm(__float_as_uint(lo + 8388608.0f), __float_as_uint(hi + 8388608.0f), 0x5410);
+  }
+  s_out = s16;
+  z_out = z16;
+  const bool in_range = fmaf(mn, rs, zf) > -0.49f && fmaf(mx, rs, zf) < 15.49f;
+  if (in_range && !(0.5f - far > tol) && far <= 0.5f) {
+    // Rare: no clamp can act, but some element sits within the bound of a rounding boundary.  Only such
+    // elements are redone with the defining arithmetic (a true division) and their codes put in place.
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {  // unrolled: every index is a constant, the arrays stay in registers
+      const float2 f = __half22float2(h2[i >> 1]);
+      const float x = (i & 1) ? f.y : f.x;
+      const float u = fmaf(x, rs, zf);
+      const float r = (u + kMagic) - kMagic;
+      if (!(0.5f - fabsf(u - r) > tol)) {
+        const float ue = __fadd_rn(__fdiv_rn(x, sf), zf);
+        const uint32_t q = __float_as_uint(ue + kMagic) & 0xFu;  // rint, ties to even; 0 .. 15 because no clamp can act
+        word[i >> 3] = (word[i >> 3] & ~(0xFu << (4 * (i & 7)))) | (q << (4 * (i & 7)));
+      }
+    }
+  } else if (!(in_range && 0.5f - far > tol)) {  // rarer: clamps, degenerate scales, non-finite values
+#pragma unroll 1
+    for (int j = 0; j < 4; ++j) {
+      float x[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h2[4 * j + i]);
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+      }
+      const QuantOut e = quantize_exact(x, mn, mx);
+      word[j] = e.word;
+      s_out = e.s;
+      z_out = e.z;
+    }
+  }
+}
+
 }  // namespace tq

@@ -19,6 +19,7 @@ from . import tq
 
 L2_BYTES = 126 << 20
 IDENTITY_PAGES = False  # --identity-pages: page i of a paged cache is pool page i (default: a random assignment)
+SEPARATE_CALLS = False  # --calls: time append / decode / combine as separate launches even where the fused step applies
 
 
 def _fill(B, H_kv, S_cap, d, n_caches, seed, outliers, sigma=1.0, lens=None, page_tokens=0):
@@ -99,8 +100,15 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
     caches = _fill(B, H_kv, S_cap, d, n, 31, outliers, sigma, lens if lens is not None else [S] * B, page_tokens)
     base_lens = torch.as_tensor(lens if lens is not None else [S] * B, dtype=torch.int32).cuda()
     span = window or S
-    C = splits or tq.tq_auto_splits(B, H_kv, H_q * S_q, d, span)
+    # one launch per step (tq_sdpa_int4_step) wherever it applies: plain decode, contiguous cache, at most 8 query
+    # heads per KV head; the tokens present before the timed steps are its stable part
+    fused = (not SEPARATE_CALLS) and S_q == 1 and window == 0 and not page_tokens and H_q // H_kv <= 8
+    C = splits or (tq.tq_auto_splits_step if fused else tq.tq_auto_splits)(B, H_kv, H_q * S_q, d, span)
     o, m, l = tq.alloc_partials(B, H_q * S_q, d, C)
+    ws = tq.alloc_step_workspace(B, H_kv, H_q, d, C) if fused else None
+    # (the stable part is one number for the whole batch: with ragged lengths the last split of the longer
+    # sequences would get everything beyond it, so the ragged batch declares none)
+    stable = 0 if lens is not None and min(lens) != max(lens) else S
     gen = torch.Generator(device="cuda").manual_seed(5)
     q = (torch.randn((B, S_q, H_q, d), generator=gen, device="cuda") * sigma).half()
     kn = (torch.randn((B, H_kv, S_q, d), generator=gen, device="cuda") * sigma).half()
@@ -114,6 +122,10 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
 
     def enqueue():
         for c in caches:
+            if fused:
+                tq.tq_sdpa_int4_step(c, kn if with_append else None, vn if with_append else None, q[:, 0], alpha, C, stable,
+                                     ws, out, status)
+                continue
             if with_append:
                 tq.tq_kv_quantize_append(c, kn, vn, status)
             if S_q == 1 and window == 0:
@@ -139,7 +151,9 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
 
         extra["dequant_then_attend_us"] = round(_time(enqueue_cmp, max(2, steps // 4), 1) / n * 1e6, 1)
     _emit(name, us, alg, B=B, H_q=H_q, H_kv=H_kv, d=d, S=S if lens is None else "ragged", S_q=S_q, window=window,
-          num_splits=C, caches_rotated=n, page_tokens=page_tokens, includes="append+decode+combine" if with_append else "decode+combine", **extra)
+          num_splits=C, caches_rotated=n, page_tokens=page_tokens,
+          includes="append+decode+combine" if with_append else "decode+combine",
+          entry="tq_sdpa_int4_step (one launch)" if fused else "separate calls", **extra)
 
 
 def bulk_quantize_workload(steps, warmup):
@@ -172,7 +186,7 @@ WORKLOADS = {
     "llama_8k": lambda a: decode_workload("llama shape, 8K context", 1, 64, 8, 128, 8192, 128 ** -0.5, a.steps, a.warmup, True),
     "llama_32k": lambda a: decode_workload("llama shape, 32K context", 1, 64, 8, 128, 32768, 128 ** -0.5, a.steps, a.warmup, True),
     "gemma_32k": lambda a: decode_workload("gemma-style d=256, 32K context", 1, 32, 16, 256, 32768, 1.0, a.steps, a.warmup,
-                                           False, sigma=0.25),
+                                           False, sigma=0.25, splits=a.splits),
     "gemma_32k_window": lambda a: decode_workload("gemma-style d=256, 32K context, window 1024", 1, 32, 16, 256, 32768, 1.0,
                                                   a.steps, a.warmup, False, sigma=0.25, window=1024),
     "gemma_32k_sq4": lambda a: decode_workload("gemma-style d=256, 32K context, 4 query tokens", 1, 32, 16, 256, 32768, 1.0,
@@ -204,9 +218,11 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--identity-pages", action="store_true", help="paged workloads: pool page i holds page i")
+    ap.add_argument("--calls", action="store_true", help="separate append / decode / combine launches everywhere")
     args = ap.parse_args()
-    global IDENTITY_PAGES
+    global IDENTITY_PAGES, SEPARATE_CALLS
     IDENTITY_PAGES = args.identity_pages
+    SEPARATE_CALLS = args.calls
     assert torch.cuda.is_available(), "needs a CUDA device (there is no CPU path)"
     for name, fn in WORKLOADS.items():
         if args.only in (None, name):
