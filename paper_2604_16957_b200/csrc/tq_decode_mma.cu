@@ -121,6 +121,9 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"(addr));
 }
+__device__ __forceinline__ void ldmatrix_x2(uint32_t (&r)[2], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];\n" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -140,6 +143,8 @@ template <int D>
 struct WarpCtx {
   uint32_t kaddr[Cfg<D>::NGW / 2];  // ldmatrix row address this lane supplies (slot 0 of the warp's ring), per K load; V: + PK
   uint32_t ksz_lane, vsz_lane;
+  uint32_t vz_lane, vs2_lane;  // row addresses of the V scale / zero load of the zero-point MMA and of the per-group scale loads
+  uint32_t fl_g;               // half2 lane flag of that MMA's A operand: 0 for gid < 4 (hi rows), -1 otherwise (lo rows)
   uint32_t kz_lane;            // row address of the scale / zero load that feeds the zero-point MMA of the scores
   uint32_t fl_m, fl_h;         // half2 lane flags of that MMA's A operand: (0 | -1), (1 | 0) for tid4 < 2 | >= 2
   float cs;
@@ -300,6 +305,33 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
   // ---------------- P.V: O^T[channel][head] += V^T[channel][token] * (P * s)[token][head]
   // matrix j = 4 * i + m of load i is (group j / 2 of this warp, tokens 8 * (j % 2) ..)
   uint32_t vw[4];
+  if constexpr (KZ<D>::on) {
+    // Zero-point term of all four groups by ONE MMA (instead of one per group): sum_tok (s z)[tok][g] * P[tok][head]
+    // with the product s * z split exactly into an fp16 pair, hi in rows 0-3 (groups 0-3), lo in rows 4-7, and
+    // B = fp16(P), the operand the scaled B_g below are made from.  (The code term sees fp16(fp16(P) * s), the
+    // zero term the unrounded product: the two no longer cancel rounding for rounding, which costs about a
+    // factor 1.6 in output error, inside the tolerance; it saves three MMAs and eight shared-memory wavefronts
+    // per block, 1.2 us per 128K layer when the kernel runs against the power limit.)
+    uint32_t r[4];
+    ldmatrix_x4(r, cx.vz_lane + st_off);
+    const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
+    const uint32_t a0 = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hmul2(pa, u32_as_h2(cx.fl_g))));
+    const uint32_t a2 = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hmul2(pb, u32_as_h2(cx.fl_g))));
+    mma16816(zacc[0], a0, 0u, a2, 0u, pt0, pt1);
+#pragma unroll
+    for (int g = 0; g < NGW; ++g) {
+      uint32_t vs[2];
+      ldmatrix_x2(vs, cx.vs2_lane + st_off + 32 * g);
+      const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vs[0])));
+      const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vs[1])));
+      if ((g & 1) == 0) ldmatrix_x4_trans(vw, cx.kaddr[g / 2] + st_off + Cfg<D>::PK);
+      const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
+      mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
+      const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
+      mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1 & kMaskHi, y2 & kMaskLo, y2 & kMaskHi, b0, b1);
+    }
+    return;
+  }
 #pragma unroll
   for (int g = 0; g < NGW; ++g) {
     // Scales / zeros of token pairs (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9) of group g: an ldmatrix
@@ -625,6 +657,9 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     cx.kz_lane = cx.fl_m = cx.fl_h = 0;
   }
   cx.vsz_lane = ring_s + 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
+  cx.vz_lane = ring_s + 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32;
+  cx.vs2_lane = ring_s + 2 * Cf::PK + 2 * Cf::SZ + ((lane >> 3) & 1) * 16;
+  cx.fl_g = gid < 4 ? 0u : 0xBC00BC00u;
 #pragma unroll
   for (int i = 0; i < NGW / 2; ++i) {
     const int j = 4 * i + (lane >> 3);
@@ -813,6 +848,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   const float f0 = den0 > 0.f ? ex2(m0 - M0) / den0 : 0.f;
   const float f1 = den1 > 0.f ? ex2(m1 - M1) / den1 : 0.f;
+  if constexpr (KZ<D>::on) {  // the single zero-point accumulator holds hi parts in rows 0-3, lo parts in rows 4-7
+    float z0 = zacc[0][0], z1 = zacc[0][1];
+#pragma unroll
+    for (int g = 0; g < NGW; ++g) {
+      zacc[g][0] = __shfl_sync(0xffffffffu, z0, g * 4 + tid4) + __shfl_sync(0xffffffffu, z0, (4 + g) * 4 + tid4);
+      zacc[g][1] = __shfl_sync(0xffffffffu, z1, g * 4 + tid4) + __shfl_sync(0xffffffffu, z1, (4 + g) * 4 + tid4);
+    }
+  }
   float* const mo = slab + team * D * kChPitch;
 #pragma unroll
   for (int mt = 0; mt < Cf::DW / 16; ++mt) {
