@@ -146,7 +146,7 @@ struct WarpCtx {
   uint32_t vz_lane, vs2_lane;  // row addresses of the V scale / zero load of the zero-point MMA and of the per-group scale loads
   uint32_t fl_g;               // half2 lane flag of that MMA's A operand: 0 for gid < 4 (hi rows), -1 otherwise (lo rows)
   uint32_t kz_lane;            // row address of the scale / zero load that feeds the zero-point MMA of the scores
-  uint32_t fl_m, fl_h;         // half2 lane flags of that MMA's A operand: (0 | -1), (1 | 0) for tid4 < 2 | >= 2
+  uint32_t fl_m;               // half2 lane flag of that MMA's A operand: 0 for tid4 < 2 (hi parts), -1 otherwise (lo parts)
   float cs;
   int gid;
 };
@@ -193,7 +193,9 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
     const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
     const uint32_t a0 = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hmul2(pa, u32_as_h2(cx.fl_m))));
     const uint32_t a1 = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hmul2(pb, u32_as_h2(cx.fl_m))));
-    const uint32_t a2 = h2_as_u32(__hmul2(pa, u32_as_h2(cx.fl_h))), a3 = h2_as_u32(__hmul2(pb, u32_as_h2(cx.fl_h)));
+    // k slots 8-15: hi parts again for the lanes whose B rows hold the lo parts of the group sums; the other
+    // lanes' B rows are zero, so whatever finite value they supply does not count
+    const uint32_t a2 = h2_as_u32(pa), a3 = h2_as_u32(pb);
     float accz[4];
     mma16816_first(accz, a0, a1, a2, a3, qz[0], qz[1], zero4);
     // scales of all four groups for tokens gid, gid + 8: matrices (g0 g1 | tokens 0-7), (g0 g1 | 8-15), (g2 g3 | ..)
@@ -652,9 +654,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     cx.ksz_lane = ring_s + 2 * Cf::PK + (2 * (lane >> 4) + (lane & 1)) * 32 + ((lane >> 3) & 1) * 16;
     cx.kz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32;
     cx.fl_m = tid4 < 2 ? 0u : 0xBC00BC00u;  // half2 (0, 0) | (-1, -1)
-    cx.fl_h = tid4 < 2 ? 0x3C003C00u : 0u;  // half2 (1, 1) | (0, 0)
   } else {
-    cx.kz_lane = cx.fl_m = cx.fl_h = 0;
+    cx.kz_lane = cx.fl_m = 0;
   }
   cx.vsz_lane = ring_s + 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
   cx.vz_lane = ring_s + 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32;
@@ -718,25 +719,23 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     __syncwarp();
     ready = true;
 #endif
-    for (; k + 4 <= nfull && !timed_out; k += 4) {
+    for (; k + 4 <= nfull; k += 4) {
 #pragma unroll
       for (int S = 0; S < 4; ++S) {
-        if (!timed_out) {
-          if (!ready && !wait_stage(bars + 8 * S, par, wait_limit)) {
-            timed_out = true;
-            kf = k + S;
-          } else {
+        if (!ready && !wait_stage(bars + 8 * S, par, wait_limit)) {  // cold: leave the loops, keep the phase order
+          timed_out = true;
+          kf = k + S;
+          goto phase_done;
+        }
 #ifndef TQ_PROBE_MATH_ONLY
-            if (k + S + 3 < nblk) issue_to(k + S + 3, (S + 3) & 3);
-            ready = mbar_test_wait(bars + 8 * ((S + 1) & 3), S == 3 ? par ^ 1 : par);
+        if (k + S + 3 < nblk) issue_to(k + S + 3, (S + 3) & 3);
+        ready = mbar_test_wait(bars + 8 * ((S + 1) & 3), S == 3 ? par ^ 1 : par);
 #endif
 #ifndef TQ_PROBE_COPIES_ONLY
-            float sc[4];
-            block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, cz, zero4, sc);
-            block_softmax_pv<D, false>(cx, S * Cf::STAGE, all, sc, oacc, zacc, m0, m1, l0, l1);
+        float sc[4];
+        block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, cz, zero4, sc);
+        block_softmax_pv<D, false>(cx, S * Cf::STAGE, all, sc, oacc, zacc, m0, m1, l0, l1);
 #endif
-          }
-        }
       }
       par ^= 1;
     }
@@ -803,6 +802,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       else block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
     }
   }
+  phase_done:;
   }  // phase
   if (timed_out) {
     // The copies of blocks kf, kf + 1, kf + 2 of this team may still be in flight into its ring: give each the
