@@ -143,8 +143,7 @@ template <int D>
 struct WarpCtx {
   uint32_t kaddr[Cfg<D>::NGW / 2];  // ldmatrix row address this lane supplies (slot 0 of the warp's ring), per K load; V: + PK
   uint32_t ksz_lane, vsz_lane;
-  uint32_t vz_lane, vs2_lane;  // row addresses of the V scale / zero load of the zero-point MMA and of the per-group scale loads
-  uint32_t fl_g;               // half2 lane flag of that MMA's A operand: 0 for gid < 4 (hi rows), -1 otherwise (lo rows)
+  uint32_t vz_lane, vs2_lane;  // row addresses of the V scale / zero load of the zero-point MMA and of the scale loads
   uint32_t kz_lane;            // row address of the scale / zero load that feeds the zero-point MMA of the scores
   uint32_t fl_m;               // half2 lane flag of that MMA's A operand: 0 for tid4 < 2 (hi parts), -1 otherwise (lo parts)
   float cs;
@@ -294,6 +293,7 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
 #pragma unroll
     for (int g = 0; g < NGW; ++g) {
       zacc[g][0] *= f0; zacc[g][1] *= f1;
+      if (KZ<D>::on && g == 0) { zacc[0][2] *= f0; zacc[0][3] *= f1; }  // the lo sums of the single zero-point MMA
     }
     d0 = a0 - m0; d1 = a1 - m1; d2 = a2 - m0; d3 = a3 - m1;
   }
@@ -309,23 +309,26 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
   uint32_t vw[4];
   if constexpr (KZ<D>::on) {
     // Zero-point term of all four groups by ONE MMA (instead of one per group): sum_tok (s z)[tok][g] * P[tok][head]
-    // with the product s * z split exactly into an fp16 pair, hi in rows 0-3 (groups 0-3), lo in rows 4-7, and
-    // B = fp16(P), the operand the scaled B_g below are made from.  (The code term sees fp16(fp16(P) * s), the
+    // with the product s * z split exactly into an fp16 pair -- hi = rn(s z) in rows 0-7 (row r: group r & 3),
+    // lo = fma(s, z, -hi) in rows 8-15, so the accumulator quad holds the hi sums in [0], [1] and the lo sums
+    // in [2], [3] -- and B = fp16(P), the operand the scaled B_g below are made from.  (The code term sees fp16(fp16(P) * s), the
     // zero term the unrounded product: the two no longer cancel rounding for rounding, which costs about a
     // factor 1.6 in output error, inside the tolerance; it saves three MMAs and eight shared-memory wavefronts
     // per block, 1.2 us per 128K layer when the kernel runs against the power limit.)
     uint32_t r[4];
     ldmatrix_x4(r, cx.vz_lane + st_off);
     const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
-    const uint32_t a0 = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hmul2(pa, u32_as_h2(cx.fl_g))));
-    const uint32_t a2 = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hmul2(pb, u32_as_h2(cx.fl_g))));
-    mma16816(zacc[0], a0, 0u, a2, 0u, pt0, pt1);
+    const uint32_t la = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hneg2(pa)));
+    const uint32_t lb = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hneg2(pb)));
+    mma16816(zacc[0], h2_as_u32(pa), la, h2_as_u32(pb), lb, pt0, pt1);
+    uint32_t vs[4];
 #pragma unroll
     for (int g = 0; g < NGW; ++g) {
-      uint32_t vs[2];
-      ldmatrix_x2(vs, cx.vs2_lane + st_off + 32 * g);
-      const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vs[0])));
-      const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vs[1])));
+      // scales of token pairs (2*tid4, +1) and (2*tid4+8, +9) for groups g, g+1 by one load of four matrices
+      // whose eight rows are each one and the same 16-byte chunk
+      if ((g & 1) == 0) ldmatrix_x4(vs, cx.vs2_lane + st_off + 32 * g);
+      const uint32_t b0 = h2_as_u32(__hmul2(u32_as_h2(pt0), u32_as_h2(vs[2 * (g & 1)])));
+      const uint32_t b1 = h2_as_u32(__hmul2(u32_as_h2(pt1), u32_as_h2(vs[2 * (g & 1) + 1])));
       if ((g & 1) == 0) ldmatrix_x4_trans(vw, cx.kaddr[g / 2] + st_off + Cfg<D>::PK);
       const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
       mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
@@ -659,8 +662,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   cx.vsz_lane = ring_s + 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
   cx.vz_lane = ring_s + 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32;
-  cx.vs2_lane = ring_s + 2 * Cf::PK + 2 * Cf::SZ + ((lane >> 3) & 1) * 16;
-  cx.fl_g = gid < 4 ? 0u : 0xBC00BC00u;
+  cx.vs2_lane = ring_s + 2 * Cf::PK + 2 * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane >> 4) * 32;
 #pragma unroll
   for (int i = 0; i < NGW / 2; ++i) {
     const int j = 4 * i + (lane >> 3);
@@ -848,12 +850,12 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   const float f0 = den0 > 0.f ? ex2(m0 - M0) / den0 : 0.f;
   const float f1 = den1 > 0.f ? ex2(m1 - M1) / den1 : 0.f;
-  if constexpr (KZ<D>::on) {  // the single zero-point accumulator holds hi parts in rows 0-3, lo parts in rows 4-7
-    float z0 = zacc[0][0], z1 = zacc[0][1];
+  if constexpr (KZ<D>::on) {  // the single zero-point accumulator: hi + lo sums of group r & 3 in the lanes of row r
+    const float z0 = zacc[0][0] + zacc[0][2], z1 = zacc[0][1] + zacc[0][3];
 #pragma unroll
     for (int g = 0; g < NGW; ++g) {
-      zacc[g][0] = __shfl_sync(0xffffffffu, z0, g * 4 + tid4) + __shfl_sync(0xffffffffu, z0, (4 + g) * 4 + tid4);
-      zacc[g][1] = __shfl_sync(0xffffffffu, z1, g * 4 + tid4) + __shfl_sync(0xffffffffu, z1, (4 + g) * 4 + tid4);
+      zacc[g][0] = __shfl_sync(0xffffffffu, z0, g * 4 + tid4);
+      zacc[g][1] = __shfl_sync(0xffffffffu, z1, g * 4 + tid4);
     }
   }
   float* const mo = slab + team * D * kChPitch;
