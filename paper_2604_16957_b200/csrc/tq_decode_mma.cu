@@ -149,7 +149,7 @@ struct WarpCtx {
   float cs;
   int gid;
 };
-template <int D> struct KZ { static constexpr bool on = Cfg<D>::DS == 1 && Cfg<D>::NGW == 4; };
+template <int D> struct KZ { static constexpr bool on = Cfg<D>::NGW == 4; };  // every warp that works on 128 channels
 
 // Which tokens of a block count, as rows relative to the block's first token.  Rows >= zrow lie past the
 // end of the sequence and hold unspecified bytes; column j (j = 0, 1: the thread's two score columns, i.e.
@@ -290,10 +290,13 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     for (int i = 0; i < Cfg<D>::DW / 16; ++i) {
       oacc[i][0] *= f0; oacc[i][1] *= f1; oacc[i][2] *= f0; oacc[i][3] *= f1;
     }
+    if constexpr (KZ<D>::on) {  // one accumulator quad for all groups: hi sums in [0], [1], lo sums in [2], [3]
+      zacc[0][0] *= f0; zacc[0][1] *= f1; zacc[0][2] *= f0; zacc[0][3] *= f1;
+    } else {
 #pragma unroll
-    for (int g = 0; g < NGW; ++g) {
-      zacc[g][0] *= f0; zacc[g][1] *= f1;
-      if (KZ<D>::on && g == 0) { zacc[0][2] *= f0; zacc[0][3] *= f1; }  // the lo sums of the single zero-point MMA
+      for (int g = 0; g < NGW; ++g) {
+        zacc[g][0] *= f0; zacc[g][1] *= f1;
+      }
     }
     d0 = a0 - m0; d1 = a1 - m1; d2 = a2 - m0; d3 = a3 - m1;
   }
@@ -654,15 +657,15 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   cx.cs = cs; cx.gid = gid;
   cx.ksz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32 + sub * NGW * 32;
   if constexpr (KZ<D>::on) {
-    cx.ksz_lane = ring_s + 2 * Cf::PK + (2 * (lane >> 4) + (lane & 1)) * 32 + ((lane >> 3) & 1) * 16;
-    cx.kz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32;
+    cx.ksz_lane = ring_s + 2 * Cf::PK + (2 * (lane >> 4) + (lane & 1)) * 32 + ((lane >> 3) & 1) * 16 + sub * NGW * 32;
+    cx.kz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32 + sub * NGW * 32;
     cx.fl_m = tid4 < 2 ? 0u : 0xBC00BC00u;  // half2 (0, 0) | (-1, -1)
   } else {
     cx.kz_lane = cx.fl_m = 0;
   }
   cx.vsz_lane = ring_s + 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
-  cx.vz_lane = ring_s + 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32;
-  cx.vs2_lane = ring_s + 2 * Cf::PK + 2 * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane >> 4) * 32;
+  cx.vz_lane = ring_s + 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32 + sub * NGW * 32;
+  cx.vs2_lane = ring_s + 2 * Cf::PK + 2 * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane >> 4) * 32 + sub * NGW * 32;
 #pragma unroll
   for (int i = 0; i < NGW / 2; ++i) {
     const int j = 4 * i + (lane >> 3);
@@ -899,16 +902,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // ---------------- fused step: Eq. 5 by the last block of this (sequence, KV head) to get here
   if (OVL && sa.out != nullptr) {
     constexpr int kWts = (Cf::MERGE + 15) & ~15;  // behind the merge arrays, inside the ring's memory
-    static_assert(kWts + kWarps * TQ_MAX_SPLITS * 4 + 16 <= Cf::PIPE, "the weights fit the ring");
+    static_assert(kWts + kWarps * TQ_MAX_SPLITS * 4 + 16 + kWarps * 4 <= Cf::PIPE, "the weights fit the ring");
     float* const wts = reinterpret_cast<float*>(smem + kWts) + warp * TQ_MAX_SPLITS;
     int* const ticket = reinterpret_cast<int*>(smem + kWts + kWarps * TQ_MAX_SPLITS * 4);
+    float* const inv_den = reinterpret_cast<float*>(smem + kWts + kWarps * TQ_MAX_SPLITS * 4 + 16);
     __threadfence();  // this block's partial is visible before its arrival is
     __syncthreads();
     if (threadIdx.x == 0) *ticket = atomicAdd(sa.counters + static_cast<long long>(b) * cache.H_kv + kvh, 1);
     __syncthreads();
     if (*ticket == C - 1) {
       __threadfence();
-      if (warp < nh) {  // one warp per query head; the partials of other blocks come from L2 (ld.cg)
+      if (warp < nh) {  // weights: one warp per query head; the partials of other blocks come from L2 (ld.cg)
         const long long prow = q_row(v0 + warp) * C;
         // weights: every lane fetches (m, l) of up to 8 splits at once, one round trip to L2
         constexpr int kPer = TQ_MAX_SPLITS / 32;
@@ -935,31 +939,35 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         }
 #pragma unroll
         for (int off = 16; off; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
-        __syncwarp();
-        const float inv = den > 0.f ? 1.f / den : 0.f;
-        const float4* const op = reinterpret_cast<const float4*>(o_part + prow * D);
-        for (int ch = lane; ch < D / 4; ch += 32) {
-          float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-          constexpr int kBatch = 16;  // partial outputs in flight per lane
-          for (int c0 = 0; c0 < C; c0 += kBatch) {
-            float4 v[kBatch];
+        if (lane == 0) inv_den[warp] = den > 0.f ? 1.f / den : 0.f;
+      }
+      __syncthreads();
+      // one float4 of one head's output per thread, the heads' rows spread over all the warps
+      for (int item = threadIdx.x; item < nh * (D / 4); item += kThreads) {
+        const int h = item / (D / 4), ch = item - h * (D / 4);
+        const float* const wh = reinterpret_cast<const float*>(smem + kWts) + h * TQ_MAX_SPLITS;
+        const float4* const op = reinterpret_cast<const float4*>(o_part + q_row(v0 + h) * C * D);
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        constexpr int kBatch = 16;  // partial outputs in flight per thread
+        for (int c0 = 0; c0 < C; c0 += kBatch) {
+          float4 v[kBatch];
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i)
-              v[i] = c0 + i < C ? __ldcg(op + static_cast<long long>(c0 + i) * (D / 4) + ch) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int i = 0; i < kBatch; ++i)
+            v[i] = c0 + i < C ? __ldcg(op + static_cast<long long>(c0 + i) * (D / 4) + ch) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int i = 0; i < kBatch; ++i) {
-              const float wc = c0 + i < C ? wts[c0 + i] : 0.f;
-              a.x = fmaf(wc, v[i].x, a.x); a.y = fmaf(wc, v[i].y, a.y); a.z = fmaf(wc, v[i].z, a.z); a.w = fmaf(wc, v[i].w, a.w);
-            }
+          for (int i = 0; i < kBatch; ++i) {
+            const float wc = c0 + i < C ? wh[c0 + i] : 0.f;
+            a.x = fmaf(wc, v[i].x, a.x); a.y = fmaf(wc, v[i].y, a.y); a.z = fmaf(wc, v[i].z, a.z); a.w = fmaf(wc, v[i].w, a.w);
           }
-          a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
-          const long long orow = q_row(v0 + warp) * D;
-          if (sa.out_fp32) {
-            reinterpret_cast<float4*>(static_cast<float*>(sa.out) + orow)[ch] = a;
-          } else {
-            __half2 h[2] = {__floats2half2_rn(a.x, a.y), __floats2half2_rn(a.z, a.w)};
-            reinterpret_cast<uint2*>(static_cast<__half*>(sa.out) + orow)[ch] = *reinterpret_cast<uint2*>(h);
-          }
+        }
+        const float inv = inv_den[h];
+        a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
+        const long long orow = q_row(v0 + h) * D;
+        if (sa.out_fp32) {
+          reinterpret_cast<float4*>(static_cast<float*>(sa.out) + orow)[ch] = a;
+        } else {
+          __half2 hh[2] = {__floats2half2_rn(a.x, a.y), __floats2half2_rn(a.z, a.w)};
+          reinterpret_cast<uint2*>(static_cast<__half*>(sa.out) + orow)[ch] = *reinterpret_cast<uint2*>(hh);
         }
       }
       if (threadIdx.x == 0) sa.counters[static_cast<long long>(b) * cache.H_kv + kvh] = 0;  // ready for the next launch
