@@ -225,6 +225,9 @@ size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, 
  * (sequence, KV head) unused: launches of these entry points overlap their predecessor, and with every slot
  * taken the blocks that finish a launch last (those that also reduce the partials) hold up the first blocks
  * of the next one.  Measured on the 128K Llama-shaped step: 36.5 us per layer with 37 splits, 32.3 us with 36.
+ * The spare slots are a share (sequences x KV heads) / slots of the machine: they are left only where that
+ * share is at most 1/32 (8 KV heads on 296 slots; with 16 KV heads the d = 256 shape measured 39.0 us with
+ * the spare slots and 37.4 us without).
  */
 int32_t tq_auto_splits_step(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len);
 size_t tq_step_counter_bytes(int32_t B, int32_t H_kv);

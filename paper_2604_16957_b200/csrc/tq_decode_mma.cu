@@ -514,6 +514,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #pragma unroll
     for (int s = 0; s < Cf::NST; ++s) mbar_init(bars + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    if (DS > 1) {  // the team's two timeout flags (see the score exchange below)
+      int* const xf = reinterpret_cast<int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
+      xf[0] = xf[1] = 0;
+    }
   }
   // The team's n-th block is block blk0 + team + n * NTEAM of this (sequence, KV head); one lane of the team
   // copies it into ring slot n mod NST.  Contiguous cache: it starts at head_blocks + block * STAGE.
@@ -672,9 +676,32 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     const int tok = (lane & 7) + 8 * (j % 2), grp = sub * NGW + j / 2;
     cx.kaddr[i] = ring_s + tok * Cf::ROWB + ((grp ^ Cf::swz(tok)) << 4);
   }
-  // score exchange of a team: [2 (parity of k)][DS][32 lanes] float4, then [2][DS] timeout flags
+  // Score exchange of a team: [2 (parity of k)][DS][32 lanes] float4, then two timeout flags (parity of k).
+  // The warps of a team each hold the scores over their own channels: they exchange and add them in a fixed
+  // order, so that every warp of the team continues with bit-identical scores.  The barrier of block k also
+  // tells that every warp is done with the slot of block k - 1, which is refilled after it.  A warp whose
+  // wait ran out raises the flag of that block's parity before the barrier (the flags start at 0 and are
+  // never lowered: nothing runs after a timeout), and the whole team stops together.
   float4* const xch = reinterpret_cast<float4*>(smem + Cf::XCH + team * Cf::XCH_TEAM);
-  int* const xflag = reinterpret_cast<int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
+  volatile int* const xflag = reinterpret_cast<volatile int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
+  auto exchange = [&](float (&sc)[4], int par01, bool arrived) -> bool {
+    float4* const xb = xch + par01 * (DS * 32);
+    xb[sub * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
+    if (!arrived && lane == 0) xflag[par01] = 1;
+    asm volatile("bar.sync %0, %1;\n" ::"r"(1 + team), "r"(32 * DS) : "memory");
+    if (DS == 2) {  // a + b in either order is the same number
+      const float4 part = xb[(sub ^ 1) * 32 + lane];
+      sc[0] += part.x; sc[1] += part.y; sc[2] += part.z; sc[3] += part.w;
+    } else {
+      sc[0] = sc[1] = sc[2] = sc[3] = 0.f;
+#pragma unroll
+      for (int w = 0; w < DS; ++w) {
+        const float4 part = xb[w * 32 + lane];
+        sc[0] += part.x; sc[1] += part.y; sc[2] += part.z; sc[3] += part.w;
+      }
+    }
+    return xflag[par01] == 0;
+  };
 
   bool timed_out = false;
   int k = 0, kf = 0;  // kf: the block whose wait ran out
@@ -749,6 +776,32 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #endif
    }
   }
+  if constexpr (DS > 1 && !GEN) {
+   if (phase == 0) {
+    // The same four-block step for a team: the scores of each block are exchanged before its softmax.
+    static_assert(Cf::NST == 4, "the unrolled loop walks a ring of four slots");
+    const RowMask all{kBlk, 0, kBlk, 0, kBlk};
+    uint32_t par = 0;
+    bool ready = k + 4 <= nfull ? mbar_test_wait(bars, 0) : false;
+    for (; k + 4 <= nfull; k += 4) {
+#pragma unroll
+      for (int S = 0; S < 4; ++S) {
+        const bool arrived = ready || wait_stage(bars + 8 * S, par, wait_limit);
+        float sc[4];
+        block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, cz, zero4, sc);
+        if (!exchange(sc, S & 1, arrived)) {
+          timed_out = true;
+          kf = k + S;
+          goto phase_done;
+        }
+        if (k + S + 3 < nblk) issue_to(k + S + 3, (S + 3) & 3);
+        ready = mbar_test_wait(bars + 8 * ((S + 1) & 3), S == 3 ? par ^ 1 : par);
+        block_softmax_pv<D, false>(cx, S * Cf::STAGE, all, sc, oacc, zacc, m0, m1, l0, l1);
+      }
+      par ^= 1;
+    }
+   }
+  }
 #pragma unroll 1
   for (; k < nblk && !timed_out; ++k) {
     // Wait for this block's bytes.  The wait is bounded: if the copy never completes (which would take
@@ -785,23 +838,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       const RowMask mk = plain ? all : mask_of_block();
       if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
       else block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
-      // The warps of the team each hold the scores over their own channels: exchange and add them in a fixed
-      // order, so that every warp of the team continues with bit-identical scores.  The barrier of
-      // iteration k also tells that every warp is done with the slot of iteration k - 1, which is refilled
-      // after it; a warp whose wait ran out says so here and the whole team stops together.
-      float4* const xb = xch + (k & 1) * (DS * 32);
-      xb[sub * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
-      if (lane == 0) xflag[(k & 1) * DS + sub] = arrived ? 0 : 1;
-      asm volatile("bar.sync %0, %1;\n" ::"r"(1 + team), "r"(32 * DS) : "memory");
-      int bad = 0;
-      sc[0] = sc[1] = sc[2] = sc[3] = 0.f;
-#pragma unroll
-      for (int w = 0; w < DS; ++w) {
-        const float4 part = xb[w * 32 + lane];
-        sc[0] += part.x; sc[1] += part.y; sc[2] += part.z; sc[3] += part.w;
-        bad |= xflag[(k & 1) * DS + w];
-      }
-      if (bad) { timed_out = true; kf = k; break; }
+      if (!exchange(sc, k & 1, arrived)) { timed_out = true; kf = k; break; }
       refill(k + Cf::NST - 1);
       if (plain) block_softmax_pv<D, false>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       else block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);

@@ -103,10 +103,10 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
     span = window or S
     # one launch per step (tq_sdpa_int4_step) wherever it applies: plain decode, contiguous cache, at most 8 query
     # heads per KV head; the tokens present before the timed steps are its stable part
-    # (measured: it wins where one wave of thread blocks serves one sequence with one-warp token blocks -- 1K to 128K
-    # Llama-shaped contexts -- and loses a few per cent on the d = 256 shape and on batches, which keep the calls)
+    # (measured: it wins where one wave of thread blocks serves one sequence -- 1K to 128K Llama-shaped contexts,
+    # the d = 256 shape -- and loses a few per cent on batches, which keep the calls)
     fused = (not SEPARATE_CALLS) and S_q == 1 and window == 0 and not page_tokens and H_q // H_kv <= 8 and (
-        FUSED_EVERYWHERE or (B == 1 and d <= 128))
+        FUSED_EVERYWHERE or (B == 1 and d <= 256))
     C = splits or (tq.tq_auto_splits_step if fused else tq.tq_auto_splits)(B, H_kv, H_q * S_q, d, span)
     o, m, l = tq.alloc_partials(B, H_q * S_q, d, C)
     ws = tq.alloc_step_workspace(B, H_kv, H_q, d, C) if fused else None
@@ -223,7 +223,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--identity-pages", action="store_true", help="paged workloads: pool page i holds page i")
     ap.add_argument("--calls", action="store_true", help="separate append / decode / combine launches everywhere")
-    ap.add_argument("--fused", action="store_true", help="tq_sdpa_int4_step wherever it applies (default: one sequence, d <= 128)")
+    ap.add_argument("--fused", action="store_true", help="tq_sdpa_int4_step wherever it applies (default: one sequence, d <= 256)")
     args = ap.parse_args()
     global IDENTITY_PAGES, SEPARATE_CALLS, FUSED_EVERYWHERE
     IDENTITY_PAGES = args.identity_pages
