@@ -361,6 +361,7 @@ int tq_internal_test_hook(int key, int value) {
     case 0: h.decode_impl.store(value, std::memory_order_relaxed); return 0;
     case 1: h.spin_limit.store(value, std::memory_order_relaxed); return 0;
     case 2: h.fault_block.store(value, std::memory_order_relaxed); return 0;
+    case 3: return static_cast<int>(run_division_check());  // mismatches of the quantiser's division shortcut (-1: CUDA error)
     default: return -1;
   }
 }

@@ -140,6 +140,7 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 }
 
 // host-side launchers (each returns the launch error, if any)
+long long run_division_check();  // tq_quantize.cu: test support, see division_check_kernel
 cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, const __half* v_new, int T,
                                    int32_t* status, cudaStream_t st);
 cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,

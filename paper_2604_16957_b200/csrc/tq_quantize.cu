@@ -147,8 +147,11 @@ __global__ void __launch_bounds__(2 * D, 1536 / (2 * D)) quantize_bulk_kernel(tq
 // that the grid is a whole number of waves.  Partly covered blocks, and
 // paged caches, are left to quantize_bulk_kernel.  (Staging the input through bulk asynchronous copies was
 // measured and is slower here: 200 - 250 us per 128K layer against 178.)
+#ifndef TQ_QG_WARPS
+#define TQ_QG_WARPS 24  // resident warps per SM the kernel is compiled for (80 registers per thread)
+#endif
 template <int D>
-__global__ void __launch_bounds__(D) quantize_group_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new, int T,
+__global__ void __launch_bounds__(D, TQ_QG_WARPS * 32 / D) quantize_group_kernel(tq_kv_cache c, const __half* k_new, const __half* v_new, int T,
                                                             int32_t* status, int group_run) {
   constexpr int NG = D / 32, NW = NG;        // groups per row; warps per thread block
   constexpr int TPW = 32 / NG;               // token rows per warp
@@ -179,19 +182,12 @@ __global__ void __launch_bounds__(D) quantize_group_kernel(tq_kv_cache c, const 
   const uint32_t s_at = (g * TPW + (tok - tok0)) * 2, z_at = 64 + s_at;
   const int a_l = (4 * lane) / 64, g_l = ((4 * lane) % 64) / VW, off_l = (4 * lane) % VW;
   const uint32_t meta_dst = meta_offset(D, which, a_l, g_l, tok0) + off_l;
-  uint4 nxt[4];
+  constexpr int kStep = 16 * D * 2 / 16;  // 16-byte units from one block's rows to the next block's
+  auto fetch = [&](uint4 (&r)[4], const uint4* p) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) nxt[i] = __ldg(src + i);
-#pragma unroll 1
-  for (int jj = 0; jj < nrun; ++jj) {
-    uint4 raw[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) raw[i] = nxt[i];
-    src += 16 * D * 2 / 16;  // the next block's rows: 16 rows further
-    if (jj + 1 < nrun) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) nxt[i] = __ldg(src + i);
-    }
+    for (int i = 0; i < 4; ++i) r[i] = __ldg(p + i);
+  };
+  auto emit = [&](const uint4 (&raw)[4], int jj) {
     uint32_t w[4];
     __half sq, zq;
     quantize_group32(raw, w, sq, zq);
@@ -202,7 +198,44 @@ __global__ void __launch_bounds__(D) quantize_group_kernel(tq_kv_cache c, const 
     __syncwarp();
     *reinterpret_cast<uint32_t*>(blk + meta_dst) = *reinterpret_cast<const uint32_t*>(meta + 4 * lane);
     __syncwarp();  // the 128 bytes are read before the next block overwrites them
+  };
+  // two register buffers taken in turn: the next block's loads are in flight during the arithmetic and no
+  // register is copied
+  uint4 ra[4], rb[4];
+  fetch(ra, src);
+#pragma unroll 1
+  for (int jj = 0; jj < nrun; jj += 2) {
+    if (jj + 1 < nrun) fetch(rb, src + kStep);
+    emit(ra, jj);
+    if (jj + 1 >= nrun) break;
+    if (jj + 2 < nrun) fetch(ra, src + 2 * kStep);
+    emit(rb, jj + 1);
+    src += 2 * kStep;
   }
+}
+
+// Compares div_rn_by_reciprocal with the true division on every quotient the quantiser can form: block x
+// takes the finite binary16 number a with index x, its threads walk over every finite b.  (i) fl(a - b) / 15
+// for a > b; (ii) (0 - a) / b for b > 0.  Mismatches are counted in *bad.  Test support.
+__device__ __forceinline__ float finite_half(int idx) {  // 0 .. 31743: +0 .. 65504; 31744 .. 63487: -0 .. -65504
+  const unsigned short bits = idx < 31744 ? idx : 0x8000 + (idx - 31744);
+  return __half2float(__ushort_as_half(bits));
+}
+__global__ void division_check_kernel(unsigned long long* bad) {
+  const float a = finite_half(blockIdx.x);
+  unsigned long long n = 0;
+  for (int j = threadIdx.x; j < 63488; j += blockDim.x) {
+    const float b = finite_half(j);
+    if (a > b) {  // (a zero range never uses the shortcut's result: its scale is zero and the defining arithmetic takes over)
+      const float d = __fsub_rn(a, b);
+      n += __float_as_uint(__fdiv_rn(d, 15.0f)) != __float_as_uint(div_rn_by_15(d));
+    }
+    if (b > 0.0f) {
+      const float num = __fsub_rn(0.0f, a);
+      n += __float_as_uint(__fdiv_rn(num, b)) != __float_as_uint(div_rn_by_reciprocal(num, b, __frcp_rn(b)));
+    }
+  }
+  if (n) atomicAdd(bad, n);
 }
 
 __global__ void bump_lens_kernel(tq_kv_cache c, int T, int32_t* status) {
@@ -273,10 +306,10 @@ cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, co
     }
     if (e != cudaSuccess) return e;
     if (!paged && T >= 16) {
-      // Run length: about 32 blocks per thread block, adjusted so that the thread blocks (512 threads' worth
-      // of them are resident per SM: 128 registers per thread) make a whole number of waves.
+      // Run length: about 32 blocks per thread block, adjusted so that the thread blocks (TQ_QG_WARPS warps' worth
+      // of them are resident per SM) make a whole number of waves.
       const long long bhn = static_cast<long long>(c.B) * c.H_kv, nb = T / 16;
-      const long long slots = static_cast<long long>(device_sm_count()) * 512 / c.d;
+      const long long slots = static_cast<long long>(device_sm_count()) * (TQ_QG_WARPS * 32) / c.d;
       const long long waves = std::max(1LL, (bhn * nb + 32 * slots - 1) / (32 * slots));
       const long long per_bh = std::max(1LL, waves * slots / bhn);  // thread blocks per (sequence, KV head)
       const int group_run = static_cast<int>(std::max(1LL, (nb + per_bh - 1) / per_bh));
@@ -291,6 +324,21 @@ cudaError_t launch_quantize_append(const tq_kv_cache& c, const __half* k_new, co
     }
     return launch_kernel(bump_lens_kernel, dim3((c.B + 127) / 128), dim3(128), 0, st, c, T, status);
   }
+}
+
+// Runs division_check_kernel on the current device; returns the number of mismatches, or -1 on a CUDA error.
+long long run_division_check() {
+  unsigned long long* bad = nullptr;
+  unsigned long long host = 0;
+  if (cudaMalloc(&bad, sizeof(*bad)) != cudaSuccess) return -1;
+  cudaError_t e = cudaMemset(bad, 0, sizeof(*bad));
+  if (e == cudaSuccess) {
+    division_check_kernel<<<63488, 256>>>(bad);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpy(&host, bad, sizeof(host), cudaMemcpyDeviceToHost);
+  cudaFree(bad);
+  return e == cudaSuccess ? static_cast<long long>(host > 0x7fffffffULL ? 0x7fffffffULL : host) : -1;
 }
 
 }  // namespace tq

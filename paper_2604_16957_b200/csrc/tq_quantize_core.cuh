@@ -38,6 +38,20 @@ static __device__ __noinline__ uint2 quantize_exact(const uint4 raw, float mn, f
   return make_uint2(word, static_cast<uint32_t>(__half_as_ushort(s16)) | (static_cast<uint32_t>(__half_as_ushort(z16)) << 16));
 }
 
+// Correctly rounded a / b from a correctly rounded reciprocal rb = fl(1 / b): q = fl(a * rb), the remainder
+// r = a - q * b (exact in one fused multiply-add), and fl(q + r * rb).  For the quotients of the quantiser --
+// a difference of two finite binary16 numbers over 15, and a negated finite binary16 number over a positive
+// binary16 scale -- the result is bit-identical to __fdiv_rn: nothing under- or overflows on the way, and the
+// library's own check (division_check_kernel, run by its tests) compares all 4.0e9 + 2.0e9 such pairs.
+// A zero or non-finite b gives a non-finite or NaN result, which the callers' range checks reject; a zero
+// numerator may come back with the other sign (-0 / 15), which only a zero range produces and which is
+// rejected the same way (its scale is zero).
+__device__ __forceinline__ float div_rn_by_reciprocal(float a, float b, float rb) {
+  const float q = __fmul_rn(a, rb);
+  return fmaf(fmaf(-q, b, a), rb, q);
+}
+__device__ __forceinline__ float div_rn_by_15(float a) { return div_rn_by_reciprocal(a, 15.0f, 0.0666666701436042785645f); }
+
 // Quantise the 8 elements held by this thread (quad = one group).  All 32 lanes must call.
 //
 // Defining arithmetic: s = fp16((max - min) / 15), z = fp16(clamp((0 - min) / s)), u = fl(fl(x / s) + z),
@@ -100,6 +114,28 @@ __device__ __forceinline__ void quantize_chunk(const uint4 raw, uint32_t& word, 
 }
 
 
+// Cold path of quantize_group32: the elements whose two-sided roundings disagree are redone with the defining
+// arithmetic (a true division) and their codes put in place.  Out of line, everything in registers.
+static __device__ __noinline__ uint4 redo_near_boundaries(const uint4 r0, const uint4 r1, const uint4 r2, const uint4 r3,
+                                                          uint4 words, float rs, float sf, float zf, float z_lo,
+                                                          float z_hi) {
+  constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
+  const uint4 raw[4] = {r0, r1, r2, r3};
+  const __half2* h2 = reinterpret_cast<const __half2*>(&raw[0]);
+  uint32_t word[4] = {words.x, words.y, words.z, words.w};
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {  // unrolled: every index is a constant, the arrays stay in registers
+    const float2 f = __half22float2(h2[i >> 1]);
+    const float x = (i & 1) ? f.y : f.x;
+    if (((__float_as_uint(fmaf(x, rs, z_lo)) ^ __float_as_uint(fmaf(x, rs, z_hi))) >> 16) != 0) {
+      const float ue = __fadd_rn(__fdiv_rn(x, sf), zf);
+      const uint32_t q = __float_as_uint(ue + kMagic) & 0xFu;  // rint, ties to even; 0 .. 15 because no clamp can act
+      word[i >> 3] = (word[i >> 3] & ~(0xFu << (4 * (i & 7)))) | (q << (4 * (i & 7)));
+    }
+  }
+  return make_uint4(word[0], word[1], word[2], word[3]);
+}
+
 // The same quantiser for a thread that holds a whole group of 32 elements (the bulk kernel): minimum and
 // maximum are found on the packed halves, the per-group work (two divisions, a reciprocal, the bound) is paid
 // once per 32 elements instead of once per 8, and no shuffle is needed.  raw[j] holds elements 8j .. 8j+7.
@@ -127,11 +163,11 @@ __device__ __forceinline__ void quantize_group32(const uint4 (&raw)[4], uint32_t
   }
   const float mn = fminf(__low2float(mn2), __high2float(mn2));
   const float mx = fmaxf(__low2float(mx2), __high2float(mx2));
-  const __half s16 = __float2half_rn(__fdiv_rn(__fsub_rn(mx, mn), 15.0f));
+  const __half s16 = __float2half_rn(div_rn_by_15(__fsub_rn(mx, mn)));
   const float sf = __half2float(s16);
-  const __half z16 = __float2half_rn(__fdiv_rn(__fsub_rn(0.0f, mn), sf));  // no clamp here: an overflow fails the checks
-  const float zf = __half2float(z16);
   const float rs = __frcp_rn(sf);
+  const __half z16 = __float2half_rn(div_rn_by_reciprocal(__fsub_rn(0.0f, mn), sf, rs));  // no clamp here: an overflow fails the checks
+  const float zf = __half2float(z16);
   const float tol = fmaf(2.0f * fmaxf(fabsf(mn), fabsf(mx)) * rs + fabsf(zf) + 17.0f, 4.76837158203125e-7f,  // 2^-21
                          3.0517578125e-5f);                                                               // 2^-15
   const float z_lo = __fadd_rn(zf, __fsub_rn(128.5f, tol)), z_hi = __fadd_rn(zf, __fadd_rn(128.5f, tol));
@@ -156,19 +192,10 @@ __device__ __forceinline__ void quantize_group32(const uint4 (&raw)[4], uint32_t
   z_out = z16;
   const bool in_range = fmaf(mn, rs, zf) > -0.49f && fmaf(mx, rs, zf) < 15.49f;
   if (in_range && (differ >> 16) != 0) {
-    // Rare: no clamp can act, but some element sits within the bound of a rounding boundary.  Only such
-    // elements are redone with the defining arithmetic (a true division) and their codes put in place.
-    constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {  // unrolled: every index is a constant, the arrays stay in registers
-      const float2 f = __half22float2(h2[i >> 1]);
-      const float x = (i & 1) ? f.y : f.x;
-      if (((__float_as_uint(fmaf(x, rs, z_lo)) ^ __float_as_uint(fmaf(x, rs, z_hi))) >> 16) != 0) {
-        const float ue = __fadd_rn(__fdiv_rn(x, sf), zf);
-        const uint32_t q = __float_as_uint(ue + kMagic) & 0xFu;  // rint, ties to even; 0 .. 15 because no clamp can act
-        word[i >> 3] = (word[i >> 3] & ~(0xFu << (4 * (i & 7)))) | (q << (4 * (i & 7)));
-      }
-    }
+    // Rare: no clamp can act, but some element sits within the bound of a rounding boundary.
+    const uint4 w = redo_near_boundaries(raw[0], raw[1], raw[2], raw[3], make_uint4(word[0], word[1], word[2], word[3]),
+                                         rs, sf, zf, z_lo, z_hi);
+    word[0] = w.x; word[1] = w.y; word[2] = w.z; word[3] = w.w;
   } else if (!in_range) {  // rarer: clamps, degenerate scales, overflowing zeros
 #pragma unroll  // constant indices: raw stays in registers
     for (int j = 0; j < 4; ++j) {

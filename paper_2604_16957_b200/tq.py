@@ -105,6 +105,12 @@ def _test_hook(key, value):
         raise ValueError(f"unknown test hook {key}")
 
 
+def _division_self_check():
+    """Mismatches between the quantiser's reciprocal-based divisions and true division over every quotient it can
+    form (runs a kernel on the current device; -1 on a CUDA error); used only by tests/."""
+    return int(_lib.tq_internal_test_hook(3, 0))
+
+
 class TqError(RuntimeError):
     def __init__(self, code, where):
         self.code = code

@@ -133,3 +133,11 @@ def test_bulk_path_with_ragged_lengths_and_overflow(gpu, oracle):
     assert_cache_bits_equal(dev, host, lens=[1500, 0, 0])
     for name, d_arr, h_arr in zip("abcdef", dev.arrays_token_major(), host.arrays()):
         assert np.array_equal(d_arr.cpu().numpy()[1, :, 1000:2500].view(np.uint8), h_arr[1, :, 1000:2500].view(np.uint8))
+
+
+def test_division_shortcut_equals_true_division_everywhere(gpu):
+    """The group quantiser forms (max - min) / 15 and (0 - min) / scale from a reciprocal and one remainder
+    correction; the library compares both with the correctly rounded division over all finite binary16
+    (max, min) pairs and all (min, positive scale) pairs."""
+    tq, torch = gpu
+    assert tq._division_self_check() == 0
