@@ -390,6 +390,35 @@ struct StepArgs {
   int wait_cycles, fault_blk;
 };
 
+// Fused step: one warp quantises the new token's K and V rows of one KV head (Eq. 2-3) into row `row` of the
+// cache block `blk`.  Out of line: its registers are not the block loop's.
+template <int D>
+__device__ __noinline__ void quantize_new_row(uint8_t* blk, int row, const __half* k_row, const __half* v_row) {
+  const int lane = threadIdx.x & 31;
+  constexpr int CPR = D / 8;  // 8-element chunks per row; K chunks first, then V
+#pragma unroll
+  for (int i0 = 0; i0 < 2 * CPR; i0 += 32) {
+    const int i = i0 + lane;
+    const bool on = i < 2 * CPR;
+    const int which = i >= CPR ? 1 : 0, cc = i - which * CPR;
+    uint4 raw = make_uint4(0, 0, 0, 0);
+    if (on) raw = *reinterpret_cast<const uint4*>((which ? v_row : k_row) + cc * 8);
+    uint32_t word;
+    __half sq, zq;
+    quantize_chunk(raw, word, sq, zq);
+    if (on) {
+      *reinterpret_cast<uint32_t*>(blk + code_offset(D, which, row, cc * 4)) = word;
+      if ((cc & 3) == 0) {
+        *reinterpret_cast<__half*>(blk + meta_offset(D, which, 0, cc >> 2, row)) = sq;
+        *reinterpret_cast<__half*>(blk + meta_offset(D, which, 1, cc >> 2, row)) = zq;
+      }
+    }
+  }
+  // the row is fetched back by this block's bulk copies (asynchronous proxy): order them after the stores
+  __threadfence();
+  asm volatile("fence.proxy.async;\n" ::: "memory");
+}
+
 // GEN = the general form: a sliding window (Appendix A) and / or several query tokens per sequence
 // (S_q > 1, the grid's S_q factor in Appendix A).  With S_q query tokens the "heads" of a KV head are its
 // G * S_q (query token, head) pairs, v = s * G + g, packed into MMA columns like plain heads; query token s
@@ -447,31 +476,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       if (old < cache.S_cap) n = old + 1;
       else if (c == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status) atomicOr(status, TQ_STATUS_CACHE_FULL);
       if (c == C - 1 && n > old) {  // one head tile per KV head in this form (checked on the host)
-        if (warp == 0) {
-          uint8_t* const blk = const_cast<uint8_t*>(head_blocks) + static_cast<size_t>(old >> 4) * Cf::STAGE;
-          constexpr int CPR = D / 8;  // 8-element chunks per row; K chunks first, then V
-#pragma unroll
-          for (int i0 = 0; i0 < 2 * CPR; i0 += 32) {
-            const int i = i0 + lane;
-            const bool on = i < 2 * CPR;
-            const int which = i >= CPR ? 1 : 0, cc = i - which * CPR;
-            uint4 raw = make_uint4(0, 0, 0, 0);
-            if (on) raw = *reinterpret_cast<const uint4*>((which ? sa.v_new : sa.k_new) + (static_cast<long long>(b) * cache.H_kv + kvh) * D + cc * 8);
-            uint32_t word;
-            __half sq, zq;
-            quantize_chunk(raw, word, sq, zq);
-            if (on) {
-              *reinterpret_cast<uint32_t*>(blk + code_offset(D, which, old & 15, cc * 4)) = word;
-              if ((cc & 3) == 0) {
-                *reinterpret_cast<__half*>(blk + meta_offset(D, which, 0, cc >> 2, old & 15)) = sq;
-                *reinterpret_cast<__half*>(blk + meta_offset(D, which, 1, cc >> 2, old & 15)) = zq;
-              }
-            }
-          }
-          // the row is fetched back by this block's bulk copies (asynchronous proxy): order them after the stores
-          __threadfence();
-          asm volatile("fence.proxy.async;\n" ::: "memory");
-        }
+        if (warp == 0)
+          quantize_new_row<D>(const_cast<uint8_t*>(head_blocks) + static_cast<size_t>(old >> 4) * Cf::STAGE, old & 15,
+                              sa.k_new + (static_cast<long long>(b) * cache.H_kv + kvh) * D,
+                              sa.v_new + (static_cast<long long>(b) * cache.H_kv + kvh) * D);
         __syncthreads();
       }
       if (threadIdx.x == 0) {

@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 
 from paper_2604_16957_b200 import inputs as I
-from util import assert_attention_close, device_cache, oracle_cache
+from util import MAX_ABS_TOL, assert_attention_close, device_cache, oracle_cache
 
 pytestmark = pytest.mark.gpu
 
@@ -286,4 +286,37 @@ def test_fused_steps_back_to_back(gpu, oracle, use_graph):
         if i in (0, 1, 4, 5, 10, steps - 1):
             assert_attention_close(got[i], oracle.attention(host, qn[i], sh.alpha), f"step {i}")
     assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
+    assert_cache_bits_equal(dev, host)
+
+
+@pytest.mark.parametrize("S", [32768, 131072])
+def test_config3_long_context_layer_through_the_one_launch_step(gpu, oracle, S):
+    """One Llama-70B-shaped layer at 32K and at 128K tokens through tq_sdpa_int4_step exactly as the benchmark
+    launches it (library-chosen split count, the tokens present before the step declared stable, the new token
+    appended by the same launch; fp32 output on the first step, fp16 on the second): the cache bit for bit, then every query head against the oracle."""
+    from util import assert_cache_bits_equal
+    tq, torch = gpu
+    sh = I.LLAMA
+    S_cap = S + 16
+    host, dev = _step_setup(tq, torch, oracle, sh, S, S_cap, [S], 30 + S // 32768)
+    C = tq.tq_auto_splits_step(sh.B, sh.H_kv, sh.H_q, sh.d, S_cap)
+    ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, C)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for step, dt in enumerate((torch.float32, torch.float16)):   # the second step's stable part ends inside the block the first wrote to
+        out = torch.zeros((sh.B, sh.H_q, sh.d), dtype=dt, device="cuda")
+        kn, vn = I.make_kv(sh, 1, 31, stream=1 + step)
+        qn = I.make_q(sh, 31, stream=step)
+        tq.tq_sdpa_int4_step(dev, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(qn).cuda(),
+                             sh.alpha, C, S, ws, out, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        host.append(kn, vn)
+        assert dev.seq_lens.cpu().tolist() == [S + step + 1]
+        ref = oracle.attention(host, qn, sh.alpha)
+        got = out.float().cpu().numpy()
+        if dt == torch.float32:
+            mx, rel = assert_attention_close(got, ref, f"S={S} step {step}")
+            print(f"llama {S} + 1 through the step entry, C={C}: max-abs {mx:.2e} rel-L2 {rel:.2e}")
+        else:
+            assert np.abs(got - ref).max() <= MAX_ABS_TOL + np.abs(ref).max() * 2.0 ** -11, f"S={S} step {step}"
     assert_cache_bits_equal(dev, host)
