@@ -201,14 +201,27 @@ __global__ void __launch_bounds__(D, TQ_QG_WARPS * 32 / D) quantize_group_kernel
   };
   // two register buffers taken in turn: the next block's loads are in flight during the arithmetic and no
   // register is copied
+#ifndef TQ_QG_PF
+#define TQ_QG_PF 2  // blocks ahead of the register loads that are prefetched into L2 (0: none; measured 128.7 / 125.6 / 129.5 / 140.0 us for 0 / 2 / 3 / 5)
+#endif
+  auto ahead = [&](const uint4* p) {  // this lane's 64 bytes of a later block, into L2
+    if (TQ_QG_PF > 0) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p));
+  };
   uint4 ra[4], rb[4];
   fetch(ra, src);
+  if (TQ_QG_PF > 1) {
+#pragma unroll
+    for (int a = 2; a <= TQ_QG_PF; ++a)
+      if (a < nrun) ahead(src + a * kStep);
+  }
 #pragma unroll 1
   for (int jj = 0; jj < nrun; jj += 2) {
     if (jj + 1 < nrun) fetch(rb, src + kStep);
+    if (jj + 1 + TQ_QG_PF < nrun) ahead(src + (1 + TQ_QG_PF) * kStep);
     emit(ra, jj);
     if (jj + 1 >= nrun) break;
     if (jj + 2 < nrun) fetch(ra, src + 2 * kStep);
+    if (jj + 2 + TQ_QG_PF < nrun) ahead(src + (2 + TQ_QG_PF) * kStep);
     emit(rb, jj + 1);
     src += 2 * kStep;
   }
