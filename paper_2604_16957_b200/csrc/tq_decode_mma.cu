@@ -72,7 +72,10 @@ struct Cfg {
   static constexpr int SWZ_SHIFT = NG == 2 ? 2 : (NG == 4 ? 1 : 0);  // chunk' = chunk ^ ((tok >> SHIFT) & (NG - 1))
   static constexpr int SZ = kBlk * NG * 2;          // bytes of one scale or zero array per stage
   static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1280 / 2560 / 5120 / 10240 bytes
-  static constexpr int NST = 4;                     // stages in a ring (power of two)
+#ifndef TQ_NST
+#define TQ_NST 4
+#endif
+  static constexpr int NST = D == 128 ? TQ_NST : 4;  // stages in a ring
   // Head dimensions above 128 are split over DS warps (a "team") that work on the same token block, each
   // on DW = 128 channels: the accumulators of one warp stay within 128 registers per thread, so two
   // blocks fit an SM at every head dimension.  A team owns one ring; the kernel has NTEAM teams.
@@ -145,7 +148,7 @@ struct WarpCtx {
   uint32_t ksz_lane, vsz_lane;
   uint32_t vz_lane, vs2_lane;  // row addresses of the V scale / zero load of the zero-point MMA and of the scale loads
   uint32_t kz_lane;            // row address of the scale / zero load that feeds the zero-point MMA of the scores
-  uint32_t fl_m;               // half2 lane flag of that MMA's A operand: 0 for tid4 < 2 (hi parts), -1 otherwise (lo parts)
+  uint32_t keep;               // all ones, except 0 in the lanes of row 4 of the P.V zero-point MMA (see block_softmax_pv)
   float cs;
   int gid;
 };
@@ -184,19 +187,18 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
   if constexpr (KZ<D>::on) {
     // Zero-point term of the scores by one MMA: sum_g (s_g z_g) * qsum_g with the product s * z split
     // exactly into an fp16 pair (hi = rn(s z), lo = s z - hi by a fused multiply-add) and qsum into
-    // hi + lo as well; k slots 0-3 hi x hi, 4-7 lo x hi, 8-11 hi x lo (lo x lo is below 2^-22 of the term).
+    // hi + lo as well.  k slots 0-7 carry the hi parts of groups 0 1 2 3 0 1 2 3, slots 8-15 the lo parts in
+    // the same order; the B rows (qz, the same register for both halves) hold the hi parts of the group sums in
+    // slots 0-3 and 8-11 and their lo parts in 4-7 and 12-15: hi x hi + hi x lo + lo x hi + lo x lo.
     // The transposing load hands lane (gid, tid4) the half2 (x[g][token], x[g+1][token]) of groups
     // g = 2 * (tid4 & 1): scales of tokens gid, gid + 8, then zeros of the same.
     uint32_t r[4];
     ldmatrix_x4_trans(r, cx.kz_lane + st_off);
     const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
-    const uint32_t a0 = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hmul2(pa, u32_as_h2(cx.fl_m))));
-    const uint32_t a1 = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hmul2(pb, u32_as_h2(cx.fl_m))));
-    // k slots 8-15: hi parts again for the lanes whose B rows hold the lo parts of the group sums; the other
-    // lanes' B rows are zero, so whatever finite value they supply does not count
-    const uint32_t a2 = h2_as_u32(pa), a3 = h2_as_u32(pb);
+    const uint32_t la = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hneg2(pa)));
+    const uint32_t lb = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hneg2(pb)));
     float accz[4];
-    mma16816_first(accz, a0, a1, a2, a3, qz[0], qz[1], zero4);
+    mma16816_first(accz, h2_as_u32(pa), h2_as_u32(pb), la, lb, qz[0], qz[0], zero4);
     // scales of all four groups for tokens gid, gid + 8: matrices (g0 g1 | tokens 0-7), (g0 g1 | 8-15), (g2 g3 | ..)
     ldmatrix_x4_trans(ksz, cx.ksz_lane + st_off);
     sc[0] = accz[0] * cz[0]; sc[1] = accz[1] * cz[1]; sc[2] = accz[2] * cz[0]; sc[3] = accz[3] * cz[1];
@@ -284,8 +286,10 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     const float f0 = ex2(m0 - n0), f1 = ex2(m1 - n1);  // m starts at -1e30: the first factor underflows to 0
     m0 = n0;
     m1 = n1;
-    l0 *= f0;
-    l1 *= f1;
+    if constexpr (!KZ<D>::on) {
+      l0 *= f0;
+      l1 *= f1;
+    }
 #pragma unroll
     for (int i = 0; i < Cfg<D>::DW / 16; ++i) {
       oacc[i][0] *= f0; oacc[i][1] *= f1; oacc[i][2] *= f0; oacc[i][3] *= f1;
@@ -301,8 +305,10 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     d0 = a0 - m0; d1 = a1 - m1; d2 = a2 - m0; d3 = a3 - m1;
   }
   const float p0 = ex2(d0), p1 = ex2(d1), p2 = ex2(d2), p3 = ex2(d3);  // ex2(-inf) = 0 for masked tokens
-  l0 += p0 + p2;
-  l1 += p1 + p3;
+  if constexpr (!KZ<D>::on) {  // (otherwise the denominator comes out of the zero-point MMA below)
+    l0 += p0 + p2;
+    l1 += p1 + p3;
+  }
   // P^T as B fragments: (tokens 2*tid4, 2*tid4+1 | head gid) and (tokens 8+2*tid4, 9+2*tid4 | head gid)
   const uint32_t pt0 = movmatrix_trans(h2_as_u32(__floats2half2_rn(p0, p1)));
   const uint32_t pt1 = movmatrix_trans(h2_as_u32(__floats2half2_rn(p2, p3)));
@@ -323,7 +329,12 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
     const uint32_t la = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hneg2(pa)));
     const uint32_t lb = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hneg2(pb)));
-    mma16816(zacc[0], h2_as_u32(pa), la, h2_as_u32(pb), lb, pt0, pt1);
+    // Rows 4-7 repeat the groups of rows 0-3 and are not read back, so row 4 is given ones instead: its
+    // accumulators become sum_tok fp16(P)[tok][head], the softmax denominator (of exactly the weights the
+    // numerator uses), at no instruction beyond the two selects.
+    constexpr uint32_t kOnes = 0x3C003C00u;  // half2 (1, 1)
+    const uint32_t ha = (h2_as_u32(pa) & cx.keep) | (~cx.keep & kOnes), hb = (h2_as_u32(pb) & cx.keep) | (~cx.keep & kOnes);
+    mma16816(zacc[0], ha, la, hb, lb, pt0, pt1);
     uint32_t vs[4];
 #pragma unroll
     for (int g = 0; g < NGW; ++g) {
@@ -563,7 +574,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     }
   };
 
-  auto issue = [&](int n) { issue_to(n, n & (Cf::NST - 1)); };
+  auto issue = [&](int n) { issue_to(n, n % Cf::NST); };
 
   // start streaming: the first stages are in flight while q is turned into fragments
 #pragma unroll
@@ -631,8 +642,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     const __half2 hi = __floats2half2_rn(sa, sb);
     const float2 hf = __half22float2(hi);
     const __half2 lo = __floats2half2_rn(sa - hf.x, sb - hf.y);
-    qz[0] = h2_as_u32(hi);
-    qz[1] = tid4 < 2 ? h2_as_u32(lo) : 0u;
+    qz[0] = qz[1] = tid4 < 2 ? h2_as_u32(hi) : h2_as_u32(lo);
     cz[0] = __shfl_sync(0xffffffffu, up24, (2 * tid4) * 4);
     cz[1] = __shfl_sync(0xffffffffu, up24, (2 * tid4 + 1) * 4);
   }
@@ -666,14 +676,13 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // per-lane byte offsets inside a stage: ldmatrix row addresses of the code, scale and zero fragments of
   // this warp's channel groups sub * NGW .. (see block_scores / block_softmax_pv)
   WarpCtx<D> cx;
-  cx.cs = cs; cx.gid = gid;
+  cx.cs = cs; cx.gid = gid; cx.keep = gid == 4 ? 0u : 0xFFFFFFFFu;
   cx.ksz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32 + sub * NGW * 32;
   if constexpr (KZ<D>::on) {
     cx.ksz_lane = ring_s + 2 * Cf::PK + (2 * (lane >> 4) + (lane & 1)) * 32 + ((lane >> 3) & 1) * 16 + sub * NGW * 32;
     cx.kz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32 + sub * NGW * 32;
-    cx.fl_m = tid4 < 2 ? 0u : 0xBC00BC00u;  // half2 (0, 0) | (-1, -1)
   } else {
-    cx.kz_lane = cx.fl_m = 0;
+    cx.kz_lane = 0;
   }
   cx.vsz_lane = ring_s + 2 * Cf::PK + (3 - ((lane >> 3) & 1)) * Cf::SZ + (lane >> 4) * 16 + sub * NGW * 32;
   cx.vz_lane = ring_s + 2 * Cf::PK + (2 + (lane >> 4)) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 3) * 32 + sub * NGW * 32;
@@ -741,35 +750,35 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
    if (phase == 0) {
     // Full blocks four at a time: ring slot, barrier and stage offsets are constants of each of the four
     // copies of the block step, so the loop carries no slot arithmetic.
-    static_assert(Cf::NST == 4, "the unrolled loop walks a ring of four slots");
+    constexpr int NST = Cf::NST;
     const RowMask all{kBlk, 0, kBlk, 0, kBlk};
     uint32_t par = 0;
     // The barrier of the next block is probed one block ahead (the probe's latency then hides behind a block
     // of arithmetic); only a probe that came back negative is followed by the blocking wait.  No warp-wide
     // synchronisation is needed before a slot is refilled: its last readers were the warp-collective loads
     // of the previous block, whose results the MMAs issued since then have already consumed.
-    bool ready = k + 4 <= nfull ? mbar_test_wait(bars, 0) : false;
+    bool ready = k + NST <= nfull ? mbar_test_wait(bars, 0) : false;
 #ifdef TQ_PROBE_MATH_ONLY
     // Timing probe (results are meaningless): the three copies issued above are awaited here, the fourth
     // slot is cleared, and the unrolled loop then runs its arithmetic on whatever the ring holds without
     // waiting for or issuing any copy; the blocks it leaves over are skipped.
     for (int s = 0; s < Cf::NST - 1; ++s)
       if (s < nblk) wait_stage(bars + 8 * s, 0);
-    for (int i = lane; i < Cf::STAGE / 4; i += 32) reinterpret_cast<uint32_t*>(ring + 3 * Cf::STAGE)[i] = 0;
+    for (int i = lane; i < Cf::STAGE / 4; i += 32) reinterpret_cast<uint32_t*>(ring + (NST - 1) * Cf::STAGE)[i] = 0;
     __syncwarp();
     ready = true;
 #endif
-    for (; k + 4 <= nfull; k += 4) {
+    for (; k + NST <= nfull; k += NST) {
 #pragma unroll
-      for (int S = 0; S < 4; ++S) {
+      for (int S = 0; S < NST; ++S) {
         if (!ready && !wait_stage(bars + 8 * S, par, wait_limit)) {  // cold: leave the loops, keep the phase order
           timed_out = true;
           kf = k + S;
           goto phase_done;
         }
 #ifndef TQ_PROBE_MATH_ONLY
-        if (k + S + 3 < nblk) issue_to(k + S + 3, (S + 3) & 3);
-        ready = mbar_test_wait(bars + 8 * ((S + 1) & 3), S == 3 ? par ^ 1 : par);
+        if (k + S + NST - 1 < nblk) issue_to(k + S + NST - 1, (S + NST - 1) % NST);
+        ready = mbar_test_wait(bars + 8 * ((S + 1) % NST), S == NST - 1 ? par ^ 1 : par);
 #endif
 #ifndef TQ_PROBE_COPIES_ONLY
         float sc[4];
@@ -814,14 +823,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   for (; k < nblk && !timed_out; ++k) {
     // Wait for this block's bytes.  The wait is bounded: if the copy never completes (which would take
     // a bad pointer), the warp flags the status word and stops consuming.
-    const bool arrived = wait_stage(bars + 8 * (k & (Cf::NST - 1)), (k / Cf::NST) & 1, wait_limit);
+    const bool arrived = wait_stage(bars + 8 * (k % Cf::NST), (k / Cf::NST) & 1, wait_limit);
     if (DS == 1) {
       if (!arrived) { timed_out = true; kf = k; break; }
       __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
       refill(k + Cf::NST - 1);
     }
-    const uint32_t st_s = (k & (Cf::NST - 1)) * Cf::STAGE;
-    const uint8_t* st = ring + (k & (Cf::NST - 1)) * Cf::STAGE;
+    const uint32_t st_s = (k % Cf::NST) * Cf::STAGE;
+    const uint8_t* st = ring + (k % Cf::NST) * Cf::STAGE;
     const bool plain = GEN ? static_cast<unsigned>(k - nhead) < nplain : k < nfull;
     auto mask_of_block = [&]() {
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
@@ -859,15 +868,20 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     // full bounded time to land before the block reuses the memory, then report.  The partial written below
     // is not valid in that case.
     for (int n = kf; n < kf + Cf::NST - 1 && n < nblk; ++n)
-      wait_stage(bars + 8 * (n & (Cf::NST - 1)), (n / Cf::NST) & 1);
+      wait_stage(bars + 8 * (n % Cf::NST), (n / Cf::NST) & 1);
     if (lane == 0 && status) atomicOr(status, TQ_STATUS_TIMEOUT);
   }
 
   // ---------------- merge the teams and write the normalised partial (o_c, m_c, l_c)
+  if constexpr (KZ<D>::on) {  // row 4 of the zero-point accumulator holds the denominators of heads 2*tid4, 2*tid4+1
+    l0 = __shfl_sync(0xffffffffu, zacc[0][0], 16 + tid4);
+    l1 = __shfl_sync(0xffffffffu, zacc[0][1], 16 + tid4);
+  } else {
 #pragma unroll
-  for (int off = 4; off <= 16; off <<= 1) {
-    l0 += __shfl_xor_sync(0xffffffffu, l0, off);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+    for (int off = 4; off <= 16; off <<= 1) {
+      l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+    }
   }
   __syncthreads();  // every warp is done with its ring; the memory is reused below
   // layout (floats): wml[NTEAM][16] = each team's m[8], l[8] | slab[NTEAM][D][kChPitch] | tb[8][kRowPitch]
