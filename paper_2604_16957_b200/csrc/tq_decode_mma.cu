@@ -139,6 +139,8 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// bytes 1 and 3 of w moved to bytes 0 and 2, the others cleared: (w >> 8) & 0x00FF00FF in one instruction
+__device__ __forceinline__ uint32_t upper_bytes(uint32_t w) { return __byte_perm(w, 0u, 0x4341); }
 __device__ __forceinline__ uint32_t h2_as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ __half2 u32_as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
 
@@ -208,6 +210,8 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
       const uint32_t w8 = kw[g / 2][2 * (g % 2) + 1];            // token gid + 8
       float acc[4];
       mma16816_first(acc, w0 & kMaskLo, w8 & kMaskLo, w0 & kMaskHi, w8 & kMaskHi, qf[g][0], qf[g][1], zero4);
+      // (The whole-byte operand of the P.V side is not used here: paired with q3 / 16 it needs q2 - q3 / 16 for
+      // nibble 2, whose fp16 rounding reaches the scores -- measured 1e-3 relative L2 at 64K, 1.8e-3 worst head.)
       const uint32_t y0 = w0 >> 8, y8 = w8 >> 8;
       mma16816(acc, y0 & kMaskLo, y8 & kMaskLo, y0 & kMaskHi, y8 & kMaskHi, qf[g][2], qf[g][3]);
       const __half2 slo = u32_as_h2(ksz[2 * (g / 2)]), shi = u32_as_h2(ksz[2 * (g / 2) + 1]);
@@ -346,8 +350,11 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
       if ((g & 1) == 0) ldmatrix_x4_trans(vw, cx.kaddr[g / 2] + st_off + Cfg<D>::PK);
       const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
       mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
-      const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
-      mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1 & kMaskHi, y2 & kMaskLo, y2 & kMaskHi, b0, b1);
+      // upper bytes: rows 0-7 take nibble 2 alone, rows 8-15 the whole byte n2 + 16 n3 (still an exact fp16
+      // subnormal); the epilogue takes the difference of the two fp32 accumulators.  One permute and one
+      // mask per register instead of a shift and two masks.
+      const uint32_t y1 = upper_bytes(r1), y2 = upper_bytes(r2);
+      mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1, y2 & kMaskLo, y2, b0, b1);
     }
     return;
   }
@@ -368,8 +375,8 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     if ((g & 1) == 0) ldmatrix_x4_trans(vw, cx.kaddr[g / 2] + st_off + Cfg<D>::PK);
     const uint32_t r1 = vw[2 * (g % 2)], r2 = vw[2 * (g % 2) + 1];
     mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
-    const uint32_t y1 = r1 >> 8, y2 = r2 >> 8;
-    mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1 & kMaskHi, y2 & kMaskLo, y2 & kMaskHi, b0, b1);
+    const uint32_t y1 = upper_bytes(r1), y2 = upper_bytes(r2);  // see the four-group form above
+    mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1, y2 & kMaskLo, y2, b0, b1);
   }
 }
 
@@ -928,8 +935,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     // even channel: codes carried 2^-24; odd channel (high nibble): 2^-20
     *reinterpret_cast<float2*>(mo + ch * kChPitch + 2 * tid4) =
         make_float2((oacc[mt][0] * 16777216.0f - zacc[g][0]) * f0, (oacc[mt][1] * 16777216.0f - zacc[g][1]) * f1);
+    // (odd M tiles: rows 8-15 accumulated the whole upper byte, n2 + 16 n3; rows 0-7 hold the n2 part)
+    const float hi0 = (mt & 1) ? oacc[mt][2] - oacc[mt][0] : oacc[mt][2], hi1 = (mt & 1) ? oacc[mt][3] - oacc[mt][1] : oacc[mt][3];
     *reinterpret_cast<float2*>(mo + (ch + 1) * kChPitch + 2 * tid4) =
-        make_float2((oacc[mt][2] * 1048576.0f - zacc[g][0]) * f0, (oacc[mt][3] * 1048576.0f - zacc[g][1]) * f1);
+        make_float2((hi0 * 1048576.0f - zacc[g][0]) * f0, (hi1 * 1048576.0f - zacc[g][1]) * f1);
   }
   __syncthreads();
   for (int idx = threadIdx.x; idx < 8 * D; idx += kThreads) {
