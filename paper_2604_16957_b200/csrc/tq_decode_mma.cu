@@ -680,6 +680,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     nhead = full_begin > first_blk ? min(nblk, (full_begin - first_blk + NTEAM - 1) / NTEAM) : 0;
   }
   const unsigned nplain = nfull > nhead ? nfull - nhead : 0;  // general form: blocks nhead <= k < nhead + nplain are full
+  const int plain_lo = GEN ? nhead : 0, plain_hi = GEN ? nhead + static_cast<int>(nplain) : nfull;  // (of the first phase)
   // per-lane byte offsets inside a stage: ldmatrix row addresses of the code, scale and zero fragments of
   // this warp's channel groups sub * NGW .. (see block_scores / block_softmax_pv)
   WarpCtx<D> cx;
@@ -753,18 +754,21 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         if (n < nblk) issue(n);
     }
   }
-  if constexpr (DS == 1 && !GEN) {
-   if (phase == 0) {
-    // Full blocks four at a time: ring slot, barrier and stage offsets are constants of each of the four
-    // copies of the block step, so the loop carries no slot arithmetic.
-    constexpr int NST = Cf::NST;
+  fast_blocks:
+  if constexpr (DS == 1) {
+   // Full blocks four at a time: ring slot, barrier and stage offsets are constants of each of the four
+   // copies of the block step, so the loop carries no slot arithmetic.  It starts on a block whose number is
+   // a multiple of four (plain decode: block 0; general form: the first such block behind the masked ones
+   // at the old end of the attended range, reached by the one-block loop below).
+   constexpr int NST = Cf::NST;
+   if (phase == 0 && k % NST == 0 && k >= plain_lo && k + NST <= plain_hi) {
     const RowMask all{kBlk, 0, kBlk, 0, kBlk};
-    uint32_t par = 0;
+    uint32_t par = (k / NST) & 1;
     // The barrier of the next block is probed one block ahead (the probe's latency then hides behind a block
     // of arithmetic); only a probe that came back negative is followed by the blocking wait.  No warp-wide
     // synchronisation is needed before a slot is refilled: its last readers were the warp-collective loads
     // of the previous block, whose results the MMAs issued since then have already consumed.
-    bool ready = k + NST <= nfull ? mbar_test_wait(bars, 0) : false;
+    bool ready = mbar_test_wait(bars, par);
 #ifdef TQ_PROBE_MATH_ONLY
     // Timing probe (results are meaningless): the three copies issued above are awaited here, the fourth
     // slot is cleared, and the unrolled loop then runs its arithmetic on whatever the ring holds without
@@ -775,7 +779,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     __syncwarp();
     ready = true;
 #endif
-    for (; k + NST <= nfull; k += NST) {
+    for (; k + NST <= plain_hi; k += NST) {
 #pragma unroll
       for (int S = 0; S < NST; ++S) {
         if (!ready && !wait_stage(bars + 8 * S, par, wait_limit)) {  // cold: leave the loops, keep the phase order
@@ -800,14 +804,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #endif
    }
   }
-  if constexpr (DS > 1 && !GEN) {
-   if (phase == 0) {
+  if constexpr (DS > 1) {
+   if (phase == 0 && k % Cf::NST == 0 && k >= plain_lo && k + Cf::NST <= plain_hi) {
     // The same four-block step for a team: the scores of each block are exchanged before its softmax.
     static_assert(Cf::NST == 4, "the unrolled loop walks a ring of four slots");
     const RowMask all{kBlk, 0, kBlk, 0, kBlk};
-    uint32_t par = 0;
-    bool ready = k + 4 <= nfull ? mbar_test_wait(bars, 0) : false;
-    for (; k + 4 <= nfull; k += 4) {
+    uint32_t par = (k / Cf::NST) & 1;
+    bool ready = mbar_test_wait(bars, par);
+    for (; k + 4 <= plain_hi; k += 4) {
 #pragma unroll
       for (int S = 0; S < 4; ++S) {
         const bool arrived = ready || wait_stage(bars + 8 * S, par, wait_limit);
@@ -858,6 +862,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
         block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       }
+      if (GEN && phase == 0 && (k + 1) % Cf::NST == 0 && k + 1 >= plain_lo && k + 1 + Cf::NST <= plain_hi) {
+        ++k;  // behind the masked blocks of the old end: the four-block loop takes the full ones
+        goto fast_blocks;
+      }
     } else {
       const RowMask mk = plain ? all : mask_of_block();
       if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
@@ -866,6 +874,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       refill(k + Cf::NST - 1);
       if (plain) block_softmax_pv<D, false>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       else block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
+      if (GEN && phase == 0 && (k + 1) % Cf::NST == 0 && k + 1 >= plain_lo && k + 1 + Cf::NST <= plain_hi) {
+        ++k;
+        goto fast_blocks;
+      }
     }
   }
   phase_done:;
