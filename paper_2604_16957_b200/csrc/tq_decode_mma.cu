@@ -124,9 +124,6 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"(addr));
 }
-__device__ __forceinline__ void ldmatrix_x2(uint32_t (&r)[2], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];\n" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
-}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -356,8 +353,7 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
       const uint32_t y1 = upper_bytes(r1), y2 = upper_bytes(r2);
       mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1, y2 & kMaskLo, y2, b0, b1);
     }
-    return;
-  }
+  } else {
 #pragma unroll
   for (int g = 0; g < NGW; ++g) {
     // Scales / zeros of token pairs (2*tid4, 2*tid4+1) and (2*tid4+8, 2*tid4+9) of group g: an ldmatrix
@@ -377,6 +373,7 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     mma16816(oacc[2 * g], r1 & kMaskLo, r1 & kMaskHi, r2 & kMaskLo, r2 & kMaskHi, b0, b1);
     const uint32_t y1 = upper_bytes(r1), y2 = upper_bytes(r2);  // see the four-group form above
     mma16816(oacc[2 * g + 1], y1 & kMaskLo, y1, y2 & kMaskLo, y2, b0, b1);
+  }
   }
 }
 
