@@ -193,41 +193,71 @@ cudaError_t launch_simple(const Src& src, const tq_kv_cache& c, const __half* q,
   return cudaGetLastError();
 }
 
-// x^ = (q - z) * s for every valid row; one thread per 8 consecutive elements.
+// x^ = (q - z) * s for every valid row, in binary32 (fsub then fmul, each rounded to nearest).  One thread per
+// quantisation group: a 16-byte load of 32 codes, the group's scale and zero, 128 (fp32) or 64 (fp16) bytes
+// stored.  The codes become floats without an integer conversion: (w & 0x000F000F) | 0x64006400 is the half2
+// (1024 + n_0, 1024 + n_4), and 1024 + 16 n for the nibbles one position up; fma(f, 1, -1024) and
+// fma(f, 1/16, -64) are exactly n.  A warp's 32 groups are one contiguous run of the output (4 KB of fp32):
+// the lanes park their pieces in shared memory and the warp stores them as contiguous 512-byte rows.
+// grid = (groups of a head's rows, sequence, 2 * H_kv: K then V per head).
 template <typename T>
 __global__ void __launch_bounds__(256) dequant_kernel(tq_kv_cache c, T* k_mat, T* v_mat) {
   pdl_launch_dependents();
   pdl_wait();
-  const int d = c.d, cpr = d >> 3;
+  const int d = c.d, ng = d >> 5, sh = 31 - __clz(ng);  // groups per row (a power of two)
   const int b = blockIdx.y;
   int len = c.seq_lens[b];
   len = len < 0 ? 0 : (len > c.S_cap ? c.S_cap : len);
-  const bool is_v = blockIdx.z != 0;
-  const long long per_seq = static_cast<long long>(c.H_kv) * len * cpr;
-  const long long local = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (local >= per_seq) return;
-  const long long r = local / cpr;  // h * len + t
-  const int cc = static_cast<int>(local - r * cpr);
-  const long long h = r / len;
-  const int t = static_cast<int>(r - h * len);
-  const long long row = (static_cast<long long>(b) * c.H_kv + h) * c.S_cap + t;
+  const bool is_v = (blockIdx.z & 1) != 0;
+  const int h = blockIdx.z >> 1;
+  const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  constexpr int kPiece = 32 * sizeof(T), kPitch = kPiece + 16;  // a lane's output bytes; its pitch in shared memory
+  __shared__ __align__(16) uint8_t park[8][32 * kPitch];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t = static_cast<int>(idx >> sh), g = static_cast<int>(idx) & (ng - 1);
+  const bool valid = t < len;
+  const int tr = valid ? t : 0;  // (lanes past the end compute row 0 and store nothing)
   bool ok;
-  const uint8_t* blk = cache_block(c, b, static_cast<int>(h), t, nullptr, ok);
-  const uint32_t w = *reinterpret_cast<const uint32_t*>(blk + code_offset(d, is_v, t & 15, cc * 4));
-  const float s = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 0, cc >> 2, t & 15)));
-  const float z = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 1, cc >> 2, t & 15)));
-  float x[8];
+  const uint8_t* blk = cache_block(c, b, h, tr, nullptr, ok);
+  const uint4 w4 = *reinterpret_cast<const uint4*>(blk + code_offset(d, is_v, tr & 15, g * 16));
+  const float s = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 0, g, tr & 15)));
+  const float z = __half2float(*reinterpret_cast<const __half*>(blk + meta_offset(d, is_v, 1, g, tr & 15)));
+  const uint32_t words[4] = {w4.x, w4.y, w4.z, w4.w};
+  uint8_t* const mine = park[warp] + lane * kPitch;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(__fsub_rn(static_cast<float>((w >> (4 * i)) & 0xF), z), s);
-  T* dst = (is_v ? v_mat : k_mat) + row * d + cc * 8;
-  if constexpr (sizeof(T) == 4) {
-    reinterpret_cast<float4*>(dst)[0] = make_float4(x[0], x[1], x[2], x[3]);
-    reinterpret_cast<float4*>(dst)[1] = make_float4(x[4], x[5], x[6], x[7]);
-  } else {
-    __half2 h2[4];
+  for (int j = 0; j < 4; ++j) {  // word j: elements 8j .. 8j+7, nibble i at bits 4i
+    float x[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) h2[i] = __floats2half2_rn(x[2 * i], x[2 * i + 1]);
-    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<uint4*>(h2);
+    for (int half = 0; half < 2; ++half) {  // bytes 0 / 2 of the word, then bytes 1 / 3
+      const uint32_t w = half ? words[j] >> 8 : words[j];
+      const uint32_t lo = (w & 0x000F000Fu) | 0x64006400u, hi = (w & 0x00F000F0u) | 0x64006400u;
+      const float2 fl = __half22float2(*reinterpret_cast<const __half2*>(&lo));  // 1024 + n of nibbles 2*half, 2*half + 4
+      const float2 fh = __half22float2(*reinterpret_cast<const __half2*>(&hi));  // 1024 + 16 n of nibbles 2*half + 1, + 5
+      x[2 * half] = __fmul_rn(__fsub_rn(__fmaf_rn(fl.x, 1.0f, -1024.0f), z), s);
+      x[2 * half + 4] = __fmul_rn(__fsub_rn(__fmaf_rn(fl.y, 1.0f, -1024.0f), z), s);
+      x[2 * half + 1] = __fmul_rn(__fsub_rn(__fmaf_rn(fh.x, 0.0625f, -64.0f), z), s);
+      x[2 * half + 5] = __fmul_rn(__fsub_rn(__fmaf_rn(fh.y, 0.0625f, -64.0f), z), s);
+    }
+    if constexpr (sizeof(T) == 4) {
+      reinterpret_cast<float4*>(mine)[2 * j] = make_float4(x[0], x[1], x[2], x[3]);
+      reinterpret_cast<float4*>(mine)[2 * j + 1] = make_float4(x[4], x[5], x[6], x[7]);
+    } else {
+      __half2 h2[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) h2[i] = __floats2half2_rn(x[2 * i], x[2 * i + 1]);
+      reinterpret_cast<uint4*>(mine)[j] = *reinterpret_cast<uint4*>(h2);
+    }
+  }
+  __syncwarp();
+  // the warp's groups idx0 .. idx0 + 31 are consecutive in the output: element offset (row0 * ng + idx0) * 32
+  const long long idx0 = idx - lane;
+  uint8_t* const out0 = reinterpret_cast<uint8_t*>((is_v ? v_mat : k_mat) +
+                                                   ((static_cast<long long>(b) * c.H_kv + h) * c.S_cap * ng + idx0) * 32);
+#pragma unroll
+  for (int i = 0; i < kPiece / 16; ++i) {
+    const int o = i * 512 + 16 * lane, src = o / kPiece;
+    if (static_cast<int>((idx0 + src) >> sh) < len)
+      *reinterpret_cast<uint4*>(out0 + o) = *reinterpret_cast<const uint4*>(park[warp] + src * kPitch + (o % kPiece));
   }
 }
 
@@ -251,6 +281,9 @@ cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q,
 cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, const void* v_mat, bool fp32,
                                        const __half* q, int H_q, float attn_scale, int C, float* o_part, float* m_part,
                                        float* l_part, int32_t* status, cudaStream_t st) {
+  // the tensor-core kernel where it applies (d = 128, at most 8 query heads per KV head), else the scalar one
+  const cudaError_t fast = launch_attend_mat_mma(c, k_mat, v_mat, fp32, q, H_q, attn_scale, C, o_part, m_part, l_part, status, st);
+  if (fast != cudaErrorNotSupported) return fast;
   auto run = [&](auto dtag, auto ttag) {
     constexpr int D = decltype(dtag)::value;
     using T = decltype(ttag);
@@ -285,8 +318,8 @@ cudaError_t launch_attend_mixed(const tq_kv_cache& c, const __half* k_fp16, cons
 }
 
 cudaError_t launch_dequant(const tq_kv_cache& c, void* k_mat, void* v_mat, bool fp32, cudaStream_t st) {
-  const long long per_seq = static_cast<long long>(c.H_kv) * c.S_cap * (c.d >> 3);
-  dim3 grid(static_cast<unsigned>((per_seq + 255) / 256), c.B, 2);
+  const long long per_head = static_cast<long long>(c.S_cap) * (c.d >> 5);
+  dim3 grid(static_cast<unsigned>((per_head + 255) / 256), c.B, 2 * c.H_kv);
   if (fp32)
     dequant_kernel<float><<<grid, 256, 0, st>>>(c, static_cast<float*>(k_mat), static_cast<float*>(v_mat));
   else

@@ -155,6 +155,9 @@ cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q,
 cudaError_t launch_combine(const float* o_part, const float* m_part, const float* l_part, int B, int H_q, int d, int C,
                            void* out, bool out_fp32, cudaStream_t st);
 cudaError_t launch_dequant(const tq_kv_cache& c, void* k_mat, void* v_mat, bool fp32, cudaStream_t st);
+cudaError_t launch_attend_mat_mma(const tq_kv_cache& c, const void* k_mat, const void* v_mat, bool fp32, const __half* q,
+                                  int H_q, float attn_scale, int C, float* o_part, float* m_part, float* l_part,
+                                  int32_t* status, cudaStream_t st);  // tq_attend_mat.cu; cudaErrorNotSupported: use the scalar kernel
 cudaError_t launch_attend_materialized(const tq_kv_cache& c, const void* k_mat, const void* v_mat, bool fp32,
                                        const __half* q, int H_q, float attn_scale, int C, float* o_part, float* m_part,
                                        float* l_part, int32_t* status, cudaStream_t st);
