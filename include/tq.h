@@ -287,7 +287,10 @@ size_t tq_partials_bytes(int32_t B, int32_t H_q, int32_t d, int32_t num_splits);
  * paragraph, Table 2).  Dequantises all valid rows of K and V into a materialised
  * [B][H_kv][S_cap][d] matrix in `workspace` (fp32 as in the paper when ws_is_fp32 = 1, fp16
  * otherwise), then runs split attention and the Eq. 5 reduction on the materialised matrices.
- * Same result as decode + combine up to rounding.
+ * Same result as decode + combine up to rounding.  Built to be limited by the bytes it moves, like the
+ * fused path (d = 128 with at most 8 query heads per KV head: tensor-core attention over the matrices, an fp32
+ * K^ entering as fp16 hi + lo parts, V^ and the softmax weights as fp16; other shapes: a scalar kernel), so
+ * that the ratio between the two paths is the ratio of their bytes.
  *   workspace_bytes >= tq_dequant_workspace_bytes(...), 16-byte aligned, contents destroyed.
  */
 int tq_sdpa_dequant_then_attend(const tq_kv_cache* cache /* host */, const void* q, int32_t H_q, float attn_scale,
