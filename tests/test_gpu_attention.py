@@ -174,6 +174,36 @@ def test_dequant_then_attend_matches_oracle(gpu, oracle, ws_fp32):
             assert np.abs(kmat[b, :, :lens[b]] - kd[b, :, :lens[b]]).max() <= 2.0 ** -22 * np.abs(kd).max()
 
 
+@pytest.mark.parametrize("H_q,H_kv", [(2, 2), (8, 2), (16, 2), (24, 2)])
+@pytest.mark.parametrize("ws_fp32", [True, False])
+def test_dequant_then_attend_head_groups_and_ragged_ends(gpu, oracle, H_q, H_kv, ws_fp32):
+    """The comparison path at d = 128 with 1, 4, 8 query heads per KV head (tensor-core attention over the
+    materialised matrices) and 12 (the scalar kernel), lengths that end inside a 16-token block, a
+    one-token and an empty sequence."""
+    tq, torch = gpu
+    sh = I.Shape("x", 4, H_q, H_kv, 128, 128 ** -0.5, k_outlier_channels=2)
+    lens = [1000, 1, 0, 4113]
+    host, dev = _both(gpu, oracle, sh, 4113, 16, S_cap=4128, lens=lens)
+    q = I.make_q(sh, 16)
+    ref = oracle.attention(host, q, sh.alpha)
+    nbytes = tq.tq_dequant_workspace_bytes(sh.B, sh.H_kv, sh.H_q, 4128, sh.d, ws_fp32)
+    ws = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda")     # rows nobody wrote are NaN patterns
+    out = torch.full((sh.B, sh.H_q, sh.d), 7.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tq.tq_sdpa_dequant_then_attend(dev, torch.from_numpy(q).cuda(), sh.alpha, ws, ws_fp32, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == tq.TQ_STATUS_EMPTY_SEQ
+    got = out.cpu().numpy()
+    assert not got[2].any()                                                  # the empty sequence: zeros
+    keep = [0, 1, 3]
+    if ws_fp32:
+        assert_attention_close(got[keep], ref[keep], f"dequant-then-attend {H_q}/{H_kv}")
+    else:
+        # an fp16 matrix rounds every v^ to 11 bits: the one-token sequence returns fp16(v^_0), half an fp16 ulp off
+        mx, rel = errors(got[keep], ref[keep])
+        assert mx <= MAX_ABS_TOL + np.abs(ref).max() * 2.0 ** -11 and rel <= 3e-3
+
+
 def test_simple_reference_kernel_matches_oracle(gpu, oracle):
     tq, torch = gpu
     sh = I.Shape("x", 2, 24, 2, 128, 128 ** -0.5)
