@@ -26,6 +26,9 @@
 //   * V: the scale varies along the contraction (token) axis, so it is folded into the other
 //     operand: B_g = fp16(p * s_g) per group, o = sum_tok B_g * n - sum_tok B_g * z_g, the
 //     second sum produced by one extra MMA per group whose A rows all hold z_g.
+//   * Warps that own 128 channels (d >= 128) do both zero-point terms with ONE MMA each, on exact fp16
+//     (hi, lo) pairs of s * z (block_scores, block_softmax_pv); a spare row of the P.V one yields the softmax
+//     denominator; the upper byte of a V code word enters as one operand, n2 + 16 n3, beside n2 alone.
 // Timing probes (evidence for where a launch's time goes; never used by the library itself): compiling this
 // file with -DTQ_PROBE_COPIES_ONLY leaves the copies and their waits but drops the arithmetic of the full
 // blocks; -DTQ_PROBE_MATH_ONLY keeps the arithmetic but stops waiting for and issuing copies after the first
