@@ -395,6 +395,40 @@ def test_multi_query_decode(gpu, oracle, d, H_q, H_kv, S_q, impl):
         tq._test_hook(tq.HOOK_DECODE_IMPL, 0)
 
 
+@pytest.mark.parametrize("d,H_q,H_kv", [(128, 16, 2), (256, 8, 4)])
+@pytest.mark.parametrize("paged", [False, True])
+def test_general_forms_on_long_ranges(gpu, oracle, d, H_q, H_kv, paged):
+    """Sliding windows and several query tokens over ranges long enough that every warp (team) first walks the
+    masked blocks at the old end of its range one by one and then enters the four-block loop, with few splits,
+    window starts inside a block and lengths that end inside one; contiguous and from a page pool."""
+    tq, torch = gpu
+    sh = I.Shape("x", 2, H_q, H_kv, d, d ** -0.5 if d != 256 else 1.0, sigma_qk=1.0 if d != 256 else 0.25)
+    lens = [9000, 5531]
+    k, v = I.make_kv(sh, 9000, 71)
+    if paged:
+        host = oracle.Cache(sh.B, sh.H_kv, 9024, sh.d)
+        dev = _paged(tq, torch, sh, 64, 9024 // 64, 71)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        host.append(k[:, :, :5531], v[:, :, :5531])
+        tq.tq_kv_quantize_append(dev, torch.from_numpy(np.ascontiguousarray(k[:, :, :5531])).cuda(),
+                                 torch.from_numpy(np.ascontiguousarray(v[:, :, :5531])).cuda(), status)
+        assert int(status.item()) == 0          # (both sequences 5531 tokens: the last block holds 11)
+    else:
+        host, dev = _both(gpu, oracle, sh, 9000, 71, S_cap=9008, lens=lens, fill_byte=0xFF)
+    for S_q, window, C in ((1, 5000, 1), (1, 777, 2), (3, 0, 1), (3, 4100, 2), (1, 8999, 3)):
+        q = np.ascontiguousarray(np.stack([I.make_q(sh, 71, stream=s) for s in range(S_q)], axis=1))
+        ref = oracle.attention_multi(host, q, sh.alpha, window)
+        o, m, l = tq.alloc_partials(sh.B, sh.H_q * S_q, sh.d, C)
+        out = torch.empty((sh.B, S_q, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        tq.tq_sdpa_int4_decode_multi(dev, torch.from_numpy(q).cuda(), sh.alpha, window, C, o, m, l, status)
+        tq.tq_sdpa_int4_combine(o, m, l, out.view(sh.B, S_q * sh.H_q, sh.d))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert_attention_close(out.cpu().numpy().reshape(sh.B, -1, sh.d), ref.reshape(sh.B, -1, sh.d),
+                               f"S_q {S_q} window {window} C {C} paged {paged}")
+
+
 @pytest.mark.parametrize("impl", ["mma", "simple"])
 def test_head_dim_512(gpu, oracle, impl):
     """Table 7's Gemma global layers: d = 512, 32 query heads per KV head (four head tiles).  Decode after a
