@@ -250,12 +250,30 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
   }
 }
 
+// A operand of the zero-point MMA of P.V (see block_softmax_pv): does not depend on the scores, so a team
+// computes it while it waits for its partner's partial scores.
+template <int D>
+__device__ __forceinline__ void pv_zero_operands(const WarpCtx<D>& cx, uint32_t st_off, uint32_t (&zop)[4]) {
+  uint32_t r[4];
+  ldmatrix_x4(r, cx.vz_lane + st_off);
+  const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
+  zop[1] = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hneg2(pa)));
+  zop[3] = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hneg2(pb)));
+  // Rows 4-7 repeat the groups of rows 0-3 and are not read back, so row 4 is given ones instead: its
+  // accumulators become sum_tok fp16(P)[tok][head], the softmax denominator (of exactly the weights the
+  // numerator uses), at no instruction beyond the two selects.
+  constexpr uint32_t kOnes = 0x3C003C00u;  // half2 (1, 1)
+  zop[0] = (h2_as_u32(pa) & cx.keep) | (~cx.keep & kOnes);
+  zop[2] = (h2_as_u32(pb) & cx.keep) | (~cx.keep & kOnes);
+}
+
 // Second half: online softmax on the complete scores, then P.V for this warp's DW output channels.
-template <int D, bool TAIL>
+// PRE: the zero-point operands were computed by the caller (pv_zero_operands).
+template <int D, bool TAIL, bool PRE = false>
 __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t st_off, const RowMask& mk,
                                                  const float (&sc)[4], float (&oacc)[Cfg<D>::DW / 16][4],
                                                  float (&zacc)[Cfg<D>::NGW][4], float& m0, float& m1, float& l0,
-                                                 float& l1) {
+                                                 float& l1, const uint32_t* pre = nullptr) {
   constexpr int NGW = Cfg<D>::NGW;
   // ---------------- online softmax in the log2 domain.  d = score - running reference m; the
   // reference is raised only when some d exceeds the threshold, so the common path is 4 FMAs.
@@ -328,17 +346,13 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
     // zero term the unrounded product: the two no longer cancel rounding for rounding, which costs about a
     // factor 1.6 in output error, inside the tolerance; it saves three MMAs and eight shared-memory wavefronts
     // per block, 1.2 us per 128K layer when the kernel runs against the power limit.)
-    uint32_t r[4];
-    ldmatrix_x4(r, cx.vz_lane + st_off);
-    const __half2 pa = __hmul2(u32_as_h2(r[0]), u32_as_h2(r[2])), pb = __hmul2(u32_as_h2(r[1]), u32_as_h2(r[3]));
-    const uint32_t la = h2_as_u32(__hfma2(u32_as_h2(r[0]), u32_as_h2(r[2]), __hneg2(pa)));
-    const uint32_t lb = h2_as_u32(__hfma2(u32_as_h2(r[1]), u32_as_h2(r[3]), __hneg2(pb)));
-    // Rows 4-7 repeat the groups of rows 0-3 and are not read back, so row 4 is given ones instead: its
-    // accumulators become sum_tok fp16(P)[tok][head], the softmax denominator (of exactly the weights the
-    // numerator uses), at no instruction beyond the two selects.
-    constexpr uint32_t kOnes = 0x3C003C00u;  // half2 (1, 1)
-    const uint32_t ha = (h2_as_u32(pa) & cx.keep) | (~cx.keep & kOnes), hb = (h2_as_u32(pb) & cx.keep) | (~cx.keep & kOnes);
-    mma16816(zacc[0], ha, la, hb, lb, pt0, pt1);
+    uint32_t zop[4];
+    if constexpr (PRE) {
+      zop[0] = pre[0]; zop[1] = pre[1]; zop[2] = pre[2]; zop[3] = pre[3];
+    } else {
+      pv_zero_operands<D>(cx, st_off, zop);
+    }
+    mma16816(zacc[0], zop[0], zop[1], zop[2], zop[3], pt0, pt1);
     uint32_t vs[4];
 #pragma unroll
     for (int g = 0; g < NGW; ++g) {
@@ -709,15 +723,24 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // never lowered: nothing runs after a timeout), and the whole team stops together.
   float4* const xch = reinterpret_cast<float4*>(smem + Cf::XCH + team * Cf::XCH_TEAM);
   volatile int* const xflag = reinterpret_cast<volatile int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
-  auto exchange = [&](float (&sc)[4], int par01, bool arrived) -> bool {
+  // Two-warp teams split the barrier in two: a warp announces its partial on its own barrier (bar.arrive, does
+  // not wait) and later waits on its partner's (bar.sync), so whatever does not depend on the scores can be
+  // issued in between.  Barrier 1 + 2 * team + sub belongs to warp `sub` of the team: 32 arrivals from its owner
+  // and 32 from the partner's wait complete a phase.  Four-warp teams keep one barrier per team.
+  auto exchange_post = [&](const float (&sc)[4], int par01, bool arrived) {
     float4* const xb = xch + par01 * (DS * 32);
     xb[sub * 32 + lane] = make_float4(sc[0], sc[1], sc[2], sc[3]);
     if (!arrived && lane == 0) xflag[par01] = 1;
-    asm volatile("bar.sync %0, %1;\n" ::"r"(1 + team), "r"(32 * DS) : "memory");
+    if (DS == 2) asm volatile("bar.arrive %0, 64;\n" ::"r"(1 + 2 * team + sub) : "memory");
+  };
+  auto exchange_wait = [&](float (&sc)[4], int par01) -> bool {
+    float4* const xb = xch + par01 * (DS * 32);
     if (DS == 2) {  // a + b in either order is the same number
+      asm volatile("bar.sync %0, 64;\n" ::"r"(1 + 2 * team + (sub ^ 1)) : "memory");
       const float4 part = xb[(sub ^ 1) * 32 + lane];
       sc[0] += part.x; sc[1] += part.y; sc[2] += part.z; sc[3] += part.w;
     } else {
+      asm volatile("bar.sync %0, %1;\n" ::"r"(1 + team), "r"(32 * DS) : "memory");
       sc[0] = sc[1] = sc[2] = sc[3] = 0.f;
 #pragma unroll
       for (int w = 0; w < DS; ++w) {
@@ -726,6 +749,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       }
     }
     return xflag[par01] == 0;
+  };
+  auto exchange = [&](float (&sc)[4], int par01, bool arrived) -> bool {
+    exchange_post(sc, par01, arrived);
+    return exchange_wait(sc, par01);
   };
 
   bool timed_out = false;
@@ -817,14 +844,19 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         const bool arrived = ready || wait_stage(bars + 8 * S, par, wait_limit);
         float sc[4];
         block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, cz, zero4, sc);
-        if (!exchange(sc, S & 1, arrived)) {
+        exchange_post(sc, S & 1, arrived);
+        // what does not depend on the scores goes between the announcement and the wait (hoisting the first V
+        // scale and code loads as well was measured: it spills and is slower)
+        uint32_t zop[4];
+        pv_zero_operands<D>(cx, S * Cf::STAGE, zop);
+        ready = mbar_test_wait(bars + 8 * ((S + 1) & 3), S == 3 ? par ^ 1 : par);
+        if (!exchange_wait(sc, S & 1)) {
           timed_out = true;
           kf = k + S;
           goto phase_done;
         }
         if (k + S + 3 < nblk) issue_to(k + S + 3, (S + 3) & 3);
-        ready = mbar_test_wait(bars + 8 * ((S + 1) & 3), S == 3 ? par ^ 1 : par);
-        block_softmax_pv<D, false>(cx, S * Cf::STAGE, all, sc, oacc, zacc, m0, m1, l0, l1);
+        block_softmax_pv<D, false, true>(cx, S * Cf::STAGE, all, sc, oacc, zacc, m0, m1, l0, l1, zop);
       }
       par ^= 1;
     }
