@@ -178,7 +178,8 @@ int tq_sdpa_int4_decode(const tq_kv_cache* cache /* host */, const void* q, int3
  * stable_tokens close to the lengths or the last split grows (inside a replayed CUDA graph the value is fixed at
  * capture time: re-capture, or update the node, every few hundred steps).
  * seq_lens[b] < stable_tokens breaks the promise: TQ_STATUS_BAD_LEN is set and that sequence's result is not valid.
- * With a paged cache, or stable_tokens / 16 below the split count, the call is exactly tq_sdpa_int4_decode.
+ * With stable_tokens / 16 below the split count the call is exactly tq_sdpa_int4_decode.  With a paged cache the
+ * promise also covers the page-table entries of the stable tokens' pages (they are read before the wait too).
  * num_splits = 0 picks tq_auto_splits_step(B, H_kv, H_q, d, S_cap).
  * Everything else (arguments, partial layout, errors, status) as tq_sdpa_int4_decode; stable_tokens < 0 or
  * > S_cap is TQ_ERR_SHAPE.  On the 128K Llama-shaped layer the overlap is worth about 3 us per launch.
@@ -212,8 +213,9 @@ void tq_split_range_stable(int32_t len, int32_t stable_tokens, int32_t C, int32_
  *                  overlap on the GPU (other streams) need workspaces of their own.
  *   out          : [B][H_q][d] fp16 or fp32, written by the last thread block of each (sequence, KV head) to finish.
  *   num_splits   : C >= 1, or 0 for tq_auto_splits_step(B, H_kv, H_q, d, S_cap).
- * Restrictions: contiguous cache (page_table == NULL) and H_q / H_kv <= 8; otherwise TQ_ERR_SHAPE -- use the three
- * calls.  Errors: TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_WORKSPACE, TQ_ERR_CUDA.  Status as the three calls.
+ * Contiguous and paged caches alike (paged: the page that the new token falls into must be in the table; an entry
+ * outside the pool sets TQ_STATUS_BAD_PAGE and that row is not written).  Restriction: H_q / H_kv <= 8; otherwise
+ * TQ_ERR_SHAPE -- use the three calls.  Errors: TQ_ERR_NULL, TQ_ERR_SHAPE, TQ_ERR_ALIGN, TQ_ERR_WORKSPACE, TQ_ERR_CUDA.  Status as the three calls.
  */
 int tq_sdpa_int4_step(const tq_kv_cache* cache /* host */, const void* k_new, const void* v_new, const void* q,
                       int32_t H_q, float attn_scale, int32_t num_splits, int32_t stable_tokens, void* workspace,

@@ -174,7 +174,7 @@ int tq_sdpa_int4_decode_overlapped(const tq_kv_cache* cache, const void* q, int3
     return TQ_ERR_ALIGN;
   if (int r = check_decode_grid(cache, H_q, 1)) return r;
   const int C = num_splits ? num_splits : tq_auto_splits_step(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
-  const bool overlapped = cache->page_table == nullptr && stable_tokens / kQuantum >= C &&
+  const bool overlapped = stable_tokens / kQuantum >= C &&
                           test_hooks().decode_impl.load(std::memory_order_relaxed) == 0;
   if (!overlapped)
     return tq_sdpa_int4_decode(cache, q, H_q, attn_scale, C, o_part, m_part, l_part, status, stream);
@@ -198,7 +198,7 @@ int tq_sdpa_int4_step(const tq_kv_cache* cache, const void* k_new, const void* v
   if (int r = check_cache(cache)) return r;
   if (!q || !workspace || !out || ((k_new == nullptr) != (v_new == nullptr))) return TQ_ERR_NULL;
   if (int r = check_heads(cache, H_q)) return r;
-  if (cache->page_table != nullptr || H_q / cache->H_kv > 8) return TQ_ERR_SHAPE;
+  if (H_q / cache->H_kv > 8) return TQ_ERR_SHAPE;
   if (stable_tokens < 0 || stable_tokens > cache->S_cap || num_splits < 0 || num_splits > TQ_MAX_SPLITS) return TQ_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(workspace) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new) ||
       (reinterpret_cast<uintptr_t>(status) & 3u))

@@ -456,7 +456,8 @@ __device__ __noinline__ void quantize_new_row(uint8_t* blk, int row, const __hal
 // G * S_q (query token, head) pairs, v = s * G + g, packed into MMA columns like plain heads; query token s
 // is the (S_q - 1 - s)-th newest cached token and attends causally: tokens [lo_s, hi_s) with
 // hi_s = len - (S_q - 1 - s), lo_s = max(0, hi_s - window).  The plain instantiation carries none of this
-// arithmetic into the block loop.  MODE: 0 plain, 1 general, 2 general over a paged cache (tq.h): the block
+// arithmetic into the block loop.  MODE: 0 plain, 1 general, 2 general over a paged cache (tq.h), 3 overlapped /
+// fused step, 4 the same over a paged cache: the block
 // addresses then come from the page table through a per-thread-block table of page addresses.
 template <int D, int MODE, bool HOOK = false>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
@@ -465,7 +466,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
                       int32_t* status, int stable_blocks, StepArgs sa) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
-  constexpr bool GEN = MODE == 1 || MODE == 2, PAGED = MODE == 2, OVL = MODE == 3;
+  constexpr bool GEN = MODE == 1 || MODE == 2, PAGED = MODE == 2 || MODE == 4, OVL = MODE == 3 || MODE == 4;
   const long long wait_limit = HOOK ? static_cast<long long>(sa.wait_cycles) : kMaxWaitCycles;
   extern __shared__ __align__(1024) uint8_t smem[];
 
@@ -495,7 +496,24 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   const bool ovl = OVL && stable_blocks > 0;
   if (!ovl) pdl_wait();
   const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
-  const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;
+  const uint8_t* const head_blocks = cache.blocks + (row0 >> 4) * Cf::STAGE;  // contiguous cache
+  // Paged cache: the address of this KV head's part of the page that table entry `entry` of the sequence names
+  // (a page outside the pool is flagged and page 0 read instead).
+  const int pshift = PAGED ? 31 - __clz(cache.page_tokens >> 4) : 0;
+  auto page_base = [&](int entry) -> const uint8_t* {
+    int pg = cache.page_table[static_cast<long long>(b) * cache.max_pages + entry];
+    if (static_cast<uint32_t>(pg) >= static_cast<uint32_t>(cache.num_pages)) {
+      if (status) atomicOr(status, TQ_STATUS_BAD_PAGE);
+      pg = 0;
+    }
+    // block index in the pool (fits 32 bits: the pool is checked to hold fewer than 2^31 blocks)
+    const uint32_t idx = (static_cast<uint32_t>(pg) * cache.H_kv + kvh) << pshift;
+    return cache.blocks + static_cast<size_t>(idx) * Cf::STAGE;
+  };
+  auto block_addr = [&](int blk) -> const uint8_t* {  // any block of this (sequence, KV head), by a table lookup if paged
+    if (PAGED) return page_base(blk >> pshift) + static_cast<size_t>(blk & ((1 << pshift) - 1)) * Cf::STAGE;
+    return head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
+  };
   // The length of this sequence; in the fused step also the place where the new token is quantised and
   // written (by the block of the last split of this KV head, which is the only one to read that row: it
   // issues its copies of the newest blocks after this) and where the length is advanced (by whichever block
@@ -508,8 +526,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       if (old < cache.S_cap) n = old + 1;
       else if (c == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status) atomicOr(status, TQ_STATUS_CACHE_FULL);
       if (c == C - 1 && n > old) {  // one head tile per KV head in this form (checked on the host)
-        if (warp == 0)
-          quantize_new_row<D>(const_cast<uint8_t*>(head_blocks) + static_cast<size_t>(old >> 4) * Cf::STAGE, old & 15,
+        bool writable = true;  // paged: a table entry outside the pool is flagged (by block_addr) and nothing is written
+        if (PAGED) {
+          const int pg = cache.page_table[static_cast<long long>(b) * cache.max_pages + ((old >> 4) >> pshift)];
+          writable = static_cast<uint32_t>(pg) < static_cast<uint32_t>(cache.num_pages);
+        }
+        uint8_t* const dst = const_cast<uint8_t*>(block_addr(old >> 4));
+        if (warp == 0 && writable)
+          quantize_new_row<D>(dst, old & 15,
                               sa.k_new + (static_cast<long long>(b) * cache.H_kv + kvh) * D,
                               sa.v_new + (static_cast<long long>(b) * cache.H_kv + kvh) * D);
         __syncthreads();
@@ -565,21 +589,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // the thread block first turns the table entries of its split into addresses of this KV head's part of each
   // page (checked against the pool once), kept in shared memory behind everything else, so that issuing a copy
   // costs a shift, a shared-memory load and a multiply-add.
-  const int pshift = PAGED ? 31 - __clz(cache.page_tokens >> 4) : 0;
+  // (In the overlapped form the table entries of the stable part are read before the wait for the preceding
+  // kernel: they belong to what the caller declared final.  The few blocks the last split attends beyond
+  // the stable part are looked up one by one after the wait.)
   const int page0 = blk0 >> pshift;
   const uint8_t** const page_ptr = reinterpret_cast<const uint8_t**>(smem + Cf::SMEM);
+  const int npages = (PAGED && blk1 > blk0) ? ((blk1 - 1) >> pshift) - page0 + 1 : 0;
   if (PAGED) {
-    const int npages = blk1 > blk0 ? ((blk1 - 1) >> pshift) - page0 + 1 : 0;
-    for (int i = threadIdx.x; i < npages; i += kThreads) {
-      int pg = cache.page_table[static_cast<long long>(b) * cache.max_pages + page0 + i];
-      if (static_cast<uint32_t>(pg) >= static_cast<uint32_t>(cache.num_pages)) {
-        if (status) atomicOr(status, TQ_STATUS_BAD_PAGE);
-        pg = 0;
-      }
-      // block index in the pool (fits 32 bits: the pool is checked to hold fewer than 2^31 blocks)
-      const uint32_t idx = (static_cast<uint32_t>(pg) * cache.H_kv + kvh) << pshift;
-      page_ptr[i] = cache.blocks + static_cast<size_t>(idx) * Cf::STAGE;
-    }
+    for (int i = threadIdx.x; i < npages; i += kThreads) page_ptr[i] = page_base(page0 + i);
   }
   if (DS > 1 || PAGED) __syncthreads();  // a team's warps wait on the same barriers; everybody reads the page addresses
   else __syncwarp();
@@ -587,8 +604,12 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     if (sub == 0 && lane == 0) {
       const int blk = blk0 + team + n * NTEAM;
       const uint8_t* src;
-      if (PAGED) src = page_ptr[(blk >> pshift) - page0] + static_cast<size_t>(blk & ((1 << pshift) - 1)) * Cf::STAGE;
-      else src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
+      if (PAGED) {
+        const int pi = (blk >> pshift) - page0;
+        src = (!OVL || pi < npages) ? page_ptr[pi] + static_cast<size_t>(blk & ((1 << pshift) - 1)) * Cf::STAGE : block_addr(blk);
+      } else {
+        src = head_blocks + static_cast<size_t>(blk) * Cf::STAGE;
+      }
       const uint32_t bar = bars + 8 * slot;
       mbar_expect_tx(bar, Cf::STAGE + ((HOOK && blk == sa.fault_blk) ? 16 : 0));
       bulk_g2s(ring_s + slot * Cf::STAGE, src, Cf::STAGE, bar);
@@ -1092,7 +1113,7 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
                    float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
                    cudaStream_t st) {
   size_t smem = Cfg<D>::SMEM;
-  if (MODE == 2) {
+  if (MODE == 2 || MODE == 4) {
     // room for the page addresses of the longest split: its blocks, rounded out to whole pages
     const long long span = (window > 0 && window < c.S_cap) ? static_cast<long long>(window) + S_q + 15 : c.S_cap;
     const long long blocks = (span + 15) / 16 + 1, per_split = (blocks + C - 1) / C + 1;
@@ -1113,6 +1134,8 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
                    float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
                    bool step, cudaStream_t st) {
   const StepArgs none = {nullptr, nullptr, nullptr, 0, nullptr, 0, -1};
+  if (step && c.page_table != nullptr)
+    return launch<D, 4>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
   if (step) return launch<D, 3>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
   if (c.page_table != nullptr) return launch<D, 2>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, none, st);
   if (window > 0 || S_q > 1) return launch<D, 1>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, 0, none, st);
@@ -1148,7 +1171,7 @@ cudaError_t launch_decode_step(const tq_kv_cache& c, const __half* k_new, const 
                                int32_t* status, cudaStream_t st) {
   const int sb = stable_tokens > 0 ? stable_tokens / kBlk : 0;
   const StepArgs sa = {k_new, v_new, out, out_fp32 ? 1 : 0, counters, 0, -1};
-  const bool step = c.page_table == nullptr && window == 0 && S_q == 1 && (sb > 0 || k_new != nullptr || out != nullptr);
+  const bool step = window == 0 && S_q == 1 && (sb > 0 || k_new != nullptr || out != nullptr);
   switch (c.d) {
     case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);
     case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);

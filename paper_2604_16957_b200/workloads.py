@@ -101,11 +101,11 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
     caches = _fill(B, H_kv, S_cap, d, n, 31, outliers, sigma, lens if lens is not None else [S] * B, page_tokens)
     base_lens = torch.as_tensor(lens if lens is not None else [S] * B, dtype=torch.int32).cuda()
     span = window or S
-    # one launch per step (tq_sdpa_int4_step) wherever it applies: plain decode, contiguous cache, at most 8 query
-    # heads per KV head; the tokens present before the timed steps are its stable part
+    # one launch per step (tq_sdpa_int4_step) wherever it applies: plain decode (contiguous or paged cache), at most 8
+    # query heads per KV head; the tokens present before the timed steps are its stable part
     # (measured: it wins where one wave of thread blocks serves one sequence -- 1K to 128K Llama-shaped contexts,
     # the d = 256 shape -- and loses a few per cent on batches, which keep the calls)
-    fused = (not SEPARATE_CALLS) and S_q == 1 and window == 0 and not page_tokens and H_q // H_kv <= 8 and (
+    fused = (not SEPARATE_CALLS) and S_q == 1 and window == 0 and H_q // H_kv <= 8 and (
         FUSED_EVERYWHERE or (B == 1 and d <= 256))
     C = splits or (tq.tq_auto_splits_step if fused else tq.tq_auto_splits)(B, H_kv, H_q * S_q, d, span)
     o, m, l = tq.alloc_partials(B, H_q * S_q, d, C)

@@ -87,8 +87,9 @@ def test_paged_cache_and_bad_arguments(gpu, oracle):
     paged = tq.PagedKVCache(1, 2, 64, 7, 9, 128)
     paged.page_table.copy_(torch.tensor([[8, 1, 5, 0, 3, 7, 2]], dtype=torch.int32))
     tq.tq_kv_quantize_append(paged, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda())
-    out, _ = _run(tq, torch, paged, q, sh.alpha, 3, 384)          # paged: served by the ordinary decode
-    assert_attention_close(out, oracle.attention(host, q, sh.alpha), "paged")
+    for stable in (384, 128, 0):                                  # paged caches take the overlapped form too
+        out, _ = _run(tq, torch, paged, q, sh.alpha, 3, stable)
+        assert_attention_close(out, oracle.attention(host, q, sh.alpha), f"paged stable={stable}")
     dev = device_cache(tq, torch, sh, k, v, 448)
     o, m, l = tq.alloc_partials(1, 8, 128, 3)
     for bad in (-1, 449):
@@ -237,10 +238,6 @@ def test_fused_step_argument_checks(gpu):
     with pytest.raises(tq.TqError) as e:
         tq.tq_sdpa_int4_step(dev, None, None, q, 1.0, 2, 0, ws[:1024], out)
     assert e.value.code == tq.TQ_ERR_WORKSPACE
-    paged = tq.PagedKVCache(1, 2, 32, 2, 3, 128)
-    with pytest.raises(tq.TqError) as e:
-        tq.tq_sdpa_int4_step(paged, None, None, q, 1.0, 2, 0, ws, out)
-    assert e.value.code == tq.TQ_ERR_SHAPE
 
 
 @pytest.mark.parametrize("use_graph", [False, True])
@@ -320,3 +317,54 @@ def test_config3_long_context_layer_through_the_one_launch_step(gpu, oracle, S):
         else:
             assert np.abs(got - ref).max() <= MAX_ABS_TOL + np.abs(ref).max() * 2.0 ** -11, f"S={S} step {step}"
     assert_cache_bits_equal(dev, host)
+
+
+@pytest.mark.parametrize("d,H_q,H_kv,page_tokens", [(128, 16, 2, 64), (256, 8, 4, 16), (64, 4, 1, 128), (512, 8, 1, 32)])
+def test_fused_step_on_a_paged_cache(gpu, oracle, d, H_q, H_kv, page_tokens):
+    """tq_sdpa_int4_step over a page pool (random page assignment): steps that append into the last page, cross
+    into the next one, and run with stable parts that end inside a page, at a page boundary and at zero; rows bit
+    for bit, lengths, outputs against the oracle; then a table entry outside the pool for the page the new token
+    falls into: flagged, nothing written."""
+    from util import assert_cache_bits_equal
+    tq, torch = gpu
+    sh = I.Shape("x", 2, H_q, H_kv, d, d ** -0.5 if d < 256 else 1.0, sigma_qk=1.0 if d < 256 else 0.25,
+                 k_outlier_channels=4 if d == 128 else 0)
+    S = 2 * page_tokens * 3 - 2                    # two tokens short of a page boundary
+    max_pages = S // page_tokens + 3
+    num_pages = sh.B * max_pages + 2
+    dev = tq.PagedKVCache(sh.B, sh.H_kv, page_tokens, max_pages, num_pages, sh.d)
+    perm = np.random.default_rng(5).permutation(num_pages)[:sh.B * max_pages].astype(np.int32)
+    dev.page_table.copy_(torch.from_numpy(perm.reshape(sh.B, max_pages)))
+    dev.blocks.fill_(0xFF)
+    host = oracle.Cache(sh.B, sh.H_kv, page_tokens * max_pages, sh.d)
+    k, v = I.make_kv(sh, S, 121)
+    host.append(k, v)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tq.tq_kv_quantize_append(dev, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
+    for step, (C, stable) in enumerate(((3, S // 16 * 16), (2, 0), (4, S - page_tokens), (1, 16), (5, S))):
+        ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, C)
+        kn, vn = I.make_kv(sh, 1, 121, stream=1 + step)
+        qn = I.make_q(sh, 121, stream=step)
+        out = torch.full((sh.B, sh.H_q, sh.d), 7.0, dtype=torch.float32, device="cuda")
+        tq.tq_sdpa_int4_step(dev, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(qn).cuda(),
+                             sh.alpha, C, stable, ws, out, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        host.append(kn, vn)
+        assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
+        assert_cache_bits_equal(dev, host)
+        assert_attention_close(out.cpu().numpy(), oracle.attention(host, qn, sh.alpha), f"paged step {step} C={C} stable={stable}")
+    # the next token of sequence 1 falls into a page whose table entry is outside the pool
+    entry = int(host.lens[1]) // page_tokens
+    before = dev.blocks.clone()
+    dev.page_table[1, entry] = num_pages + 7
+    kn, vn = I.make_kv(sh, 1, 121, stream=99)
+    ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, 2)
+    out = torch.zeros((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
+    tq.tq_sdpa_int4_step(dev, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(I.make_q(sh, 121)).cuda(),
+                         sh.alpha, 2, 0, ws, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & tq.TQ_STATUS_BAD_PAGE
+    per_page = dev.blocks.numel() // num_pages
+    changed = (dev.blocks != before).view(num_pages, per_page).any(dim=1).nonzero().flatten().tolist()
+    assert set(changed) <= {int(perm.reshape(sh.B, max_pages)[0, int(host.lens[0]) // page_tokens])}   # only sequence 0's row
