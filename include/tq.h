@@ -220,6 +220,20 @@ void tq_split_range_stable(int32_t len, int32_t stable_tokens, int32_t C, int32_
 int tq_sdpa_int4_step(const tq_kv_cache* cache /* host */, const void* k_new, const void* v_new, const void* q,
                       int32_t H_q, float attn_scale, int32_t num_splits, int32_t stable_tokens, void* workspace,
                       size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream);
+/*
+ * The same step with one stable part PER SEQUENCE, for batches of unequal lengths (the ragged batch of decode
+ * steps): stable_lens is a DEVICE array of B int32, stable_lens[b] = the number of oldest cached tokens of sequence
+ * b that are final before the preceding work in the stream starts; the array itself and q are covered by the same
+ * promise (the kernel reads them before it waits for its predecessor).  Values are clamped to [0, S_cap] and
+ * rounded down to a multiple of 16; a sequence whose stable part holds fewer 16-token blocks than there are splits
+ * starts nothing early.  seq_lens[b] < stable_lens[b] sets TQ_STATUS_BAD_LEN.  Everything else as
+ * tq_sdpa_int4_step; stable_lens == NULL is TQ_ERR_NULL.  The paper has no counterpart (its batches are single
+ * sequences).
+ */
+int tq_sdpa_int4_step_ragged(const tq_kv_cache* cache /* host */, const void* k_new, const void* v_new, const void* q,
+                             int32_t H_q, float attn_scale, int32_t num_splits, const int32_t* stable_lens /* device */,
+                             void* workspace, size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status,
+                             void* stream);
 size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t num_splits);
 /*
  * Split count that tq_sdpa_int4_step and tq_sdpa_int4_decode_overlapped pick for num_splits = 0 (host function).
@@ -229,7 +243,8 @@ size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, 
  * of the next one.  Measured on the 128K Llama-shaped step: 36.5 us per layer with 37 splits, 32.3 us with 36.
  * The spare slots are a share (sequences x KV heads) / slots of the machine: they are left only where that
  * share is at most 1/32 (8 KV heads on 296 slots; with 16 KV heads the d = 256 shape measured 39.0 us with
- * the spare slots and 37.4 us without).
+ * the spare slots and 37.4 us without).  For a batch (more than a quarter of the slots per split) it picks about
+ * three and a half waves of thread blocks instead of tq_auto_splits' four: the overlap fills a launch's tail.
  */
 int32_t tq_auto_splits_step(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len);
 size_t tq_step_counter_bytes(int32_t B, int32_t H_kv);

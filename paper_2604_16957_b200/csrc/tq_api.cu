@@ -100,8 +100,8 @@ int tq_kv_quantize_append(const tq_kv_cache* cache, const void* k_new, const voi
                                        status, static_cast<cudaStream_t>(stream)));
 }
 
-int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len) {
-  (void)d;
+// waves2: thread-block waves of a batch launch, in halves (8 = four waves)
+static int32_t auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t max_seq_len, int waves2) {
   if (B < 1 || H_kv < 1 || H_q < H_kv || max_seq_len < 1) return 1;
   const long long G = H_q / H_kv;
   const long long base = static_cast<long long>(B) * H_kv * ((G + 7) / 8);
@@ -112,10 +112,9 @@ int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t 
     C = slots / base;
     min_tokens = 512;
   } else {
-    // a batch: about four waves of blocks, so that sequences of different lengths even out (measured on
-    // 16 sequences of 4K..64K tokens: 216 us with one wave of 2 splits, 158 us with 10 splits; equal
-    // lengths cost the same either way)
-    C = (4 * slots + base - 1) / base;
+    // a batch: several waves of blocks, so that sequences of different lengths even out (measured on
+    // 16 sequences of 4K..64K tokens: 216 us with one wave of 2 splits, 158 us with 10 splits)
+    C = waves2 == 8 ? (waves2 * slots + 2 * base - 1) / (2 * base) : (waves2 * slots) / (2 * base);  // (four waves: rounded up)
     min_tokens = 2048;
   }
   const long long by_len = max_seq_len / min_tokens;  // keep splits from getting too short
@@ -125,8 +124,17 @@ int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t 
   return static_cast<int32_t>(C);
 }
 
+int32_t tq_auto_splits(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len) {
+  (void)d;
+  return auto_splits(B, H_kv, H_q, max_seq_len, 8);  // separate launches: about four waves for a batch
+}
+
 int32_t tq_auto_splits_step(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len) {
-  const int32_t C = tq_auto_splits(B, H_kv, H_q, d, max_seq_len);
+  (void)d;
+  // Launches of these entry points overlap their predecessor, which fills the tail of a batch launch: fewer, longer
+  // thread blocks do better (16 sequences, 296 slots: ragged 4K..64K 134.0 us with 10 splits, 132.6 with 8; equal
+  // 32K 120.0 and 118.7; 6 splits: 134.9 and 114.5).
+  const int32_t C = auto_splits(B, H_kv, H_q, max_seq_len, 7);
   if (B < 1 || H_kv < 1 || H_q < H_kv) return C;
   const long long base = static_cast<long long>(B) * H_kv * ((H_q / H_kv + 7) / 8);
   const long long slots = 2LL * device_sm_count();
@@ -192,16 +200,18 @@ size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, 
   return tq_step_counter_bytes(B, H_kv) + tq_partials_bytes(B, H_q, d, num_splits);
 }
 
-int tq_sdpa_int4_step(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
-                      float attn_scale, int32_t num_splits, int32_t stable_tokens, void* workspace,
-                      size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
+// Both forms of the fused step: one stable part for the whole batch, or one per sequence (device array).
+static int step_common(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
+                       float attn_scale, int32_t num_splits, int32_t stable_tokens, const int32_t* stable_lens,
+                       void* workspace, size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status,
+                       void* stream) {
   if (int r = check_cache(cache)) return r;
   if (!q || !workspace || !out || ((k_new == nullptr) != (v_new == nullptr))) return TQ_ERR_NULL;
   if (int r = check_heads(cache, H_q)) return r;
   if (H_q / cache->H_kv > 8) return TQ_ERR_SHAPE;
   if (stable_tokens < 0 || stable_tokens > cache->S_cap || num_splits < 0 || num_splits > TQ_MAX_SPLITS) return TQ_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(workspace) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new) ||
-      (reinterpret_cast<uintptr_t>(status) & 3u))
+      (reinterpret_cast<uintptr_t>(status) & 3u) || (reinterpret_cast<uintptr_t>(stable_lens) & 3u))
     return TQ_ERR_ALIGN;
   const int C = num_splits ? num_splits : tq_auto_splits_step(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
   if (workspace_bytes < tq_step_workspace_bytes(cache->B, cache->H_kv, H_q, cache->d, C)) return TQ_ERR_WORKSPACE;
@@ -214,7 +224,22 @@ int tq_sdpa_int4_step(const tq_kv_cache* cache, const void* k_new, const void* v
   const int stable = stable_tokens / kQuantum >= C ? stable_tokens : 0;
   return finish(launch_decode_step(*cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new),
                                    static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, stable, o_part, m_part, l_part,
-                                   counters, out, out_is_fp32 != 0, status, static_cast<cudaStream_t>(stream)));
+                                   counters, out, out_is_fp32 != 0, status, static_cast<cudaStream_t>(stream), stable_lens));
+}
+
+int tq_sdpa_int4_step(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
+                      float attn_scale, int32_t num_splits, int32_t stable_tokens, void* workspace,
+                      size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
+  return step_common(cache, k_new, v_new, q, H_q, attn_scale, num_splits, stable_tokens, nullptr, workspace,
+                     workspace_bytes, out, out_is_fp32, status, stream);
+}
+
+int tq_sdpa_int4_step_ragged(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
+                             float attn_scale, int32_t num_splits, const int32_t* stable_lens, void* workspace,
+                             size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
+  if (!stable_lens) return TQ_ERR_NULL;
+  return step_common(cache, k_new, v_new, q, H_q, attn_scale, num_splits, 0, stable_lens, workspace, workspace_bytes, out,
+                     out_is_fp32, status, stream);
 }
 
 int tq_sdpa_int4_decode_window(const tq_kv_cache* cache, const void* q, int32_t H_q, float attn_scale, int32_t window,

@@ -416,6 +416,7 @@ struct StepArgs {
   void* out;            // [B][H_q][D]: written by the last block to finish of each (sequence, KV head) (null: no reduction)
   int out_fp32;
   int32_t* counters;    // [B * H_kv] arrivals, then [B] length readers; zero between launches
+  const int32_t* stable_lens;  // [B] device: per-sequence stable part in tokens, instead of the launch argument (null: not used)
   // instrumented instantiation only (the library's own tests, see TestHooks): poll limit of the stage waits in
   // SM cycles, and the 16-token block of each (sequence, KV head) whose copy announces 16 bytes too many, so
   // that its barrier never completes although the data lands
@@ -463,7 +464,7 @@ template <int D, int MODE, bool HOOK = false>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, int S_q, float attn_scale, int window,
                       int C, float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
-                      int32_t* status, int stable_blocks, StepArgs sa) {
+                      int32_t* status, int stable_blocks_arg, StepArgs sa) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
   constexpr bool GEN = MODE == 1 || MODE == 2, PAGED = MODE == 2 || MODE == 4, OVL = MODE == 3 || MODE == 4;
@@ -493,6 +494,13 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // computes without waiting for the kernel before it, waits once the stable part is done, reads the length
   // and lets its last split take the tokens beyond the stable part.  Every other form waits here, before its
   // first global access.
+  // the stable part of this sequence in 16-token blocks: the launch argument, or the caller's per-sequence array
+  // (final before the preceding work starts, like what it describes; fewer blocks than splits: no early start)
+  int stable_blocks = stable_blocks_arg;
+  if (OVL && sa.stable_lens != nullptr) {
+    const int st = min(max(sa.stable_lens[blockIdx.z], 0), cache.S_cap) / kBlk;
+    stable_blocks = st >= C ? st : 0;
+  }
   const bool ovl = OVL && stable_blocks > 0;
   if (!ovl) pdl_wait();
   const long long row0 = (static_cast<long long>(b) * cache.H_kv + kvh) * cache.S_cap;
@@ -1133,7 +1141,7 @@ template <int D>
 cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
                    float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
                    bool step, cudaStream_t st) {
-  const StepArgs none = {nullptr, nullptr, nullptr, 0, nullptr, 0, -1};
+  const StepArgs none = {nullptr, nullptr, nullptr, 0, nullptr, nullptr, 0, -1};
   if (step && c.page_table != nullptr)
     return launch<D, 4>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
   if (step) return launch<D, 3>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
@@ -1145,7 +1153,7 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
     const int lim = test_hooks().spin_limit.load(std::memory_order_relaxed);
     const int fb = test_hooks().fault_block.load(std::memory_order_relaxed);
     if (lim > 0 || fb >= 0) {
-      const StepArgs hook = {nullptr, nullptr, nullptr, 0, nullptr, lim > 0 ? lim : static_cast<int>(kMaxWaitCycles), fb};
+      const StepArgs hook = {nullptr, nullptr, nullptr, 0, nullptr, nullptr, lim > 0 ? lim : static_cast<int>(kMaxWaitCycles), fb};
       return launch<D, 0, true>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, 0, hook, st);
     }
   }
@@ -1159,7 +1167,7 @@ cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, in
                               int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st,
                               int stable_tokens) {
   return launch_decode_step(c, nullptr, nullptr, q, H_q, S_q, attn_scale, window, C, stable_tokens, o_part, m_part, l_part,
-                            nullptr, nullptr, false, status, st);
+                            nullptr, nullptr, false, status, st, nullptr);
 }
 
 // The fused step (tq_sdpa_int4_step): k_new / v_new non-null appends one token, out non-null reduces in the
@@ -1168,10 +1176,10 @@ cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, in
 cudaError_t launch_decode_step(const tq_kv_cache& c, const __half* k_new, const __half* v_new, const __half* q, int H_q,
                                int S_q, float attn_scale, int window, int C, int stable_tokens, float* o_part,
                                float* m_part, float* l_part, int32_t* counters, void* out, bool out_fp32,
-                               int32_t* status, cudaStream_t st) {
+                               int32_t* status, cudaStream_t st, const int32_t* stable_lens) {
   const int sb = stable_tokens > 0 ? stable_tokens / kBlk : 0;
-  const StepArgs sa = {k_new, v_new, out, out_fp32 ? 1 : 0, counters, 0, -1};
-  const bool step = window == 0 && S_q == 1 && (sb > 0 || k_new != nullptr || out != nullptr);
+  const StepArgs sa = {k_new, v_new, out, out_fp32 ? 1 : 0, counters, stable_lens, 0, -1};
+  const bool step = window == 0 && S_q == 1 && (sb > 0 || k_new != nullptr || out != nullptr || stable_lens != nullptr);
   switch (c.d) {
     case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);
     case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);

@@ -149,7 +149,7 @@ cudaError_t launch_decode_mma(const tq_kv_cache& c, const __half* q, int H_q, in
 cudaError_t launch_decode_step(const tq_kv_cache& c, const __half* k_new, const __half* v_new, const __half* q, int H_q,
                                int S_q, float attn_scale, int window, int C, int stable_tokens, float* o_part,
                                float* m_part, float* l_part, int32_t* counters, void* out, bool out_fp32,
-                               int32_t* status, cudaStream_t st);
+                               int32_t* status, cudaStream_t st, const int32_t* stable_lens = nullptr);
 cudaError_t launch_decode_simple(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window,
                                  int C, float* o_part, float* m_part, float* l_part, int32_t* status, cudaStream_t st);
 cudaError_t launch_combine(const float* o_part, const float* m_part, const float* l_part, int B, int H_q, int d, int C,

@@ -103,18 +103,16 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
     span = window or S
     # one launch per step (tq_sdpa_int4_step) wherever it applies: plain decode (contiguous or paged cache), at most 8
     # query heads per KV head; the tokens present before the timed steps are its stable part
-    # (measured: it wins wherever the sequences share a stable part -- 1K to 128K Llama-shaped contexts, the d = 256
-    # shape, batches of equal lengths by 2 % -- and loses 2 % on the ragged batch, which has no common stable part
-    # and keeps the calls)
+    # (measured: it wins on 1K to 128K Llama-shaped contexts, the d = 256 shape, and by 2 % on batches, where the
+    # ragged one gives every sequence its own stable part)
     ragged = lens is not None and min(lens) != max(lens)
-    fused = (not SEPARATE_CALLS) and S_q == 1 and window == 0 and H_q // H_kv <= 8 and (
-        FUSED_EVERYWHERE or (not ragged and d <= 256))
+    fused = (not SEPARATE_CALLS) and S_q == 1 and window == 0 and H_q // H_kv <= 8 and (FUSED_EVERYWHERE or d <= 256)
     C = splits or (tq.tq_auto_splits_step if fused else tq.tq_auto_splits)(B, H_kv, H_q * S_q, d, span)
     o, m, l = tq.alloc_partials(B, H_q * S_q, d, C)
     ws = tq.alloc_step_workspace(B, H_kv, H_q, d, C) if fused else None
     # (the stable part is one number for the whole batch: with ragged lengths the last split of the longer
     # sequences would get everything beyond it, so the ragged batch declares none)
-    stable = 0 if ragged else S
+    stable = base_lens.clone() if ragged else S  # ragged: one stable part per sequence (tq_sdpa_int4_step_ragged)
     gen = torch.Generator(device="cuda").manual_seed(5)
     q = (torch.randn((B, S_q, H_q, d), generator=gen, device="cuda") * sigma).half()
     kn = (torch.randn((B, H_kv, S_q, d), generator=gen, device="cuda") * sigma).half()

@@ -368,3 +368,50 @@ def test_fused_step_on_a_paged_cache(gpu, oracle, d, H_q, H_kv, page_tokens):
     per_page = dev.blocks.numel() // num_pages
     changed = (dev.blocks != before).view(num_pages, per_page).any(dim=1).nonzero().flatten().tolist()
     assert set(changed) <= {int(perm.reshape(sh.B, max_pages)[0, int(host.lens[0]) // page_tokens])}   # only sequence 0's row
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_fused_step_with_one_stable_part_per_sequence(gpu, oracle, paged):
+    """tq_sdpa_int4_step_ragged: a batch of unequal lengths, each sequence with its own stable part (its length
+    before the steps; one sequence too short to start early, one with a stable part of zero, one with a value
+    beyond its capacity that is clamped), several steps, against the oracle; then a stable part longer than a
+    sequence: flagged."""
+    from util import assert_cache_bits_equal
+    tq, torch = gpu
+    sh = I.Shape("x", 5, 16, 2, 128, 128 ** -0.5, k_outlier_channels=4)
+    lens = [3000, 517, 40, 2049, 1200]
+    S_cap = 3072
+    k, v = I.make_kv(sh, 3000, 131)
+    if paged:
+        dev = tq.PagedKVCache(sh.B, sh.H_kv, 64, S_cap // 64, sh.B * (S_cap // 64) + 1, sh.d)
+        perm = np.random.default_rng(6).permutation(dev.num_pages)[:sh.B * dev.max_pages].astype(np.int32)
+        dev.page_table.copy_(torch.from_numpy(perm.reshape(sh.B, dev.max_pages)))
+        host = oracle_cache(oracle, sh, k, v, S_cap, lens)
+        flat = device_cache(tq, torch, sh, k, v, S_cap, lens)     # the ragged fill, then moved into the pool page by page
+        pages = flat.blocks.view(sh.B, sh.H_kv, S_cap // 64, 4, -1).permute(0, 2, 1, 3, 4).reshape(sh.B * (S_cap // 64), sh.H_kv, 4, -1)
+        dev.blocks[torch.from_numpy(perm).long()] = pages
+        dev.seq_lens.copy_(flat.seq_lens)
+    else:
+        host = oracle_cache(oracle, sh, k, v, S_cap, lens)
+        dev = device_cache(tq, torch, sh, k, v, S_cap, lens, fill_byte=0xFF)
+    stable = torch.tensor([3000, 517, 40, 0, 99999], dtype=torch.int32, device="cuda")   # 99999 clamps to S_cap > 1200
+    stable[4] = 1200
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for step, C in enumerate((4, 7, 1)):
+        ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, C)
+        kn, vn = I.make_kv(sh, 1, 131, stream=1 + step)
+        qn = I.make_q(sh, 131, stream=step)
+        out = torch.full((sh.B, sh.H_q, sh.d), 7.0, dtype=torch.float32, device="cuda")
+        tq.tq_sdpa_int4_step(dev, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(qn).cuda(),
+                             sh.alpha, C, stable, ws, out, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        host.append(kn, vn)
+        assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
+        assert_cache_bits_equal(dev, host)
+        assert_attention_close(out.cpu().numpy(), oracle.attention(host, qn, sh.alpha), f"ragged step {step} C={C}")
+    stable[1] = 1024                               # longer than sequence 1 (520 tokens now): a broken promise
+    ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, 4)
+    tq.tq_sdpa_int4_step(dev, None, None, torch.from_numpy(I.make_q(sh, 131)).cuda(), sh.alpha, 4, stable, ws, out, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & tq.TQ_STATUS_BAD_LEN
