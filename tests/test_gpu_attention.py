@@ -276,9 +276,11 @@ def test_full_size_128k_llama_layer_in_bench_configuration(gpu, oracle):
     print(f"llama 128K C={C}: max-abs {mx:.2e} rel-L2 {rel:.2e}")
 
 
-def test_config5_ragged_batch_64_decode_steps(gpu, oracle):
+@pytest.mark.parametrize("entry", ["calls", "step"])
+def test_config5_ragged_batch_64_decode_steps(gpu, oracle, entry):
     """Batched ragged decode: B = 16, Llama-70B head shapes, context lengths uniform in [4096, 65536],
-    64 consecutive steps of quantize-append followed by fused attention.  The shortest and the longest
+    64 consecutive steps of quantize-append followed by fused attention, as three calls per step or as one
+    launch per step (tq_sdpa_int4_step_ragged, every sequence's length before the steps as its stable part).  The shortest and the longest
     sequence carry seeded data and are checked against the oracle at the first and the last step (cache
     bit-exact, attention within tolerance); the other sequences hold zeros but have their drawn lengths,
     so the launch has the real ragged work distribution."""
@@ -298,8 +300,10 @@ def test_config5_ragged_batch_64_decode_steps(gpu, oracle):
         view = tq.tq_kv_cache(dev.blocks[b].data_ptr(), dev.seq_lens[b:b + 1].data_ptr(), 1, sh.H_kv, S_cap, sh.d)
         tq.tq_kv_quantize_append(view, torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda(), status)
     dev.seq_lens.copy_(torch.from_numpy(lens))
-    C = tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q, sh.d, S_cap)
+    C = (tq.tq_auto_splits if entry == "calls" else tq.tq_auto_splits_step)(sh.B, sh.H_kv, sh.H_q, sh.d, S_cap)
     o, m, l = tq.alloc_partials(sh.B, sh.H_q, sh.d, C)
+    ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, C)
+    stable = torch.from_numpy(lens.astype(np.int32)).cuda()
     out = torch.empty((sh.B, sh.H_q, sh.d), dtype=torch.float32, device="cuda")
     for step in range(64):
         k_new = np.zeros((sh.B, sh.H_kv, 1, sh.d), np.float16)
@@ -310,9 +314,13 @@ def test_config5_ragged_batch_64_decode_steps(gpu, oracle):
             k_new[b], v_new[b] = kb[0], vb[0]
             q[b] = I.make_q(one, seed=500 + b, stream=step)[0]
             host[b].append(kb, vb)
-        tq.tq_kv_quantize_append(dev, torch.from_numpy(k_new).cuda(), torch.from_numpy(v_new).cuda(), status)
-        tq.tq_sdpa_int4_decode(dev, torch.from_numpy(q).cuda(), sh.alpha, C, o, m, l, status)
-        tq.tq_sdpa_int4_combine(o, m, l, out)
+        if entry == "calls":
+            tq.tq_kv_quantize_append(dev, torch.from_numpy(k_new).cuda(), torch.from_numpy(v_new).cuda(), status)
+            tq.tq_sdpa_int4_decode(dev, torch.from_numpy(q).cuda(), sh.alpha, C, o, m, l, status)
+            tq.tq_sdpa_int4_combine(o, m, l, out)
+        else:
+            tq.tq_sdpa_int4_step(dev, torch.from_numpy(k_new).cuda(), torch.from_numpy(v_new).cuda(),
+                                 torch.from_numpy(q).cuda(), sh.alpha, C, stable, ws, out, status)
         if step in (0, 63):
             torch.cuda.synchronize()
             got = out.cpu().numpy()
