@@ -123,6 +123,17 @@ def test_argument_validation_without_gpu(lib):
     cs = tq.tq_kv_cache(**{**ok_paged, "page_table": fake + 2})
     assert tq._lib.tq_kv_quantize_append(C.byref(cs), fake, fake, 1, None, None) == tq.TQ_ERR_ALIGN
     assert tq._lib.tq_sdpa_int4_attend_static(C.byref(cs), fake, 8, 1.0, fake, 1, None, None) == tq.TQ_ERR_ALIGN
+    # the one-launch step and its per-sequence form: same checks, plus their own arguments
+    cs = tq.tq_kv_cache(fake, fake, 1, 2, 64, 128)
+    wsb = tq._lib.tq_step_workspace_bytes(1, 2, 8, 128, 2)
+    step, ragged = tq._lib.tq_sdpa_int4_step, tq._lib.tq_sdpa_int4_step_ragged
+    assert step(C.byref(cs), fake, None, fake, 8, 1.0, 2, 0, fake, wsb, fake, 1, None, None) == tq.TQ_ERR_NULL
+    assert step(C.byref(cs), None, None, fake, 8, 1.0, 2, 65, fake, wsb, fake, 1, None, None) == tq.TQ_ERR_SHAPE
+    assert step(C.byref(cs), None, None, fake, 24, 1.0, 2, 0, fake, wsb, fake, 1, None, None) == tq.TQ_ERR_SHAPE   # 12 heads per KV head
+    assert step(C.byref(cs), None, None, fake, 8, 1.0, 2, 0, fake, wsb - 1, fake, 1, None, None) == tq.TQ_ERR_WORKSPACE
+    assert ragged(C.byref(cs), None, None, fake, 8, 1.0, 2, None, fake, wsb, fake, 1, None, None) == tq.TQ_ERR_NULL
+    assert ragged(C.byref(cs), None, None, fake, 8, 1.0, 2, fake + 2, fake, wsb, fake, 1, None, None) == tq.TQ_ERR_ALIGN
+    assert ragged(C.byref(cs), None, None, fake, 8, 1.0, 300, fake, fake, wsb, fake, 1, None, None) == tq.TQ_ERR_SHAPE
     # split ranges under a window tile exactly the window
     for length, window, Cn in ((3000, 1024, 5), (1029, 1024, 3), (7, 1024, 2), (100, 1, 4), (0, 5, 2)):
         prev = max(0, length - window)
