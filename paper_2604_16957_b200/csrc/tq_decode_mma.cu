@@ -151,7 +151,7 @@ struct WarpCtx {
   uint32_t vz_lane, vs2_lane;  // row addresses of the V scale / zero load of the zero-point MMA and of the scale loads
   uint32_t kz_lane;            // row address of the scale / zero load that feeds the zero-point MMA of the scores
   uint32_t keep;               // all ones, except 0 in the lanes of row 4 of the P.V zero-point MMA (see block_softmax_pv)
-  float cs;
+  float cs0, cs1;              // score -> log2 units of the softmax for the thread's two columns (heads 2*tid4, 2*tid4+1)
   int gid;
 };
 template <int D> struct KZ { static constexpr bool on = Cfg<D>::NGW == 4; };  // every warp that works on 128 channels
@@ -168,7 +168,7 @@ struct RowMask {
 template <int D, bool TAIL>
 __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t* st, uint32_t st_off, const RowMask& mk,
                                              const uint32_t (&qf)[Cfg<D>::NGW][4], const float (&qs)[Cfg<D>::NGW][2],
-                                             const uint32_t (&qz)[2], const float (&cz)[2],
+                                             const uint32_t (&qz)[2],
                                              const float (&zero4)[4], float (&sc)[4]) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW;
@@ -203,7 +203,8 @@ __device__ __forceinline__ void block_scores(const WarpCtx<D>& cx, const uint8_t
     mma16816_first(accz, h2_as_u32(pa), h2_as_u32(pb), la, lb, qz[0], qz[0], zero4);
     // scales of all four groups for tokens gid, gid + 8: matrices (g0 g1 | tokens 0-7), (g0 g1 | 8-15), (g2 g3 | ..)
     ldmatrix_x4_trans(ksz, cx.ksz_lane + st_off);
-    sc[0] = accz[0] * cz[0]; sc[1] = accz[1] * cz[1]; sc[2] = accz[2] * cz[0]; sc[3] = accz[3] * cz[1];
+    // (q was scaled so that this term and the code terms below carry the same power of two: no multiply here)
+    sc[0] = accz[0]; sc[1] = accz[1]; sc[2] = accz[2]; sc[3] = accz[3];
 #pragma unroll
     for (int g = 0; g < NGW; ++g) {
       const uint32_t w0 = kw[g / 2][2 * (g % 2)];                // token gid
@@ -277,8 +278,8 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
   constexpr int NGW = Cfg<D>::NGW;
   // ---------------- online softmax in the log2 domain.  d = score - running reference m; the
   // reference is raised only when some d exceeds the threshold, so the common path is 4 FMAs.
-  float d0 = fmaf(sc[0], cx.cs, -m0), d1 = fmaf(sc[1], cx.cs, -m1);
-  float d2 = fmaf(sc[2], cx.cs, -m0), d3 = fmaf(sc[3], cx.cs, -m1);
+  float d0 = fmaf(sc[0], cx.cs0, -m0), d1 = fmaf(sc[1], cx.cs1, -m1);
+  float d2 = fmaf(sc[2], cx.cs0, -m0), d3 = fmaf(sc[3], cx.cs1, -m1);
   // rows gid (d0, d1) and gid + 8 (d2, d3); columns 0 (d0, d2) and 1 (d1, d3)
   const bool off0 = TAIL && (cx.gid < mk.lo0 || cx.gid >= mk.hi0), off1 = TAIL && (cx.gid < mk.lo1 || cx.gid >= mk.hi1);
   const bool off2 = TAIL && (cx.gid + 8 < mk.lo0 || cx.gid + 8 >= mk.hi0);
@@ -291,7 +292,7 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
   }
   const bool need = fmaxf(fmaxf(d0, d2), fmaxf(d1, d3)) > kRescaleThreshold;
   if (__any_sync(0xffffffffu, need)) {
-    float a0 = sc[0] * cx.cs, a1 = sc[1] * cx.cs, a2 = sc[2] * cx.cs, a3 = sc[3] * cx.cs;
+    float a0 = sc[0] * cx.cs0, a1 = sc[1] * cx.cs1, a2 = sc[2] * cx.cs0, a3 = sc[3] * cx.cs1;
     if (TAIL) {
       if (off0) a0 = -INFINITY;
       if (off1) a1 = -INFINITY;
@@ -661,12 +662,15 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     qs[g][1] = __shfl_sync(0xffffffffu, sum, (2 * tid4 + 1) * 4);
   }
 
-  // B operand and per-column factor of the zero-point MMA of the scores (see block_scores)
+  // B operand of the zero-point MMA of the scores (see block_scores) and the softmax scale of the thread's columns
   uint32_t qz[2] = {0u, 0u};
-  float cz[2] = {0.f, 0.f};
+  float cs0 = attn_scale * kLog2e * 16777216.0f, cs1 = cs0;  // scores carry 2^-24 from the code operands
   if constexpr (KZ<D>::on) {
-    // head gid's row scaled by a power of two so that its largest magnitude lies in [1, 2): the group sums
-    // then fit fp16 pairs whatever the size of q
+    // Head gid's row is scaled by a power of two, 2^(14 - e) with e = floor(log2(largest magnitude)), so that it
+    // fills the fp16 range whatever the size of q: the code terms then carry 2^(-24 + 14 - e), and the group sums
+    // of q are given the same factor, 2^(-10 - e) (they stay below 2^-3 and are split into an fp16 pair), so
+    // that the zero-point MMA's result adds to the code terms as it stands.  The factor goes into the softmax
+    // scale of the column.  A team agrees on e over the whole row.
     float mx = 0.f, sumg[NGW];
 #pragma unroll
     for (int g = 0; g < NGW; ++g) {
@@ -684,17 +688,43 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     }
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    if constexpr (DS > 1) {  // through the half of the exchange buffer that block 1 is the first to use
+      float* const qmx = reinterpret_cast<float*>(smem + Cf::XCH + team * Cf::XCH_TEAM + DS * 32 * 16);
+      qmx[sub * 32 + lane] = mx;
+      // (named barriers 9 + team: 1 .. 8 belong to the score exchange of the block loop)
+      asm volatile("bar.sync %0, %1;\n" ::"r"(9 + team), "r"(32 * DS) : "memory");
+#pragma unroll
+      for (int w = 0; w < DS; ++w) mx = fmaxf(mx, qmx[w * 32 + lane]);
+      asm volatile("bar.sync %0, %1;\n" ::"r"(9 + team), "r"(32 * DS) : "memory");
+    }
     int e = ((__float_as_int(mx) >> 23) & 0xff) - 127;  // floor(log2(max)); an all-zero row gives -127
     e = max(-24, min(e, 15));
-    const float down = __int_as_float((127 - e) << 23);       // 2^-e
-    const float up24 = __int_as_float((127 + e - 24) << 23);  // 2^(e - 24): the code operands carry 2^-24
-    const float sa = -(tid4 & 1 ? sumg[2] : sumg[0]) * down, sb = -(tid4 & 1 ? sumg[3] : sumg[1]) * down;
+    const float up = __int_as_float((127 + 14 - e) << 23);     // 2^(14 - e)
+    const float dn = __int_as_float((127 - 10 - e) << 23);     // 2^(-10 - e)
+    const float back = __int_as_float((127 + 10 + e) << 23);   // 2^(10 + e): what the scores carry
+#pragma unroll
+    for (int g = 0; g < NGW; ++g) {
+      const __half2* h2 = reinterpret_cast<const __half2*>(&qraw[g]);
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h2[i]);
+        w[i] = h2_as_u32(__floats2half2_rn(f.x * up, f.y * up));  // exact: a power of two, inside the fp16 range
+      }
+      const __half2 sixteenth = __float2half2_rn(0.0625f);
+      qf[g][0] = __byte_perm(w[0], w[2], 0x5410);
+      qf[g][1] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(w[0], w[2], 0x7632)), sixteenth));
+      qf[g][2] = __byte_perm(w[1], w[3], 0x5410);
+      qf[g][3] = h2_as_u32(__hmul2(u32_as_h2(__byte_perm(w[1], w[3], 0x7632)), sixteenth));
+    }
+    const float sa = -(tid4 & 1 ? sumg[2] : sumg[0]) * dn, sb = -(tid4 & 1 ? sumg[3] : sumg[1]) * dn;
     const __half2 hi = __floats2half2_rn(sa, sb);
     const float2 hf = __half22float2(hi);
     const __half2 lo = __floats2half2_rn(sa - hf.x, sb - hf.y);
     qz[0] = qz[1] = tid4 < 2 ? h2_as_u32(hi) : h2_as_u32(lo);
-    cz[0] = __shfl_sync(0xffffffffu, up24, (2 * tid4) * 4);
-    cz[1] = __shfl_sync(0xffffffffu, up24, (2 * tid4 + 1) * 4);
+    const float csh = attn_scale * kLog2e * back;
+    cs0 = __shfl_sync(0xffffffffu, csh, (2 * tid4) * 4);
+    cs1 = __shfl_sync(0xffffffffu, csh, (2 * tid4 + 1) * 4);
   }
 
   float oacc[Cf::DW / 16][4];  // [M tile][c0..c3]: rows = channels, cols = heads 2*tid4, 2*tid4+1
@@ -707,7 +737,6 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #pragma unroll
   for (int g = 0; g < NGW; ++g) zacc[g][0] = zacc[g][1] = zacc[g][2] = zacc[g][3] = 0.f;
   float m0 = kNoMax, m1 = kNoMax, l0 = 0.f, l1 = 0.f;
-  const float cs = attn_scale * kLog2e * 16777216.0f;  // scores carry 2^-24 from the code operands
 
   // Blocks in which every token counts for every column go through the plain step, the others through the
   // masking one.  Plain decode: only the block holding the end of the sequence is partial.  General form:
@@ -727,7 +756,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // per-lane byte offsets inside a stage: ldmatrix row addresses of the code, scale and zero fragments of
   // this warp's channel groups sub * NGW .. (see block_scores / block_softmax_pv)
   WarpCtx<D> cx;
-  cx.cs = cs; cx.gid = gid; cx.keep = gid == 4 ? 0u : 0xFFFFFFFFu;
+  cx.cs0 = cs0; cx.cs1 = cs1; cx.gid = gid; cx.keep = gid == 4 ? 0u : 0xFFFFFFFFu;
   cx.ksz_lane = ring_s + 2 * Cf::PK + (lane >> 4) * Cf::SZ + ((lane >> 3) & 1) * 16 + (lane & 1) * 32 + sub * NGW * 32;
   if constexpr (KZ<D>::on) {
     cx.ksz_lane = ring_s + 2 * Cf::PK + (2 * (lane >> 4) + (lane & 1)) * 32 + ((lane >> 3) & 1) * 16 + sub * NGW * 32;
@@ -849,7 +878,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 #endif
 #ifndef TQ_PROBE_COPIES_ONLY
         float sc[4];
-        block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, cz, zero4, sc);
+        block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, zero4, sc);
         block_softmax_pv<D, false>(cx, S * Cf::STAGE, all, sc, oacc, zacc, m0, m1, l0, l1);
 #endif
       }
@@ -872,7 +901,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       for (int S = 0; S < 4; ++S) {
         const bool arrived = ready || wait_stage(bars + 8 * S, par, wait_limit);
         float sc[4];
-        block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, cz, zero4, sc);
+        block_scores<D, false>(cx, nullptr, S * Cf::STAGE, all, qf, qs, qz, zero4, sc);
         exchange_post(sc, S & 1, arrived);
         // what does not depend on the scores goes between the announcement and the wait (hoisting the first V
         // scale and code loads as well was measured: it spills and is slower)
@@ -916,11 +945,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     float sc[4];
     if (DS == 1) {
       if (plain) {
-        block_scores<D, false>(cx, st, st_s, all, qf, qs, qz, cz, zero4, sc);
+        block_scores<D, false>(cx, st, st_s, all, qf, qs, qz, zero4, sc);
         block_softmax_pv<D, false>(cx, st_s, all, sc, oacc, zacc, m0, m1, l0, l1);
       } else {
         const RowMask mk = mask_of_block();
-        block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
+        block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, zero4, sc);
         block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       }
       if (GEN && phase == 0 && (k + 1) % Cf::NST == 0 && k + 1 >= plain_lo && k + 1 + Cf::NST <= plain_hi) {
@@ -929,8 +958,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       }
     } else {
       const RowMask mk = plain ? all : mask_of_block();
-      if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
-      else block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, cz, zero4, sc);
+      if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, qz, zero4, sc);
+      else block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, zero4, sc);
       if (!exchange(sc, k & 1, arrived)) { timed_out = true; kf = k; break; }
       refill(k + Cf::NST - 1);
       if (plain) block_softmax_pv<D, false>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
