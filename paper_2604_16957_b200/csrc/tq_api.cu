@@ -204,16 +204,20 @@ size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, 
 static int step_common(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
                        float attn_scale, int32_t num_splits, int32_t stable_tokens, const int32_t* stable_lens,
                        void* workspace, size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status,
-                       void* stream) {
+                       void* stream, int32_t window = 0) {
   if (int r = check_cache(cache)) return r;
   if (!q || !workspace || !out || ((k_new == nullptr) != (v_new == nullptr))) return TQ_ERR_NULL;
   if (int r = check_heads(cache, H_q)) return r;
   if (H_q / cache->H_kv > 8) return TQ_ERR_SHAPE;
+  if (window < 0 || (window > 0 && cache->page_table != nullptr)) return TQ_ERR_SHAPE;  // windowed step: contiguous caches
   if (stable_tokens < 0 || stable_tokens > cache->S_cap || num_splits < 0 || num_splits > TQ_MAX_SPLITS) return TQ_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(workspace) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new) ||
       (reinterpret_cast<uintptr_t>(status) & 3u) || (reinterpret_cast<uintptr_t>(stable_lens) & 3u))
     return TQ_ERR_ALIGN;
-  const int C = num_splits ? num_splits : tq_auto_splits_step(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap);
+  const int span = (window > 0 && window < cache->S_cap) ? window : cache->S_cap;
+  const int C = num_splits ? num_splits
+                           : (window > 0 ? tq_auto_splits(cache->B, cache->H_kv, H_q, cache->d, span)
+                                         : tq_auto_splits_step(cache->B, cache->H_kv, H_q, cache->d, cache->S_cap));
   if (workspace_bytes < tq_step_workspace_bytes(cache->B, cache->H_kv, H_q, cache->d, C)) return TQ_ERR_WORKSPACE;
   char* ws = static_cast<char*>(workspace);
   int32_t* counters = reinterpret_cast<int32_t*>(ws);
@@ -223,7 +227,7 @@ static int step_common(const tq_kv_cache* cache, const void* k_new, const void* 
   float* l_part = reinterpret_cast<float*>(reinterpret_cast<char*>(m_part) + align256(n * sizeof(float)));
   const int stable = stable_tokens / kQuantum >= C ? stable_tokens : 0;
   return finish(launch_decode_step(*cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new),
-                                   static_cast<const __half*>(q), H_q, 1, attn_scale, 0, C, stable, o_part, m_part, l_part,
+                                   static_cast<const __half*>(q), H_q, 1, attn_scale, window, C, stable, o_part, m_part, l_part,
                                    counters, out, out_is_fp32 != 0, status, static_cast<cudaStream_t>(stream), stable_lens));
 }
 
@@ -232,6 +236,14 @@ int tq_sdpa_int4_step(const tq_kv_cache* cache, const void* k_new, const void* v
                       size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
   return step_common(cache, k_new, v_new, q, H_q, attn_scale, num_splits, stable_tokens, nullptr, workspace,
                      workspace_bytes, out, out_is_fp32, status, stream);
+}
+
+int tq_sdpa_int4_step_window(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
+                             float attn_scale, int32_t window, int32_t num_splits, void* workspace,
+                             size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
+  if (window < 1) return TQ_ERR_SHAPE;
+  return step_common(cache, k_new, v_new, q, H_q, attn_scale, num_splits, 0, nullptr, workspace, workspace_bytes, out,
+                     out_is_fp32, status, stream, window);
 }
 
 int tq_sdpa_int4_step_ragged(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,

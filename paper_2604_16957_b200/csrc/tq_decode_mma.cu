@@ -400,8 +400,9 @@ __device__ __forceinline__ void block_softmax_pv(const WarpCtx<D>& cx, uint32_t 
 // being kept in registers across the block loop.  `col` = the thread's first score column in the KV head,
 // `first` = the block's first token.
 __device__ __noinline__ RowMask general_row_mask(const int32_t* seq_lens, int b, int S_cap, int S_q, int window, int C,
-                                                 int c, int G, int col, int first) {
-  const int n = checked_len(seq_lens, b, S_cap, nullptr);
+                                                 int c, int G, int col, int first, int len_known) {
+  // (the fused step passes the length it works with: the one in memory is advanced by another thread block meanwhile)
+  const int n = len_known >= 0 ? len_known : checked_len(seq_lens, b, S_cap, nullptr);
   int a, e;  // this split's token range, as at the top of the kernel
   split_range(query_lo(n, S_q, 0, window), n, C, c, a, e);
   const int s0 = min(col / G, S_q - 1), s1 = min((col + 1) / G, S_q - 1);
@@ -459,7 +460,7 @@ __device__ __noinline__ void quantize_new_row(uint8_t* blk, int row, const __hal
 // is the (S_q - 1 - s)-th newest cached token and attends causally: tokens [lo_s, hi_s) with
 // hi_s = len - (S_q - 1 - s), lo_s = max(0, hi_s - window).  The plain instantiation carries none of this
 // arithmetic into the block loop.  MODE: 0 plain, 1 general, 2 general over a paged cache (tq.h), 3 overlapped /
-// fused step, 4 the same over a paged cache: the block
+// fused step, 4 the same over a paged cache, 5 the fused step with a sliding window (general form, contiguous): the block
 // addresses then come from the page table through a per-thread-block table of page addresses.
 template <int D, int MODE, bool HOOK = false>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
@@ -468,7 +469,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
                       int32_t* status, int stable_blocks_arg, StepArgs sa) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
-  constexpr bool GEN = MODE == 1 || MODE == 2, PAGED = MODE == 2 || MODE == 4, OVL = MODE == 3 || MODE == 4;
+  constexpr bool GEN = MODE == 1 || MODE == 2 || MODE == 5, PAGED = MODE == 2 || MODE == 4, OVL = MODE == 3 || MODE == 4;
+  constexpr bool STEP = OVL || MODE == 5;  // the forms that can append the new token and reduce the partials themselves
   const long long wait_limit = HOOK ? static_cast<long long>(sa.wait_cycles) : kMaxWaitCycles;
   extern __shared__ __align__(1024) uint8_t smem[];
 
@@ -530,7 +532,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // wait for the preceding kernel.
   auto read_len = [&]() -> int {
     int n = checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
-    if (OVL && sa.k_new != nullptr) {
+    if (STEP && sa.k_new != nullptr) {
       const int old = n;
       if (old < cache.S_cap) n = old + 1;
       else if (c == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status) atomicOr(status, TQ_STATUS_CACHE_FULL);
@@ -563,7 +565,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     t0 = static_cast<int>((static_cast<long long>(stable_blocks) * c) / C) * kBlk;
     t1 = static_cast<int>((static_cast<long long>(stable_blocks) * (c + 1)) / C) * kBlk;
   } else {
-    len = OVL ? read_len() : checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
+    len = STEP ? read_len() : checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
     split_range(GEN ? query_lo(len, S_q, 0, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
   }
 
@@ -937,7 +939,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
       if (GEN) {
         mk = general_row_mask(cache.seq_lens, blockIdx.z, cache.S_cap, S_q, window, C, blockIdx.x, H_q / cache.H_kv,
-                              (blockIdx.y % tiles) * 8 + 2 * (threadIdx.x & 3), (blk0 + team + k * NTEAM) * kBlk);
+                              (blockIdx.y % tiles) * 8 + 2 * (threadIdx.x & 3), (blk0 + team + k * NTEAM) * kBlk,
+                              STEP ? len : -1);
       }
       return mk;
     };
@@ -1070,7 +1073,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
 
   // ---------------- fused step: Eq. 5 by the last block of this (sequence, KV head) to get here
-  if (OVL && sa.out != nullptr) {
+  if (STEP && sa.out != nullptr) {
     constexpr int kWts = (Cf::MERGE + 15) & ~15;  // behind the merge arrays, inside the ring's memory
     static_assert(kWts + kWarps * TQ_MAX_SPLITS * 4 + 16 + kWarps * 4 <= Cf::PIPE, "the weights fit the ring");
     float* const wts = reinterpret_cast<float*>(smem + kWts) + warp * TQ_MAX_SPLITS;
@@ -1171,6 +1174,8 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
                    float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
                    bool step, cudaStream_t st) {
   const StepArgs none = {nullptr, nullptr, nullptr, 0, nullptr, nullptr, 0, -1};
+  if (step && window > 0)
+    return launch<D, 5>(c, q, H_q, 1, attn_scale, window, C, o_part, m_part, l_part, status, 0, sa, st);
   if (step && c.page_table != nullptr)
     return launch<D, 4>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
   if (step) return launch<D, 3>(c, q, H_q, 1, attn_scale, 0, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
@@ -1208,7 +1213,8 @@ cudaError_t launch_decode_step(const tq_kv_cache& c, const __half* k_new, const 
                                int32_t* status, cudaStream_t st, const int32_t* stable_lens) {
   const int sb = stable_tokens > 0 ? stable_tokens / kBlk : 0;
   const StepArgs sa = {k_new, v_new, out, out_fp32 ? 1 : 0, counters, stable_lens, 0, -1};
-  const bool step = window == 0 && S_q == 1 && (sb > 0 || k_new != nullptr || out != nullptr || stable_lens != nullptr);
+  // (a window with the step's extras selects the windowed step form: contiguous caches, checked by the caller)
+  const bool step = S_q == 1 && (k_new != nullptr || out != nullptr || (window == 0 && (sb > 0 || stable_lens != nullptr)));
   switch (c.d) {
     case 64: return launch<64>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);
     case 128: return launch<128>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status, sb, sa, step, st);

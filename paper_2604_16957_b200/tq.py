@@ -30,7 +30,7 @@ SYMBOLS = ("tq_kv_quantize_append", "tq_auto_splits", "tq_split_range", "tq_sdpa
            "tq_result_string", "tq_last_cuda_error", "tq_version", "tq_sdpa_int4_attend_static",
            "tq_cache_code_offset", "tq_cache_meta_offset", "tq_sdpa_int4_decode_window", "tq_split_range_window",
            "tq_sdpa_int4_decode_multi", "tq_sdpa_mixed_precision_attend", "tq_sdpa_int4_decode_overlapped",
-           "tq_split_range_stable", "tq_sdpa_int4_step", "tq_sdpa_int4_step_ragged", "tq_step_workspace_bytes", "tq_step_counter_bytes", "tq_auto_splits_step")
+           "tq_split_range_stable", "tq_sdpa_int4_step", "tq_sdpa_int4_step_ragged", "tq_sdpa_int4_step_window", "tq_step_workspace_bytes", "tq_step_counter_bytes", "tq_auto_splits_step")
 
 
 class tq_kv_cache(C.Structure):
@@ -63,6 +63,8 @@ _lib.tq_sdpa_int4_step.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _i
 _lib.tq_sdpa_int4_step.restype = C.c_int
 _lib.tq_sdpa_int4_step_ragged.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _vp, _vp, _sz, _vp, _i32, _vp, _vp]
 _lib.tq_sdpa_int4_step_ragged.restype = C.c_int
+_lib.tq_sdpa_int4_step_window.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _i32, _vp, _sz, _vp, _i32, _vp, _vp]
+_lib.tq_sdpa_int4_step_window.restype = C.c_int
 _lib.tq_step_workspace_bytes.argtypes = [_i32] * 5
 _lib.tq_step_workspace_bytes.restype = _sz
 _lib.tq_step_counter_bytes.argtypes = [_i32] * 2
@@ -284,6 +286,20 @@ def tq_sdpa_int4_step(cache, k_new, v_new, q, attn_scale, num_splits, stable_tok
     _check(_lib.tq_sdpa_int4_step(C.byref(cs), _ptr(k_new), _ptr(v_new), _ptr(q), q.shape[1], float(attn_scale),
                                   int(num_splits), int(stable_tokens), _ptr(workspace), workspace.numel(), _ptr(out),
                                   int(out.dtype == torch.float32), _ptr(status), _stream(stream)), "tq_sdpa_int4_step")
+
+
+def tq_sdpa_int4_step_window(cache, k_new, v_new, q, attn_scale, window, num_splits, workspace, out, status=None,
+                             stream=None):
+    """append + attention over the last `window` tokens + split reduction, one launch (contiguous caches)."""
+    assert q.is_contiguous() and q.dtype == torch.float16 and q.dim() == 3
+    assert out.is_contiguous() and out.shape == q.shape and out.dtype in (torch.float16, torch.float32)
+    for t in (k_new, v_new):
+        assert t is None or (t.is_contiguous() and t.dtype == torch.float16 and t.shape == (cache.B, cache.H_kv, 1, cache.d))
+    cs = _cs(cache)
+    _check(_lib.tq_sdpa_int4_step_window(C.byref(cs), _ptr(k_new), _ptr(v_new), _ptr(q), q.shape[1], float(attn_scale),
+                                         int(window), int(num_splits), _ptr(workspace), workspace.numel(), _ptr(out),
+                                         int(out.dtype == torch.float32), _ptr(status), _stream(stream)),
+           "tq_sdpa_int4_step_window")
 
 
 def tq_split_range_stable(length, stable_tokens, C_, c):

@@ -415,3 +415,41 @@ def test_fused_step_with_one_stable_part_per_sequence(gpu, oracle, paged):
     tq.tq_sdpa_int4_step(dev, None, None, torch.from_numpy(I.make_q(sh, 131)).cuda(), sh.alpha, 4, stable, ws, out, status)
     torch.cuda.synchronize()
     assert int(status.item()) & tq.TQ_STATUS_BAD_LEN
+
+
+@pytest.mark.parametrize("d,H_q,H_kv", [(256, 32, 16), (128, 16, 2), (64, 4, 1), (512, 8, 1)])
+def test_fused_step_with_a_sliding_window(gpu, oracle, d, H_q, H_kv):
+    """tq_sdpa_int4_step_window: append + attention over the last `window` tokens + reduction in one launch, over
+    several steps (lengths pass a block boundary, one sequence is shorter than the window, one is full), windows that
+    start inside a block, split counts from 1 up; rows bit for bit, lengths, outputs against the oracle."""
+    from util import assert_cache_bits_equal
+    tq, torch = gpu
+    sh = I.Shape("x", 4, H_q, H_kv, d, d ** -0.5 if d < 256 else 1.0, sigma_qk=1.0 if d < 256 else 0.25,
+                 k_outlier_channels=4 if d == 128 else 0)
+    lens = [3000, 1024, 30, 3055]
+    S_cap = 3056
+    host, dev = _step_setup(tq, torch, oracle, sh, 3055, S_cap, lens, 141)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for step, (window, C) in enumerate(((1024, 0), (1000, 3), (17, 1), (5000, 4), (1, 2), (1024, 7))):
+        Cn = C or tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q, sh.d, window)
+        ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, Cn)
+        kn, vn = I.make_kv(sh, 1, 141, stream=1 + step)
+        qn = I.make_q(sh, 141, stream=step)
+        out = torch.full((sh.B, sh.H_q, sh.d), 7.0, dtype=torch.float32, device="cuda")
+        tq.tq_sdpa_int4_step_window(dev, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(qn).cuda(),
+                                    sh.alpha, window, C, ws, out, status)
+        torch.cuda.synchronize()
+        skipped = host.append(kn, vn)
+        full = int(status.item()) & tq.TQ_STATUS_CACHE_FULL
+        assert bool(full) == (skipped > 0) and int(status.item()) & ~tq.TQ_STATUS_CACHE_FULL == 0
+        status.zero_()
+        assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
+        assert_cache_bits_equal(dev, host)
+        assert_attention_close(out.cpu().numpy(), oracle.attention_window(host, qn, sh.alpha, window),
+                               f"window step {step} w={window} C={C}")
+    paged = tq.PagedKVCache(1, sh.H_kv, 32, 2, 3, sh.d)
+    q1 = torch.zeros((1, sh.H_q, sh.d), dtype=torch.float16, device="cuda")
+    with pytest.raises(tq.TqError) as e:
+        tq.tq_sdpa_int4_step_window(paged, None, None, q1, 1.0, 16, 1, tq.alloc_step_workspace(1, sh.H_kv, sh.H_q, sh.d, 1),
+                                    torch.zeros_like(q1, dtype=torch.float32), status)
+    assert e.value.code == tq.TQ_ERR_SHAPE
