@@ -237,15 +237,24 @@ int tq_sdpa_int4_step_ragged(const tq_kv_cache* cache /* host */, const void* k_
 /*
  * The same step over a sliding window (Appendix A: Gemma's sliding-attention layers, w = 1024): append, attention
  * over the last `window` tokens of every sequence (the new one included) and the reduction in one launch.  A
- * window layer's step is made of launches more than of bytes (5 MB at w = 1024 with 16 KV heads of d = 256), so
- * one launch instead of three is what counts.  Nothing is read before the preceding kernel has finished (the
- * window moves with the length).  window >= 1; num_splits = 0 picks tq_auto_splits(B, H_kv, H_q, d, window);
- * contiguous caches only (a paged cache is TQ_ERR_SHAPE: use the three calls); everything else as
- * tq_sdpa_int4_step.
+ * window layer's step is made of latencies more than of bytes (5 MB at w = 1024 with 16 KV heads of d = 256), so
+ * what counts is one launch instead of three and not waiting for the preceding kernel before streaming:
+ *   stable_tokens : 0, or a promise as in tq_sdpa_int4_decode_overlapped, here with an upper bound too: every
+ *                   sequence's length when the kernel reads it lies in [stable_tokens, stable_tokens +
+ *                   TQ_WINDOW_SLACK], the tokens below stable_tokens and q are final.  The blocks that are inside
+ *                   the window for every such length (from stable_tokens + TQ_WINDOW_SLACK - window up to
+ *                   stable_tokens) are then attended before the wait for the preceding kernel, split evenly; the
+ *                   last split attends the few tokens at the two ends after it.  A length outside the promised
+ *                   range sets TQ_STATUS_BAD_LEN.  0, or fewer such blocks than splits: nothing is read early
+ *                   (the general windowed form).
+ * window >= 1; num_splits = 0 picks tq_auto_splits(B, H_kv, H_q, d, window); contiguous caches only (a paged cache
+ * is TQ_ERR_SHAPE: use the three calls); everything else as tq_sdpa_int4_step.
  */
+#define TQ_WINDOW_SLACK 128
 int tq_sdpa_int4_step_window(const tq_kv_cache* cache /* host */, const void* k_new, const void* v_new, const void* q,
-                             int32_t H_q, float attn_scale, int32_t window, int32_t num_splits, void* workspace,
-                             size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream);
+                             int32_t H_q, float attn_scale, int32_t window, int32_t num_splits, int32_t stable_tokens,
+                             void* workspace, size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status,
+                             void* stream);
 size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t num_splits);
 /*
  * Split count that tq_sdpa_int4_step and tq_sdpa_int4_decode_overlapped pick for num_splits = 0 (host function).

@@ -3,6 +3,8 @@
 #include <cstdlib>
 #include <cstring>
 
+#include <algorithm>
+
 #include "tq_internal.cuh"
 
 namespace tq {
@@ -225,7 +227,13 @@ static int step_common(const tq_kv_cache* cache, const void* k_new, const void* 
   float* o_part = reinterpret_cast<float*>(ws + tq_step_counter_bytes(cache->B, cache->H_kv));
   float* m_part = reinterpret_cast<float*>(reinterpret_cast<char*>(o_part) + align256(n * cache->d * sizeof(float)));
   float* l_part = reinterpret_cast<float*>(reinterpret_cast<char*>(m_part) + align256(n * sizeof(float)));
-  const int stable = stable_tokens / kQuantum >= C ? stable_tokens : 0;
+  int stable = stable_tokens / kQuantum >= C ? stable_tokens : 0;
+  if (window > 0 && stable > 0) {
+    // windowed step: the early region (see the kernel) must hold at least one block per split, else the general form
+    const long long sb = stable / kQuantum, lo = sb * kQuantum + TQ_WINDOW_SLACK - window;
+    const long long early0 = lo > 0 ? std::min((lo + kQuantum - 1) / kQuantum, sb) : 0;
+    if (sb - early0 < C) stable = 0;
+  }
   return finish(launch_decode_step(*cache, static_cast<const __half*>(k_new), static_cast<const __half*>(v_new),
                                    static_cast<const __half*>(q), H_q, 1, attn_scale, window, C, stable, o_part, m_part, l_part,
                                    counters, out, out_is_fp32 != 0, status, static_cast<cudaStream_t>(stream), stable_lens));
@@ -239,11 +247,11 @@ int tq_sdpa_int4_step(const tq_kv_cache* cache, const void* k_new, const void* v
 }
 
 int tq_sdpa_int4_step_window(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,
-                             float attn_scale, int32_t window, int32_t num_splits, void* workspace,
+                             float attn_scale, int32_t window, int32_t num_splits, int32_t stable_tokens, void* workspace,
                              size_t workspace_bytes, void* out, int32_t out_is_fp32, int32_t* status, void* stream) {
   if (window < 1) return TQ_ERR_SHAPE;
-  return step_common(cache, k_new, v_new, q, H_q, attn_scale, num_splits, 0, nullptr, workspace, workspace_bytes, out,
-                     out_is_fp32, status, stream, window);
+  return step_common(cache, k_new, v_new, q, H_q, attn_scale, num_splits, stable_tokens, nullptr, workspace,
+                     workspace_bytes, out, out_is_fp32, status, stream, window);
 }
 
 int tq_sdpa_int4_step_ragged(const tq_kv_cache* cache, const void* k_new, const void* v_new, const void* q, int32_t H_q,

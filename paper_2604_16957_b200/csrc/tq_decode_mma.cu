@@ -63,6 +63,7 @@ constexpr int kBlk = 16;              // tokens per stage = MMA M (scores) = MMA
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 4.0f;  // log2 units
+constexpr int kWinSlack = TQ_WINDOW_SLACK;  // tokens a windowed overlapped step may find beyond its stable part
 constexpr float kNoMax = -1.0e30f;         // running reference before any token was seen
 constexpr uint32_t kMaskLo = 0x000F000Fu;  // nibbles 0 / 4 of a 32-bit word: n * 2^-24 as fp16
 constexpr uint32_t kMaskHi = 0x00F000F0u;  // nibbles 1 / 5: n * 2^-20 as fp16
@@ -460,7 +461,8 @@ __device__ __noinline__ void quantize_new_row(uint8_t* blk, int row, const __hal
 // is the (S_q - 1 - s)-th newest cached token and attends causally: tokens [lo_s, hi_s) with
 // hi_s = len - (S_q - 1 - s), lo_s = max(0, hi_s - window).  The plain instantiation carries none of this
 // arithmetic into the block loop.  MODE: 0 plain, 1 general, 2 general over a paged cache (tq.h), 3 overlapped /
-// fused step, 4 the same over a paged cache, 5 the fused step with a sliding window (general form, contiguous): the block
+// fused step, 4 the same over a paged cache, 5 the fused step with a sliding window (general form, contiguous), 6 the
+// overlapped fused step with a sliding window: the block
 // addresses then come from the page table through a per-thread-block table of page addresses.
 template <int D, int MODE, bool HOOK = false>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
@@ -469,7 +471,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
                       int32_t* status, int stable_blocks_arg, StepArgs sa) {
   using Cf = Cfg<D>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
-  constexpr bool GEN = MODE == 1 || MODE == 2 || MODE == 5, PAGED = MODE == 2 || MODE == 4, OVL = MODE == 3 || MODE == 4;
+  constexpr bool GEN = MODE == 1 || MODE == 2 || MODE == 5, PAGED = MODE == 2 || MODE == 4;
+  constexpr bool OVL = MODE == 3 || MODE == 4 || MODE == 6, WIN = MODE == 6;  // WIN: overlapped step over a sliding window
   constexpr bool STEP = OVL || MODE == 5;  // the forms that can append the new token and reduce the partials themselves
   const long long wait_limit = HOOK ? static_cast<long long>(sa.wait_cycles) : kMaxWaitCycles;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -560,10 +563,21 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     }
     return n;
   };
+  // Windowed overlapped step (WIN): the caller promises stable_tokens <= length <= stable_tokens + kWinSlack, so
+  // the blocks from `early0` up to the end of the stable part lie inside the window whatever the length turns
+  // out to be, and are final: the splits partition those and stream them before the wait.  The few blocks at
+  // the two ends (the window's start, the newest tokens) are attended by the last split after the wait, with
+  // row masks.  (The host sends shapes with fewer early blocks than splits to the general form instead.)
+  int early0 = 0;
+  if (WIN) {
+    const int lo = stable_blocks * kBlk + kWinSlack - window;
+    early0 = lo > 0 ? min((lo + kBlk - 1) / kBlk, stable_blocks) : 0;
+  }
   int len = 0, t0, t1;
   if (ovl) {
-    t0 = static_cast<int>((static_cast<long long>(stable_blocks) * c) / C) * kBlk;
-    t1 = static_cast<int>((static_cast<long long>(stable_blocks) * (c + 1)) / C) * kBlk;
+    const long long ne = stable_blocks - early0;
+    t0 = (early0 + static_cast<int>((ne * c) / C)) * kBlk;
+    t1 = (early0 + static_cast<int>((ne * (c + 1)) / C)) * kBlk;
   } else {
     len = STEP ? read_len() : checked_len(cache.seq_lens, b, cache.S_cap, (c == 0 && blockIdx.y == 0) ? status : nullptr);
     split_range(GEN ? query_lo(len, S_q, 0, window) : 0, len, C, c, t0, t1);  // attended tokens of this split
@@ -580,6 +594,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
   // ---- this team's token blocks: blk0 + team, blk0 + team + NTEAM, ...
   int blk0 = t0 / kBlk;
+  int stride = NTEAM;  // blocks between a team's consecutive blocks (windowed overlapped step: changes for the last phase)
+  (void)stride;
   const int blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
   int nblk = blk1 - blk0 > team ? (blk1 - blk0 - team + NTEAM - 1) / NTEAM : 0;
   uint8_t* const ring = smem + team * (Cf::NST * Cf::STAGE);
@@ -613,7 +629,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   else __syncwarp();
   auto issue_to = [&](int n, int slot) {
     if (sub == 0 && lane == 0) {
-      const int blk = blk0 + team + n * NTEAM;
+      const int blk = blk0 + team + n * (WIN ? stride : NTEAM);
       const uint8_t* src;
       if (PAGED) {
         const int pi = (blk >> pshift) - page0;
@@ -818,14 +834,15 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   bool timed_out = false;
   int k = 0, kf = 0;  // kf: the block whose wait ran out
 #pragma unroll 1
-  for (int phase = 0; phase < (ovl ? 2 : 1); ++phase) {
+  for (int phase = 0; phase < (ovl ? (WIN ? 3 : 2) : 1); ++phase) {
   if (ovl && phase == 1) {
     // the stable part is done: from here on this kernel is ordered after the one before it
     pdl_wait();
     len = read_len();
     const int stable_tokens = stable_blocks * kBlk;
-    if (len < stable_tokens && c == 0 && blockIdx.y == 0 && threadIdx.x == 0 && status)
-      atomicOr(status, TQ_STATUS_BAD_LEN);  // the promise did not hold: tokens beyond the length were attended
+    if ((len < stable_tokens || (WIN && len > stable_tokens + kWinSlack)) && c == 0 && blockIdx.y == 0 && threadIdx.x == 0 &&
+        status)
+      atomicOr(status, TQ_STATUS_BAD_LEN);  // the promise did not hold: tokens outside the attended range were attended
     int next = 0;
     if (c == C - 1 && len > stable_tokens && !timed_out) {
       const int eb1 = (len + kBlk - 1) / kBlk;
@@ -836,6 +853,23 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     nblk += next;
     rem_last = next > 0 ? len - (blk0 + team + (nblk - 1) * NTEAM) * kBlk : kBlk;
     nfull = rem_last < kBlk ? nblk - 1 : nblk;
+    if (WIN) nfull = k;  // every block from here on goes through the masking step (window start, end of the sequence)
+    if (next > 0) {
+      for (int n = k; n < k + Cf::NST - 1; ++n)
+        if (n < nblk) issue(n);
+    }
+  }
+  if (WIN && phase == 2) {
+    // the blocks between the window's start and the early region: dealt out over all the teams of all the splits
+    // of this KV head (nothing still running writes them), so that no thread block has more than one or two
+    int next = 0;
+    const int hb0 = max(0, len - window) / kBlk;
+    stride = C * NTEAM;
+    const int mine = c * NTEAM + team;  // this team's place among them
+    if (early0 - hb0 > mine && !timed_out) next = (early0 - hb0 - mine + stride - 1) / stride;
+    blk0 = hb0 + c * NTEAM - nblk * stride;
+    nblk += next;
+    nfull = k;
     if (next > 0) {
       for (int n = k; n < k + Cf::NST - 1; ++n)
         if (n < nblk) issue(n);
@@ -937,6 +971,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     const bool plain = GEN ? static_cast<unsigned>(k - nhead) < nplain : k < nfull;
     auto mask_of_block = [&]() {
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
+      if (WIN) {  // rows of the block inside [max(0, len - window), len)
+        const int first = (blk0 + team + k * stride) * kBlk, lo = max(0, len - window) - first, hi = len - first;
+        mk = RowMask{hi, lo, hi, lo, hi};
+      }
       if (GEN) {
         mk = general_row_mask(cache.seq_lens, blockIdx.z, cache.S_cap, S_q, window, C, blockIdx.x, H_q / cache.H_kv,
                               (blockIdx.y % tiles) * 8 + 2 * (threadIdx.x & 3), (blk0 + team + k * NTEAM) * kBlk,
@@ -1174,6 +1212,8 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
                    float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
                    bool step, cudaStream_t st) {
   const StepArgs none = {nullptr, nullptr, nullptr, 0, nullptr, nullptr, 0, -1};
+  if (step && window > 0 && stable_blocks > 0)
+    return launch<D, 6>(c, q, H_q, 1, attn_scale, window, C, o_part, m_part, l_part, status, stable_blocks, sa, st);
   if (step && window > 0)
     return launch<D, 5>(c, q, H_q, 1, attn_scale, window, C, o_part, m_part, l_part, status, 0, sa, st);
   if (step && c.page_table != nullptr)

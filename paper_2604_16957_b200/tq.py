@@ -63,7 +63,7 @@ _lib.tq_sdpa_int4_step.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _i
 _lib.tq_sdpa_int4_step.restype = C.c_int
 _lib.tq_sdpa_int4_step_ragged.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _vp, _vp, _sz, _vp, _i32, _vp, _vp]
 _lib.tq_sdpa_int4_step_ragged.restype = C.c_int
-_lib.tq_sdpa_int4_step_window.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _i32, _vp, _sz, _vp, _i32, _vp, _vp]
+_lib.tq_sdpa_int4_step_window.argtypes = [_cache_p, _vp, _vp, _vp, _i32, _f32, _i32, _i32, _i32, _vp, _sz, _vp, _i32, _vp, _vp]
 _lib.tq_sdpa_int4_step_window.restype = C.c_int
 _lib.tq_step_workspace_bytes.argtypes = [_i32] * 5
 _lib.tq_step_workspace_bytes.restype = _sz
@@ -288,8 +288,8 @@ def tq_sdpa_int4_step(cache, k_new, v_new, q, attn_scale, num_splits, stable_tok
                                   int(out.dtype == torch.float32), _ptr(status), _stream(stream)), "tq_sdpa_int4_step")
 
 
-def tq_sdpa_int4_step_window(cache, k_new, v_new, q, attn_scale, window, num_splits, workspace, out, status=None,
-                             stream=None):
+def tq_sdpa_int4_step_window(cache, k_new, v_new, q, attn_scale, window, num_splits, stable_tokens, workspace, out,
+                             status=None, stream=None):
     """append + attention over the last `window` tokens + split reduction, one launch (contiguous caches)."""
     assert q.is_contiguous() and q.dtype == torch.float16 and q.dim() == 3
     assert out.is_contiguous() and out.shape == q.shape and out.dtype in (torch.float16, torch.float32)
@@ -297,7 +297,7 @@ def tq_sdpa_int4_step_window(cache, k_new, v_new, q, attn_scale, window, num_spl
         assert t is None or (t.is_contiguous() and t.dtype == torch.float16 and t.shape == (cache.B, cache.H_kv, 1, cache.d))
     cs = _cs(cache)
     _check(_lib.tq_sdpa_int4_step_window(C.byref(cs), _ptr(k_new), _ptr(v_new), _ptr(q), q.shape[1], float(attn_scale),
-                                         int(window), int(num_splits), _ptr(workspace), workspace.numel(), _ptr(out),
+                                         int(window), int(num_splits), int(stable_tokens), _ptr(workspace), workspace.numel(), _ptr(out),
                                          int(out.dtype == torch.float32), _ptr(status), _stream(stream)),
            "tq_sdpa_int4_step_window")
 

@@ -106,9 +106,7 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
     # (measured: it wins on 1K to 128K Llama-shaped contexts, the d = 256 shape, and by 2 % on batches, where the
     # ragged one gives every sequence its own stable part)
     ragged = lens is not None and min(lens) != max(lens)
-    # tq_sdpa_int4_step_window (contiguous caches) only on request: a window layer's step is a chain of dependent
-    # launches either way (12.8 us as one launch against 12.4 us as decode + combine on the d = 256, w = 1024 shape)
-    windowed = FUSED_EVERYWHERE and window > 0 and window < S_cap and not page_tokens
+    windowed = window > 0 and window < S_cap and not page_tokens and lens is None  # tq_sdpa_int4_step_window
     fused = (not SEPARATE_CALLS) and S_q == 1 and (window == 0 or windowed) and H_q // H_kv <= 8 and (
         FUSED_EVERYWHERE or d <= 256)
     C = splits or (tq.tq_auto_splits_step if fused and not window else tq.tq_auto_splits)(B, H_kv, H_q * S_q, d, span)
@@ -132,7 +130,7 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
         for c in caches:
             if fused and window:
                 tq.tq_sdpa_int4_step_window(c, kn if with_append else None, vn if with_append else None, q[:, 0], alpha,
-                                            window, C, ws, out, status)
+                                            window, C, S, ws, out, status)
                 continue
             if fused:
                 tq.tq_sdpa_int4_step(c, kn if with_append else None, vn if with_append else None, q[:, 0], alpha, C, stable,

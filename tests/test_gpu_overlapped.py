@@ -421,7 +421,9 @@ def test_fused_step_with_one_stable_part_per_sequence(gpu, oracle, paged):
 def test_fused_step_with_a_sliding_window(gpu, oracle, d, H_q, H_kv):
     """tq_sdpa_int4_step_window: append + attention over the last `window` tokens + reduction in one launch, over
     several steps (lengths pass a block boundary, one sequence is shorter than the window, one is full), windows that
-    start inside a block, split counts from 1 up; rows bit for bit, lengths, outputs against the oracle."""
+    start inside a block, split counts from 1 up; rows bit for bit, lengths, outputs against the oracle.  First
+    without a stable part (the general windowed form), then with one (the overlapped form: lengths from the stable
+    part itself up to TQ_WINDOW_SLACK beyond it), then a length beyond the promised range: flagged."""
     from util import assert_cache_bits_equal
     tq, torch = gpu
     sh = I.Shape("x", 4, H_q, H_kv, d, d ** -0.5 if d < 256 else 1.0, sigma_qk=1.0 if d < 256 else 0.25,
@@ -430,26 +432,45 @@ def test_fused_step_with_a_sliding_window(gpu, oracle, d, H_q, H_kv):
     S_cap = 3056
     host, dev = _step_setup(tq, torch, oracle, sh, 3055, S_cap, lens, 141)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    for step, (window, C) in enumerate(((1024, 0), (1000, 3), (17, 1), (5000, 4), (1, 2), (1024, 7))):
+
+    def run(step, window, C, stable, append=True):
         Cn = C or tq.tq_auto_splits(sh.B, sh.H_kv, sh.H_q, sh.d, window)
         ws = tq.alloc_step_workspace(sh.B, sh.H_kv, sh.H_q, sh.d, Cn)
         kn, vn = I.make_kv(sh, 1, 141, stream=1 + step)
         qn = I.make_q(sh, 141, stream=step)
         out = torch.full((sh.B, sh.H_q, sh.d), 7.0, dtype=torch.float32, device="cuda")
-        tq.tq_sdpa_int4_step_window(dev, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(qn).cuda(),
-                                    sh.alpha, window, C, ws, out, status)
+        tq.tq_sdpa_int4_step_window(dev, torch.from_numpy(kn).cuda() if append else None,
+                                    torch.from_numpy(vn).cuda() if append else None, torch.from_numpy(qn).cuda(),
+                                    sh.alpha, window, C, stable, ws, out, status)
         torch.cuda.synchronize()
-        skipped = host.append(kn, vn)
+        skipped = host.append(kn, vn) if append else 0
+        return out.cpu().numpy(), qn, skipped
+
+    for step, (window, C) in enumerate(((1024, 0), (1000, 3), (17, 1), (5000, 4), (1, 2), (1024, 7))):
+        got, qn, skipped = run(step, window, C, 0)
         full = int(status.item()) & tq.TQ_STATUS_CACHE_FULL
         assert bool(full) == (skipped > 0) and int(status.item()) & ~tq.TQ_STATUS_CACHE_FULL == 0
         status.zero_()
         assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
         assert_cache_bits_equal(dev, host)
-        assert_attention_close(out.cpu().numpy(), oracle.attention_window(host, qn, sh.alpha, window),
-                               f"window step {step} w={window} C={C}")
+        assert_attention_close(got, oracle.attention_window(host, qn, sh.alpha, window), f"window step {step} w={window} C={C}")
+
+    # overlapped form: every sequence between `stable` and `stable` + 128 tokens long
+    lens2 = [2000, 2001, 2120, 2064]
+    host, dev = _step_setup(tq, torch, oracle, sh, 2120, S_cap, lens2, 142)
+    for step, (window, C) in enumerate(((1024, 0), (1000, 3), (1024, 7), (400, 2), (2500, 5))):
+        stable = 2000 if step < 4 else 2010          # (2010: not a multiple of 16; rounded down by the library)
+        got, qn, _ = run(10 + step, window, C, stable, append=step != 2)
+        assert int(status.item()) == 0
+        assert dev.seq_lens.cpu().tolist() == host.lens.tolist()
+        assert_cache_bits_equal(dev, host)
+        assert_attention_close(got, oracle.attention_window(host, qn, sh.alpha, window), f"overlapped window step {step} w={window} C={C}")
+    run(20, 1024, 2, 1856, append=False)             # sequence 2 holds 2124 tokens now: more than 1856 + 128
+    assert int(status.item()) & tq.TQ_STATUS_BAD_LEN
+    status.zero_()
     paged = tq.PagedKVCache(1, sh.H_kv, 32, 2, 3, sh.d)
     q1 = torch.zeros((1, sh.H_q, sh.d), dtype=torch.float16, device="cuda")
     with pytest.raises(tq.TqError) as e:
-        tq.tq_sdpa_int4_step_window(paged, None, None, q1, 1.0, 16, 1, tq.alloc_step_workspace(1, sh.H_kv, sh.H_q, sh.d, 1),
+        tq.tq_sdpa_int4_step_window(paged, None, None, q1, 1.0, 16, 1, 0, tq.alloc_step_workspace(1, sh.H_kv, sh.H_q, sh.d, 1),
                                     torch.zeros_like(q1, dtype=torch.float32), status)
     assert e.value.code == tq.TQ_ERR_SHAPE
