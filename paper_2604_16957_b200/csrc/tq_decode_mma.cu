@@ -594,8 +594,9 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
   // ---- this team's token blocks: blk0 + team, blk0 + team + NTEAM, ...
   int blk0 = t0 / kBlk;
-  int stride = NTEAM;  // blocks between a team's consecutive blocks (windowed overlapped step: changes for the last phase)
-  (void)stride;
+  // windowed overlapped step: a second run of blocks behind the first (see the phase after the wait)
+  int seg_n = 0x7fffffff, blk0b = 0, strideb = NTEAM;
+  (void)seg_n; (void)blk0b; (void)strideb;
   const int blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
   int nblk = blk1 - blk0 > team ? (blk1 - blk0 - team + NTEAM - 1) / NTEAM : 0;
   uint8_t* const ring = smem + team * (Cf::NST * Cf::STAGE);
@@ -629,7 +630,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   else __syncwarp();
   auto issue_to = [&](int n, int slot) {
     if (sub == 0 && lane == 0) {
-      const int blk = blk0 + team + n * (WIN ? stride : NTEAM);
+      const int blk = (WIN && n >= seg_n) ? blk0b + team + n * strideb : blk0 + team + n * NTEAM;
       const uint8_t* src;
       if (PAGED) {
         const int pi = (blk >> pshift) - page0;
@@ -834,7 +835,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   bool timed_out = false;
   int k = 0, kf = 0;  // kf: the block whose wait ran out
 #pragma unroll 1
-  for (int phase = 0; phase < (ovl ? (WIN ? 3 : 2) : 1); ++phase) {
+  for (int phase = 0; phase < (ovl ? 2 : 1); ++phase) {
   if (ovl && phase == 1) {
     // the stable part is done: from here on this kernel is ordered after the one before it
     pdl_wait();
@@ -853,23 +854,22 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     nblk += next;
     rem_last = next > 0 ? len - (blk0 + team + (nblk - 1) * NTEAM) * kBlk : kBlk;
     nfull = rem_last < kBlk ? nblk - 1 : nblk;
-    if (WIN) nfull = k;  // every block from here on goes through the masking step (window start, end of the sequence)
-    if (next > 0) {
-      for (int n = k; n < k + Cf::NST - 1; ++n)
-        if (n < nblk) issue(n);
+    if (WIN) {
+      // Windowed step: every block from here on goes through the masking step.  Behind the newest blocks come the
+      // blocks between the window's start and the early region, dealt out over all the teams of all the splits of
+      // this KV head (nothing still running writes them), so that no thread block has more than one or two; they
+      // are issued together with the newest ones: one memory latency, not two.  Blocks n >= seg_n of this team
+      // are blk0b + team + n * strideb.
+      nfull = k;
+      const int hb0 = max(0, len - window) / kBlk, mine = c * NTEAM + team;
+      strideb = C * NTEAM;
+      seg_n = nblk;
+      int more = 0;
+      if (early0 - hb0 > mine && !timed_out) more = (early0 - hb0 - mine + strideb - 1) / strideb;
+      blk0b = hb0 + c * NTEAM - nblk * strideb;
+      nblk += more;
+      next += more;
     }
-  }
-  if (WIN && phase == 2) {
-    // the blocks between the window's start and the early region: dealt out over all the teams of all the splits
-    // of this KV head (nothing still running writes them), so that no thread block has more than one or two
-    int next = 0;
-    const int hb0 = max(0, len - window) / kBlk;
-    stride = C * NTEAM;
-    const int mine = c * NTEAM + team;  // this team's place among them
-    if (early0 - hb0 > mine && !timed_out) next = (early0 - hb0 - mine + stride - 1) / stride;
-    blk0 = hb0 + c * NTEAM - nblk * stride;
-    nblk += next;
-    nfull = k;
     if (next > 0) {
       for (int n = k; n < k + Cf::NST - 1; ++n)
         if (n < nblk) issue(n);
@@ -972,7 +972,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     auto mask_of_block = [&]() {
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
       if (WIN) {  // rows of the block inside [max(0, len - window), len)
-        const int first = (blk0 + team + k * stride) * kBlk, lo = max(0, len - window) - first, hi = len - first;
+        const int first = (k >= seg_n ? blk0b + team + k * strideb : blk0 + team + k * NTEAM) * kBlk;
+        const int lo = max(0, len - window) - first, hi = len - first;
         mk = RowMask{hi, lo, hi, lo, hi};
       }
       if (GEN) {
