@@ -266,6 +266,8 @@ size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, 
  * share is at most 1/32 (8 KV heads on 296 slots; with 16 KV heads the d = 256 shape measured 39.0 us with
  * the spare slots and 37.4 us without).  For a batch (more than a quarter of the slots per split) it picks about
  * three and a half waves of thread blocks instead of tq_auto_splits' four: the overlap fills a launch's tail.
+ * Up to 1024 tokens it picks one split: with num_splits = 1 the step's thread blocks write `out` themselves
+ * (Eq. 5 with a single term), without partials, arrival counter or second pass.
  */
 int32_t tq_auto_splits_step(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t max_seq_len);
 size_t tq_step_counter_bytes(int32_t B, int32_t H_kv);

@@ -138,6 +138,8 @@ int32_t tq_auto_splits_step(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int
   // 32K 120.0 and 118.7; 6 splits: 134.9 and 114.5).
   const int32_t C = auto_splits(B, H_kv, H_q, max_seq_len, 7);
   if (B < 1 || H_kv < 1 || H_q < H_kv) return C;
+  // up to 1K tokens one split does best: its thread block writes the result itself (no partials, no second pass)
+  if (max_seq_len <= 1024) return 1;
   const long long base = static_cast<long long>(B) * H_kv * ((H_q / H_kv + 7) / 8);
   const long long slots = 2LL * device_sm_count();
   // One wave that takes every slot: leave one per (sequence, KV head) to the stragglers of the launch before.

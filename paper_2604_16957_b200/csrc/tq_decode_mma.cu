@@ -1093,6 +1093,18 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     tb[h * kRowPitch + x] = sum;
   }
   __syncthreads();
+  if (STEP && sa.out != nullptr && C == 1) {
+    // One split: its normalised partial is the result (Eq. 5 with a single term).  No partials, no arrival counter,
+    // no second pass: the step of a short context ends here.
+    for (int idx = threadIdx.x; idx < nh * (D / 2); idx += kThreads) {
+      const int h = idx / (D / 2), x = 2 * (idx - h * (D / 2));
+      const float2 v = *reinterpret_cast<const float2*>(tb + h * kRowPitch + x);
+      const long long orow = q_row(v0 + h) * D + x;
+      if (sa.out_fp32) *reinterpret_cast<float2*>(static_cast<float*>(sa.out) + orow) = v;
+      else *reinterpret_cast<__half2*>(static_cast<__half*>(sa.out) + orow) = __floats2half2_rn(v.x, v.y);
+    }
+    return;
+  }
   for (int idx = threadIdx.x; idx < nh * D; idx += kThreads) {  // coalesced: one head row after the other
     const int h = idx / D, x = idx - h * D;
     const long long pidx = q_row(v0 + h) * C + c;

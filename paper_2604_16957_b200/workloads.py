@@ -20,6 +20,7 @@ from . import tq
 L2_BYTES = 126 << 20
 IDENTITY_PAGES = False  # --identity-pages: page i of a paged cache is pool page i (default: a random assignment)
 FUSED_EVERYWHERE = False  # --fused: the one-launch step wherever it applies
+NO_STABLE = False  # --no-stable: the fused step declares no stable part (every step waits for the one before it: latency, not throughput)
 SEPARATE_CALLS = False  # --calls: time append / decode / combine as separate launches even where the fused step applies
 
 
@@ -115,6 +116,8 @@ def decode_workload(name, B, H_q, H_kv, d, S, alpha, steps, warmup, outliers, si
     # (the stable part is one number for the whole batch: with ragged lengths the last split of the longer
     # sequences would get everything beyond it, so the ragged batch declares none)
     stable = base_lens.clone() if ragged else S  # ragged: one stable part per sequence (tq_sdpa_int4_step_ragged)
+    if NO_STABLE:
+        stable = 0
     gen = torch.Generator(device="cuda").manual_seed(5)
     q = (torch.randn((B, S_q, H_q, d), generator=gen, device="cuda") * sigma).half()
     kn = (torch.randn((B, H_kv, S_q, d), generator=gen, device="cuda") * sigma).half()
@@ -191,14 +194,14 @@ def ragged_lengths():
 
 
 WORKLOADS = {
-    "llama_1k": lambda a: decode_workload("llama shape, 1K context", 1, 64, 8, 128, 1024, 128 ** -0.5, a.steps, a.warmup, True),
-    "llama_4k": lambda a: decode_workload("llama shape, 4K context", 1, 64, 8, 128, 4096, 128 ** -0.5, a.steps, a.warmup, True),
-    "llama_8k": lambda a: decode_workload("llama shape, 8K context", 1, 64, 8, 128, 8192, 128 ** -0.5, a.steps, a.warmup, True),
-    "llama_32k": lambda a: decode_workload("llama shape, 32K context", 1, 64, 8, 128, 32768, 128 ** -0.5, a.steps, a.warmup, True),
+    "llama_1k": lambda a: decode_workload("llama shape, 1K context", 1, 64, 8, 128, 1024, 128 ** -0.5, a.steps, a.warmup, True, splits=a.splits),
+    "llama_4k": lambda a: decode_workload("llama shape, 4K context", 1, 64, 8, 128, 4096, 128 ** -0.5, a.steps, a.warmup, True, splits=a.splits),
+    "llama_8k": lambda a: decode_workload("llama shape, 8K context", 1, 64, 8, 128, 8192, 128 ** -0.5, a.steps, a.warmup, True, splits=a.splits),
+    "llama_32k": lambda a: decode_workload("llama shape, 32K context", 1, 64, 8, 128, 32768, 128 ** -0.5, a.steps, a.warmup, True, splits=a.splits),
     "gemma_32k": lambda a: decode_workload("gemma-style d=256, 32K context", 1, 32, 16, 256, 32768, 1.0, a.steps, a.warmup,
                                            False, sigma=0.25, splits=a.splits),
     "gemma_32k_window": lambda a: decode_workload("gemma-style d=256, 32K context, window 1024", 1, 32, 16, 256, 32768, 1.0,
-                                                  a.steps, a.warmup, False, sigma=0.25, window=1024),
+                                                  a.steps, a.warmup, False, sigma=0.25, window=1024, splits=a.splits),
     "gemma_32k_sq4": lambda a: decode_workload("gemma-style d=256, 32K context, 4 query tokens", 1, 32, 16, 256, 32768, 1.0,
                                                a.steps, a.warmup, False, sigma=0.25, S_q=4),
     "llama_32k_sq4": lambda a: decode_workload("llama shape, 32K context, 4 query tokens", 1, 64, 8, 128, 32768,
@@ -224,16 +227,18 @@ WORKLOADS = {
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--only", default=None, choices=sorted(WORKLOADS))
-    ap.add_argument("--splits", type=int, default=0, help="sequence splits for the batch workloads (0 = library default)")
+    ap.add_argument("--splits", type=int, default=0, help="sequence splits (batch, short-context and window workloads (0 = library default)")
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--identity-pages", action="store_true", help="paged workloads: pool page i holds page i")
     ap.add_argument("--calls", action="store_true", help="separate append / decode / combine launches everywhere")
+    ap.add_argument("--no-stable", action="store_true", help="fused steps declare no stable part: each step waits for its predecessor before reading anything")
     ap.add_argument("--fused", action="store_true", help="tq_sdpa_int4_step wherever it applies (default: one sequence, d <= 256)")
     args = ap.parse_args()
-    global IDENTITY_PAGES, SEPARATE_CALLS, FUSED_EVERYWHERE
+    global IDENTITY_PAGES, SEPARATE_CALLS, FUSED_EVERYWHERE, NO_STABLE
     IDENTITY_PAGES = args.identity_pages
     SEPARATE_CALLS = args.calls
+    NO_STABLE = args.no_stable
     FUSED_EVERYWHERE = args.fused
     assert torch.cuda.is_available(), "needs a CUDA device (there is no CPU path)"
     for name, fn in WORKLOADS.items():
