@@ -267,11 +267,11 @@ def main():
     # step / the overlapped decode may attend without waiting for the kernel before it (tq.h).
     ws = tq.alloc_step_workspace(1, H_KV, H_Q, D, C, device=dev)
 
-    def enqueue(append=True, decode=True, combine=True, classic=args.classic):
+    def enqueue(append=True, decode=True, combine=True, classic=args.classic, stable=S):
         fused = append and decode and combine and not classic
         for i in range(L):
             if fused:   # one launch: quantize-append + fused int4 attention + split reduction
-                tq.tq_sdpa_int4_step(caches[i], kn_l[i], vn_l[i], q_l[i], ALPHA, C, S, ws, out_l[i], status)
+                tq.tq_sdpa_int4_step(caches[i], kn_l[i], vn_l[i], q_l[i], ALPHA, C, stable, ws, out_l[i], status)
                 continue
             if append:
                 tq.tq_kv_quantize_append(caches[i], kn_l[i], vn_l[i], status)
@@ -319,6 +319,7 @@ def main():
     g_append = make_graph(decode=False, combine=False)
     g_decode_classic = make_graph(append=False, combine=False, classic=True)
     g_three = make_graph(classic=True)
+    g_step_dependent = make_graph(stable=0)   # the fused step with no stable part: every launch waits for its predecessor
 
     W, K = args.warmup, args.steps
     with ClockSampler(local_rank) as clocks:
@@ -332,6 +333,7 @@ def main():
     decode_us = t_decode / K / L * 1e6
     decode_classic_us = time_graph(g_decode_classic, W, K) / K / L * 1e6
     three_us = time_graph(g_three, W, K) / K / L * 1e6
+    step_dependent_us = time_graph(g_step_dependent, W, K) / K / L * 1e6
 
     # ---- end to end through host buffers: pinned host inputs -> device, the step, outputs -> pinned host
     h_in = torch.empty_like(inp, device="cpu").pin_memory()
@@ -379,6 +381,7 @@ def main():
             "breakdown_us_per_layer": {"append+decode+combine": us_per_layer, "decode+combine": t_attn / K / L * 1e6,
                                        "decode": decode_us, "append": t_append / K / L * 1e6,
                                        "decode_waiting_for_predecessor": decode_classic_us,
+                                       "append+decode+combine waiting for predecessor (stable_tokens=0)": step_dependent_us,
                                        "append+decode+combine as three calls": three_us},
             "step_entry": ("tq_kv_quantize_append + tq_sdpa_int4_decode + tq_sdpa_int4_combine" if args.classic else
                            f"tq_sdpa_int4_step(stable_tokens={S}): one launch per layer"),
