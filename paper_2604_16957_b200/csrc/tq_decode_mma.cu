@@ -89,7 +89,7 @@ struct Cfg {
   static constexpr int NTEAM = kWarps / DS;
   static constexpr int MINB = 2;                    // resident blocks per SM
   static constexpr int PIPE = NTEAM * NST * STAGE;  // 40 KB (D = 64), 80 KB otherwise
-  static constexpr int MERGE = (NTEAM * 16 + NTEAM * D * 10 + 8 * (D + 4)) * 4;
+  static constexpr int MERGE = (NTEAM * 16 + NTEAM * 8 * D) * 4;  // merge arrays of the epilogue (inside the ring's memory)
   static constexpr int BARS = PIPE > MERGE ? PIPE : MERGE;  // offset of the mbarriers: [NTEAM][NST] x 8 bytes
   static constexpr int XCH = BARS + NTEAM * NST * 8;        // score exchange of the teams: [NTEAM][2][DS][32] float4 + flags
   static constexpr int XCH_TEAM = DS > 1 ? 2 * DS * 32 * 16 + 2 * DS * 4 : 0;
@@ -1035,34 +1035,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     }
   }
   __syncthreads();  // every warp is done with its ring; the memory is reused below
-  // layout (floats): wml[NTEAM][16] = each team's m[8], l[8] | slab[NTEAM][D][kChPitch] | tb[8][kRowPitch]
-  constexpr int kChPitch = 10;       // 8 heads per channel row, padded: the float2 fragment stores are conflict free
-  constexpr int kRowPitch = D + 4;   // transposed [head][channel] tile, conflict free for the writes below
+  // layout (floats): wml[NTEAM][16] = each team's m[8], l[8] | slab[NTEAM][8 heads][D] = each team's unnormalised
+  // output rows.  The 16-byte chunks of a row are XOR-swizzled inside every run of 8 chunks by the head's pair
+  // index, which makes both the fragment stores below and the row reads after them conflict free.
   float* const wml = reinterpret_cast<float*>(smem);
   float* const slab = wml + NTEAM * 16;
-  float* const tb = slab + NTEAM * D * kChPitch;
   if (gid == 0 && sub == 0) {  // the warps of a team hold identical m and l
     wml[team * 16 + 2 * tid4] = m0;
     wml[team * 16 + 2 * tid4 + 1] = m1;
     wml[team * 16 + 8 + 2 * tid4] = l0;
     wml[team * 16 + 8 + 2 * tid4 + 1] = l1;
   }
-  __syncthreads();
-  // every thread: unit-wide reference M, denominator and this team's weight for its two heads
-  float M0 = kNoMax, M1 = kNoMax;
-#pragma unroll
-  for (int w = 0; w < NTEAM; ++w) {
-    M0 = fmaxf(M0, wml[w * 16 + 2 * tid4]);
-    M1 = fmaxf(M1, wml[w * 16 + 2 * tid4 + 1]);
-  }
-  float den0 = 0.f, den1 = 0.f;
-#pragma unroll
-  for (int w = 0; w < NTEAM; ++w) {  // a team that saw no token has m = -1e30 and l = 0
-    den0 = fmaf(ex2(wml[w * 16 + 2 * tid4] - M0), wml[w * 16 + 8 + 2 * tid4], den0);
-    den1 = fmaf(ex2(wml[w * 16 + 2 * tid4 + 1] - M1), wml[w * 16 + 8 + 2 * tid4 + 1], den1);
-  }
-  const float f0 = den0 > 0.f ? ex2(m0 - M0) / den0 : 0.f;
-  const float f1 = den1 > 0.f ? ex2(m1 - M1) / den1 : 0.f;
   if constexpr (KZ<D>::on) {  // the single zero-point accumulator: hi + lo sums of group r & 3 in the lanes of row r
     const float z0 = zacc[0][0] + zacc[0][2], z1 = zacc[0][1] + zacc[0][3];
 #pragma unroll
@@ -1071,57 +1054,65 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       zacc[g][1] = __shfl_sync(0xffffffffu, z1, g * 4 + tid4);
     }
   }
-  float* const mo = slab + team * D * kChPitch;
 #pragma unroll
-  for (int mt = 0; mt < Cf::DW / 16; ++mt) {
-    const int g = mt >> 1;
-    const int ch = sub * Cf::DW + 32 * g + 4 * gid + 2 * (mt & 1);
-    // even channel: codes carried 2^-24; odd channel (high nibble): 2^-20
-    *reinterpret_cast<float2*>(mo + ch * kChPitch + 2 * tid4) =
-        make_float2((oacc[mt][0] * 16777216.0f - zacc[g][0]) * f0, (oacc[mt][1] * 16777216.0f - zacc[g][1]) * f1);
-    // (odd M tiles: rows 8-15 accumulated the whole upper byte, n2 + 16 n3; rows 0-7 hold the n2 part)
-    const float hi0 = (mt & 1) ? oacc[mt][2] - oacc[mt][0] : oacc[mt][2], hi1 = (mt & 1) ? oacc[mt][3] - oacc[mt][1] : oacc[mt][3];
-    *reinterpret_cast<float2*>(mo + (ch + 1) * kChPitch + 2 * tid4) =
-        make_float2((hi0 * 1048576.0f - zacc[g][0]) * f0, (hi1 * 1048576.0f - zacc[g][1]) * f1);
-  }
-  __syncthreads();
-  for (int idx = threadIdx.x; idx < 8 * D; idx += kThreads) {
-    const int x = idx >> 3, h = idx & 7;  // consecutive threads take consecutive heads of one channel
-    float sum = 0.f;
-#pragma unroll
-    for (int w = 0; w < NTEAM; ++w) sum += slab[(w * D + x) * kChPitch + h];
-    tb[h * kRowPitch + x] = sum;
-  }
-  __syncthreads();
-  if (STEP && sa.out != nullptr && C == 1) {
-    // One split: its normalised partial is the result (Eq. 5 with a single term).  No partials, no arrival counter,
-    // no second pass: the step of a short context ends here.
-    for (int idx = threadIdx.x; idx < nh * (D / 2); idx += kThreads) {
-      const int h = idx / (D / 2), x = 2 * (idx - h * (D / 2));
-      const float2 v = *reinterpret_cast<const float2*>(tb + h * kRowPitch + x);
-      const long long orow = q_row(v0 + h) * D + x;
-      if (sa.out_fp32) *reinterpret_cast<float2*>(static_cast<float*>(sa.out) + orow) = v;
-      else *reinterpret_cast<__half2*>(static_cast<__half*>(sa.out) + orow) = __floats2half2_rn(v.x, v.y);
-    }
-    return;
-  }
-  for (int idx = threadIdx.x; idx < nh * D; idx += kThreads) {  // coalesced: one head row after the other
-    const int h = idx / D, x = idx - h * D;
-    const long long pidx = q_row(v0 + h) * C + c;
-    o_part[pidx * D + x] = tb[h * kRowPitch + x];
-  }
-  if (warp == 0 && gid == 0) {  // lanes 0..3 hold heads 2*tid4, 2*tid4+1
+  for (int g = 0; g < NGW; ++g) {
+    // channels sub * DW + 32 g + 4 gid + {0, 1, 2, 3} of heads 2*tid4 + j: M tile 2g holds channels +0 (rows 0-7:
+    // codes carried 2^-24) and +1 (rows 8-15, high nibble: 2^-20), M tile 2g + 1 channels +2 and +3, where
+    // rows 8-15 accumulated the whole upper byte n2 + 16 n3 and rows 0-7 hold the n2 part
+    const int chunk = sub * (Cf::DW / 4) + 8 * g + (gid ^ (2 * tid4));  // swizzled position of the 16-byte chunk
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
-      const int h = 2 * tid4 + j;
-      if (h < nh) {
-        const float den = j ? den1 : den0, M = j ? M1 : M0;
-        const long long pidx = q_row(v0 + h) * C + c;
-        m_part[pidx] = den > 0.f ? M * kLn2 : -INFINITY;  // natural-log units of attn_scale * q.k^
-        l_part[pidx] = den;
-      }
+      const float z = zacc[g][j];
+      float4 v;
+      v.x = oacc[2 * g][j] * 16777216.0f - z;
+      v.y = oacc[2 * g][2 + j] * 1048576.0f - z;
+      v.z = oacc[2 * g + 1][j] * 16777216.0f - z;
+      v.w = (oacc[2 * g + 1][2 + j] - oacc[2 * g + 1][j]) * 1048576.0f - z;
+      *reinterpret_cast<float4*>(slab + ((team * 8 + 2 * tid4 + j) * D + 4 * chunk)) = v;
     }
   }
+  __syncthreads();
+  // warp h merges head h: reference M over the teams, weights, denominator, then the weighted sum of the rows
+  const bool direct = STEP && sa.out != nullptr && C == 1;  // one split: its partial is the result (Eq. 5 with one term)
+  if (warp < nh) {
+    const int h = warp;
+    float fw[NTEAM], M = kNoMax, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < NTEAM; ++w) M = fmaxf(M, wml[w * 16 + h]);
+#pragma unroll
+    for (int w = 0; w < NTEAM; ++w) {  // a team that saw no token has m = -1e30 and l = 0
+      fw[w] = ex2(wml[w * 16 + h] - M);
+      den = fmaf(fw[w], wml[w * 16 + 8 + h], den);
+    }
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    const long long pidx = q_row(v0 + h) * C + c;
+    for (int qd = lane; qd < D / 4; qd += 32) {
+      const int phys = (qd & ~7) | ((qd & 7) ^ (h & 6));
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int w = 0; w < NTEAM; ++w) {
+        const float4 v = *reinterpret_cast<const float4*>(slab + ((w * 8 + h) * D + 4 * phys));
+        a.x = fmaf(fw[w], v.x, a.x); a.y = fmaf(fw[w], v.y, a.y); a.z = fmaf(fw[w], v.z, a.z); a.w = fmaf(fw[w], v.w, a.w);
+      }
+      a.x *= inv; a.y *= inv; a.z *= inv; a.w *= inv;
+      if (direct) {  // no partials, no arrival counter, no second pass: the step of a short context ends here
+        const long long orow = q_row(v0 + h) * D + 4 * qd;
+        if (sa.out_fp32) {
+          *reinterpret_cast<float4*>(static_cast<float*>(sa.out) + orow) = a;
+        } else {
+          __half2 hh[2] = {__floats2half2_rn(a.x, a.y), __floats2half2_rn(a.z, a.w)};
+          *reinterpret_cast<uint2*>(static_cast<__half*>(sa.out) + orow) = *reinterpret_cast<uint2*>(hh);
+        }
+      } else {
+        *reinterpret_cast<float4*>(o_part + pidx * D + 4 * qd) = a;
+      }
+    }
+    if (lane == 0 && !direct) {
+      m_part[pidx] = den > 0.f ? M * kLn2 : -INFINITY;  // natural-log units of attn_scale * q.k^
+      l_part[pidx] = den;
+    }
+  }
+  if (direct) return;
 
   // ---------------- fused step: Eq. 5 by the last block of this (sequence, KV head) to get here
   if (STEP && sa.out != nullptr) {
