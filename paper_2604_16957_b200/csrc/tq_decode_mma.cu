@@ -76,10 +76,6 @@ struct Cfg {
   static constexpr int SWZ_SHIFT = NG == 2 ? 2 : (NG == 4 ? 1 : 0);  // chunk' = chunk ^ ((tok >> SHIFT) & (NG - 1))
   static constexpr int SZ = kBlk * NG * 2;          // bytes of one scale or zero array per stage
   static constexpr int STAGE = 2 * PK + 4 * SZ;     // 1280 / 2560 / 5120 / 10240 bytes
-#ifndef TQ_NST
-#define TQ_NST 4
-#endif
-  static constexpr int NST = D == 128 ? TQ_NST : 4;  // stages in a ring
   // Head dimensions above 128 are split over DS warps (a "team") that work on the same token block, each
   // on DW = 128 channels: the accumulators of one warp stay within 128 registers per thread, so two
   // blocks fit an SM at every head dimension.  A team owns one ring; the kernel has NTEAM teams.
@@ -88,15 +84,36 @@ struct Cfg {
   static constexpr int NGW = DW / 32;               // groups per warp
   static constexpr int NTEAM = kWarps / DS;
   static constexpr int MINB = 2;                    // resident blocks per SM
-  static constexpr int PIPE = NTEAM * NST * STAGE;  // 40 KB (D = 64), 80 KB otherwise
-  static constexpr int MERGE = (NTEAM * 16 + NTEAM * 8 * D) * 4;  // merge arrays of the epilogue (inside the ring's memory)
-  static constexpr int BARS = PIPE > MERGE ? PIPE : MERGE;  // offset of the mbarriers: [NTEAM][NST] x 8 bytes
+  static_assert(STAGE == TQ_BLOCK_BYTES(D), "a stage is one cache block");
+  static_assert(kWarps % DS == 0, "teams tile the block");
+  __host__ __device__ static constexpr int swz(int tok) { return (tok >> SWZ_SHIFT) & (NG - 1); }
+};
+
+// Shared memory of one thread block.  Two layouts:
+//  * SEP = false: rings of four stages; the merge arrays of the epilogue and the weights of the fused step's
+//    reduction reuse the rings' memory once every warp is done with its ring (80 KB at d >= 128).
+//  * SEP = true (d = 128): rings of three stages and merge arrays of their own beside them (101 KB), so a warp that
+//    has finished its blocks stores its rows without first waiting for the other warps' rings to drain.  Measured:
+//    0.3 - 0.5 us less per 128K layer and per 32K step; but the larger footprint itself costs a short step (8K:
+//    +0.5 us, measured with padding alone) and three stages cost a batch that runs in several waves 1.5 %, so the
+//    launch takes this layout only for long splits that run in one wave.
+template <int D, bool SEP>
+struct Layout {
+  using Cf = Cfg<D>;
+  static_assert(!SEP || D == 128, "the separate merge arrays fit beside the rings at d = 128 only");
+  static constexpr int NTEAM = Cf::NTEAM, DS = Cf::DS;
+  static constexpr int NST = SEP ? 3 : 4;           // stages in a ring
+  static constexpr int PIPE = NTEAM * NST * Cf::STAGE;  // 40 KB (D = 64), 60 or 80 KB (D = 128), 80 KB otherwise
+  static constexpr int MERGE = (NTEAM * 16 + NTEAM * 8 * D) * 4;  // merge arrays of the epilogue
+  static constexpr int BARS = SEP ? PIPE : (PIPE > MERGE ? PIPE : MERGE);  // offset of the mbarriers: [NTEAM][NST] x 8 bytes
   static constexpr int XCH = BARS + NTEAM * NST * 8;        // score exchange of the teams: [NTEAM][2][DS][32] float4 + flags
   static constexpr int XCH_TEAM = DS > 1 ? 2 * DS * 32 * 16 + 2 * DS * 4 : 0;
-  static constexpr int SMEM = XCH + NTEAM * XCH_TEAM;
-  static_assert(STAGE == TQ_BLOCK_BYTES(D), "a stage is one cache block");
-  static_assert(kWarps % DS == 0 && XCH % 16 == 0 && SMEM % 8 == 0, "teams tile the block");
-  __host__ __device__ static constexpr int swz(int tok) { return (tok >> SWZ_SHIFT) & (NG - 1); }
+  static constexpr int MERGE_OFF = SEP ? XCH + NTEAM * XCH_TEAM : 0;
+  static constexpr int WTS = MERGE_OFF + ((MERGE + 15) & ~15);  // weights of the fused step's reduction
+  static constexpr int WTS_BYTES = 8 * TQ_MAX_SPLITS * 4 + 16 + 8 * 4;  // [8 heads][splits] + ticket + 1 / denominators
+  static constexpr int SMEM = SEP ? WTS + WTS_BYTES : XCH + NTEAM * XCH_TEAM;
+  static_assert(XCH % 16 == 0 && SMEM % 8 == 0, "alignment of the exchange arrays and the page addresses");
+  static_assert(SEP || WTS + WTS_BYTES <= PIPE, "the weights fit the rings");
 };
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -464,12 +481,13 @@ __device__ __noinline__ void quantize_new_row(uint8_t* blk, int row, const __hal
 // fused step, 4 the same over a paged cache, 5 the fused step with a sliding window (general form, contiguous), 6 the
 // overlapped fused step with a sliding window: the block
 // addresses then come from the page table through a per-thread-block table of page addresses.
-template <int D, int MODE, bool HOOK = false>
+template <int D, int MODE, bool HOOK = false, bool SEP = false>
 __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     decode_mma_kernel(tq_kv_cache cache, const __half* __restrict__ q, int H_q, int S_q, float attn_scale, int window,
                       int C, float* __restrict__ o_part, float* __restrict__ m_part, float* __restrict__ l_part,
                       int32_t* status, int stable_blocks_arg, StepArgs sa) {
   using Cf = Cfg<D>;
+  using Ly = Layout<D, SEP>;
   constexpr int NGW = Cf::NGW, DS = Cf::DS, NTEAM = Cf::NTEAM;
   constexpr bool GEN = MODE == 1 || MODE == 2 || MODE == 5, PAGED = MODE == 2 || MODE == 4;
   constexpr bool OVL = MODE == 3 || MODE == 4 || MODE == 6, WIN = MODE == 6;  // WIN: overlapped step over a sliding window
@@ -599,15 +617,15 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   (void)seg_n; (void)blk0b; (void)strideb;
   const int blk1 = t1 > t0 ? (t1 + kBlk - 1) / kBlk : blk0;  // an empty split owns no block
   int nblk = blk1 - blk0 > team ? (blk1 - blk0 - team + NTEAM - 1) / NTEAM : 0;
-  uint8_t* const ring = smem + team * (Cf::NST * Cf::STAGE);
+  uint8_t* const ring = smem + team * (Ly::NST * Cf::STAGE);
   const uint32_t ring_s = static_cast<uint32_t>(__cvta_generic_to_shared(ring));
-  const uint32_t bars = static_cast<uint32_t>(__cvta_generic_to_shared(smem + Cf::BARS)) + team * (Cf::NST * 8);
+  const uint32_t bars = static_cast<uint32_t>(__cvta_generic_to_shared(smem + Ly::BARS)) + team * (Ly::NST * 8);
   if (sub == 0 && lane == 0) {
 #pragma unroll
-    for (int s = 0; s < Cf::NST; ++s) mbar_init(bars + 8 * s, 1);
+    for (int s = 0; s < Ly::NST; ++s) mbar_init(bars + 8 * s, 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     if (DS > 1) {  // the team's two timeout flags (see the score exchange below)
-      int* const xf = reinterpret_cast<int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
+      int* const xf = reinterpret_cast<int*>(smem + Ly::XCH + team * Ly::XCH_TEAM + 2 * DS * 32 * 16);
       xf[0] = xf[1] = 0;
     }
   }
@@ -621,7 +639,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // kernel: they belong to what the caller declared final.  The few blocks the last split attends beyond
   // the stable part are looked up one by one after the wait.)
   const int page0 = blk0 >> pshift;
-  const uint8_t** const page_ptr = reinterpret_cast<const uint8_t**>(smem + Cf::SMEM);
+  const uint8_t** const page_ptr = reinterpret_cast<const uint8_t**>(smem + Ly::SMEM);
   const int npages = (PAGED && blk1 > blk0) ? ((blk1 - 1) >> pshift) - page0 + 1 : 0;
   if (PAGED) {
     for (int i = threadIdx.x; i < npages; i += kThreads) page_ptr[i] = page_base(page0 + i);
@@ -644,11 +662,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     }
   };
 
-  auto issue = [&](int n) { issue_to(n, n % Cf::NST); };
+  auto issue = [&](int n) { issue_to(n, n % Ly::NST); };
 
   // start streaming: the first stages are in flight while q is turned into fragments
 #pragma unroll
-  for (int s = 0; s < Cf::NST - 1; ++s)
+  for (int s = 0; s < Ly::NST - 1; ++s)
     if (s < nblk) issue(s);
   // issue the team's n-th block, if it has one
   auto refill = [&](int n) {
@@ -708,7 +726,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
     if constexpr (DS > 1) {  // through the half of the exchange buffer that block 1 is the first to use
-      float* const qmx = reinterpret_cast<float*>(smem + Cf::XCH + team * Cf::XCH_TEAM + DS * 32 * 16);
+      float* const qmx = reinterpret_cast<float*>(smem + Ly::XCH + team * Ly::XCH_TEAM + DS * 32 * 16);
       qmx[sub * 32 + lane] = mx;
       // (named barriers 9 + team: 1 .. 8 belong to the score exchange of the block loop)
       asm volatile("bar.sync %0, %1;\n" ::"r"(9 + team), "r"(32 * DS) : "memory");
@@ -798,8 +816,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   // tells that every warp is done with the slot of block k - 1, which is refilled after it.  A warp whose
   // wait ran out raises the flag of that block's parity before the barrier (the flags start at 0 and are
   // never lowered: nothing runs after a timeout), and the whole team stops together.
-  float4* const xch = reinterpret_cast<float4*>(smem + Cf::XCH + team * Cf::XCH_TEAM);
-  volatile int* const xflag = reinterpret_cast<volatile int*>(smem + Cf::XCH + team * Cf::XCH_TEAM + 2 * DS * 32 * 16);
+  float4* const xch = reinterpret_cast<float4*>(smem + Ly::XCH + team * Ly::XCH_TEAM);
+  volatile int* const xflag = reinterpret_cast<volatile int*>(smem + Ly::XCH + team * Ly::XCH_TEAM + 2 * DS * 32 * 16);
   // Two-warp teams split the barrier in two: a warp announces its partial on its own barrier (bar.arrive, does
   // not wait) and later waits on its partner's (bar.sync), so whatever does not depend on the scores can be
   // issued in between.  Barrier 1 + 2 * team + sub belongs to warp `sub` of the team: 32 arrivals from its owner
@@ -871,7 +889,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       next += more;
     }
     if (next > 0) {
-      for (int n = k; n < k + Cf::NST - 1; ++n)
+      for (int n = k; n < k + Ly::NST - 1; ++n)
         if (n < nblk) issue(n);
     }
   }
@@ -881,7 +899,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
    // copies of the block step, so the loop carries no slot arithmetic.  It starts on a block whose number is
    // a multiple of four (plain decode: block 0; general form: the first such block behind the masked ones
    // at the old end of the attended range, reached by the one-block loop below).
-   constexpr int NST = Cf::NST;
+   constexpr int NST = Ly::NST;
    if (phase == 0 && k % NST == 0 && k >= plain_lo && k + NST <= plain_hi) {
     const RowMask all{kBlk, 0, kBlk, 0, kBlk};
     uint32_t par = (k / NST) & 1;
@@ -894,7 +912,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     // Timing probe (results are meaningless): the three copies issued above are awaited here, the fourth
     // slot is cleared, and the unrolled loop then runs its arithmetic on whatever the ring holds without
     // waiting for or issuing any copy; the blocks it leaves over are skipped.
-    for (int s = 0; s < Cf::NST - 1; ++s)
+    for (int s = 0; s < Ly::NST - 1; ++s)
       if (s < nblk) wait_stage(bars + 8 * s, 0);
     for (int i = lane; i < Cf::STAGE / 4; i += 32) reinterpret_cast<uint32_t*>(ring + (NST - 1) * Cf::STAGE)[i] = 0;
     __syncwarp();
@@ -926,11 +944,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
    }
   }
   if constexpr (DS > 1) {
-   if (phase == 0 && k % Cf::NST == 0 && k >= plain_lo && k + Cf::NST <= plain_hi) {
+   if (phase == 0 && k % Ly::NST == 0 && k >= plain_lo && k + Ly::NST <= plain_hi) {
     // The same four-block step for a team: the scores of each block are exchanged before its softmax.
-    static_assert(Cf::NST == 4, "the unrolled loop walks a ring of four slots");
+    static_assert(Ly::NST == 4, "the unrolled loop walks a ring of four slots");
     const RowMask all{kBlk, 0, kBlk, 0, kBlk};
-    uint32_t par = (k / Cf::NST) & 1;
+    uint32_t par = (k / Ly::NST) & 1;
     bool ready = mbar_test_wait(bars, par);
     for (; k + 4 <= plain_hi; k += 4) {
 #pragma unroll
@@ -960,14 +978,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   for (; k < nblk && !timed_out; ++k) {
     // Wait for this block's bytes.  The wait is bounded: if the copy never completes (which would take
     // a bad pointer), the warp flags the status word and stops consuming.
-    const bool arrived = wait_stage(bars + 8 * (k % Cf::NST), (k / Cf::NST) & 1, wait_limit);
+    const bool arrived = wait_stage(bars + 8 * (k % Ly::NST), (k / Ly::NST) & 1, wait_limit);
     if (DS == 1) {
       if (!arrived) { timed_out = true; kf = k; break; }
       __syncwarp();  // every lane is done with the slot consumed in the previous iteration: refill it
-      refill(k + Cf::NST - 1);
+      refill(k + Ly::NST - 1);
     }
-    const uint32_t st_s = (k % Cf::NST) * Cf::STAGE;
-    const uint8_t* st = ring + (k % Cf::NST) * Cf::STAGE;
+    const uint32_t st_s = (k % Ly::NST) * Cf::STAGE;
+    const uint8_t* st = ring + (k % Ly::NST) * Cf::STAGE;
     const bool plain = GEN ? static_cast<unsigned>(k - nhead) < nplain : k < nfull;
     auto mask_of_block = [&]() {
       RowMask mk{rem_last, 0, rem_last, 0, rem_last};
@@ -994,7 +1012,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
         block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, zero4, sc);
         block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       }
-      if (GEN && phase == 0 && (k + 1) % Cf::NST == 0 && k + 1 >= plain_lo && k + 1 + Cf::NST <= plain_hi) {
+      if (GEN && phase == 0 && (k + 1) % Ly::NST == 0 && k + 1 >= plain_lo && k + 1 + Ly::NST <= plain_hi) {
         ++k;  // behind the masked blocks of the old end: the four-block loop takes the full ones
         goto fast_blocks;
       }
@@ -1003,10 +1021,10 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       if (plain) block_scores<D, false>(cx, st, st_s, mk, qf, qs, qz, zero4, sc);
       else block_scores<D, true>(cx, st, st_s, mk, qf, qs, qz, zero4, sc);
       if (!exchange(sc, k & 1, arrived)) { timed_out = true; kf = k; break; }
-      refill(k + Cf::NST - 1);
+      refill(k + Ly::NST - 1);
       if (plain) block_softmax_pv<D, false>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
       else block_softmax_pv<D, true>(cx, st_s, mk, sc, oacc, zacc, m0, m1, l0, l1);
-      if (GEN && phase == 0 && (k + 1) % Cf::NST == 0 && k + 1 >= plain_lo && k + 1 + Cf::NST <= plain_hi) {
+      if (GEN && phase == 0 && (k + 1) % Ly::NST == 0 && k + 1 >= plain_lo && k + 1 + Ly::NST <= plain_hi) {
         ++k;
         goto fast_blocks;
       }
@@ -1018,8 +1036,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
     // The copies of blocks kf, kf + 1, kf + 2 of this team may still be in flight into its ring: give each the
     // full bounded time to land before the block reuses the memory, then report.  The partial written below
     // is not valid in that case.
-    for (int n = kf; n < kf + Cf::NST - 1 && n < nblk; ++n)
-      wait_stage(bars + 8 * (n % Cf::NST), (n / Cf::NST) & 1);
+    for (int n = kf; n < kf + Ly::NST - 1 && n < nblk; ++n)
+      wait_stage(bars + 8 * (n % Ly::NST), (n / Ly::NST) & 1);
     if (lane == 0 && status) atomicOr(status, TQ_STATUS_TIMEOUT);
   }
 
@@ -1034,11 +1052,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
       l1 += __shfl_xor_sync(0xffffffffu, l1, off);
     }
   }
-  __syncthreads();  // every warp is done with its ring; the memory is reused below
+  if constexpr (!SEP) __syncthreads();  // every warp is done with its ring; the memory is reused below
   // layout (floats): wml[NTEAM][16] = each team's m[8], l[8] | slab[NTEAM][8 heads][D] = each team's unnormalised
   // output rows.  The 16-byte chunks of a row are XOR-swizzled inside every run of 8 chunks by the head's pair
   // index, which makes both the fragment stores below and the row reads after them conflict free.
-  float* const wml = reinterpret_cast<float*>(smem);
+  float* const wml = reinterpret_cast<float*>(smem + Ly::MERGE_OFF);
   float* const slab = wml + NTEAM * 16;
   if (gid == 0 && sub == 0) {  // the warps of a team hold identical m and l
     wml[team * 16 + 2 * tid4] = m0;
@@ -1116,9 +1134,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
   // ---------------- fused step: Eq. 5 by the last block of this (sequence, KV head) to get here
   if (STEP && sa.out != nullptr) {
-    constexpr int kWts = (Cf::MERGE + 15) & ~15;  // behind the merge arrays, inside the ring's memory
-    static_assert(kWts + kWarps * TQ_MAX_SPLITS * 4 + 16 + kWarps * 4 <= Cf::PIPE, "the weights fit the ring");
-    float* const wts = reinterpret_cast<float*>(smem + kWts) + warp * TQ_MAX_SPLITS;
+    constexpr int kWts = Ly::WTS;  // behind the merge arrays
+        float* const wts = reinterpret_cast<float*>(smem + kWts) + warp * TQ_MAX_SPLITS;
     int* const ticket = reinterpret_cast<int*>(smem + kWts + kWarps * TQ_MAX_SPLITS * 4);
     float* const inv_den = reinterpret_cast<float*>(smem + kWts + kWarps * TQ_MAX_SPLITS * 4 + 16);
     __threadfence();  // this block's partial is visible before its arrival is
@@ -1190,11 +1207,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
 }
 
-template <int D, int MODE, bool HOOK = false>
-cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
-                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
-                   cudaStream_t st) {
-  size_t smem = Cfg<D>::SMEM;
+template <int D, int MODE, bool HOOK = false, bool SEP = false>
+cudaError_t launch_layout(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
+                          float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
+                          cudaStream_t st) {
+  size_t smem = Layout<D, SEP>::SMEM;
   if (MODE == 2 || MODE == 4) {
     // room for the page addresses of the longest split: its blocks, rounded out to whole pages
     const long long span = (window > 0 && window < c.S_cap) ? static_cast<long long>(window) + S_q + 15 : c.S_cap;
@@ -1202,13 +1219,29 @@ cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, floa
     smem += 8 * static_cast<size_t>(per_split / (c.page_tokens / 16) + 2);
     if (smem > 227 * 1024) return cudaErrorInvalidConfiguration;  // tiny pages and too few splits for this capacity
   }
-  const cudaError_t attr =
-      cudaFuncSetAttribute(decode_mma_kernel<D, MODE, HOOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  const cudaError_t attr = cudaFuncSetAttribute(decode_mma_kernel<D, MODE, HOOK, SEP>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (attr != cudaSuccess) return attr;
   const int GV = (H_q / c.H_kv) * S_q;
   dim3 grid(C, c.H_kv * ((GV + 7) / 8), c.B);
-  return launch_kernel(decode_mma_kernel<D, MODE, HOOK>, grid, dim3(kThreads), smem, st, c, q, H_q, S_q, attn_scale, window, C,
-                       o_part, m_part, l_part, status, stable_blocks, sa);
+  return launch_kernel(decode_mma_kernel<D, MODE, HOOK, SEP>, grid, dim3(kThreads), smem, st, c, q, H_q, S_q, attn_scale,
+                       window, C, o_part, m_part, l_part, status, stable_blocks, sa);
+}
+
+template <int D, int MODE, bool HOOK = false>
+cudaError_t launch(const tq_kv_cache& c, const __half* q, int H_q, int S_q, float attn_scale, int window, int C,
+                   float* o_part, float* m_part, float* l_part, int32_t* status, int stable_blocks, const StepArgs& sa,
+                   cudaStream_t st) {
+  if constexpr (D == 128 && !HOOK && (MODE == 0 || MODE == 3)) {
+    // Separate merge arrays (see Layout) where they were measured to pay: every split at least 48 token blocks
+    // of capacity (six per warp) and the whole grid resident at once.
+    const long long blocks = static_cast<long long>(c.B) * c.H_kv * ((H_q / c.H_kv + 7) / 8) * C;
+    if (c.S_cap / C >= 48 * kBlk && blocks <= Cfg<D>::MINB * device_sm_count())
+      return launch_layout<D, MODE, false, true>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status,
+                                                 stable_blocks, sa, st);
+  }
+  return launch_layout<D, MODE, HOOK, false>(c, q, H_q, S_q, attn_scale, window, C, o_part, m_part, l_part, status,
+                                             stable_blocks, sa, st);
 }
 
 template <int D>
