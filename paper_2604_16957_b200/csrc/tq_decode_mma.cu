@@ -92,11 +92,12 @@ struct Cfg {
 // Shared memory of one thread block.  Two layouts:
 //  * SEP = false: rings of four stages; the merge arrays of the epilogue and the weights of the fused step's
 //    reduction reuse the rings' memory once every warp is done with its ring (80 KB at d >= 128).
-//  * SEP = true (d = 128): rings of three stages and merge arrays of their own beside them (101 KB), so a warp that
-//    has finished its blocks stores its rows without first waiting for the other warps' rings to drain.  Measured:
-//    0.3 - 0.5 us less per 128K layer and per 32K step; but the larger footprint itself costs a short step (8K:
-//    +0.5 us, measured with padding alone) and three stages cost a batch that runs in several waves 1.5 %, so the
-//    launch takes this layout only for long splits that run in one wave.
+//  * SEP = true (d = 128): rings of three stages and merge arrays of their own beside them (93 KB; only the
+//    reduction's weights still reuse the rings), so a warp that has finished its blocks stores its rows without
+//    first waiting for the other warps' rings to drain.  Measured: 0.3 - 0.5 us less per 128K layer and per 32K
+//    step; but three stages cost a batch that runs in several waves 1.5 %, and a footprint above 98 KB (two
+//    blocks then need the largest shared-memory carve-out) costs a short step 0.5 us, so the weights stay in the
+//    rings and the launch takes this layout only for long splits that run in one wave.
 template <int D, bool SEP>
 struct Layout {
   using Cf = Cfg<D>;
@@ -109,11 +110,11 @@ struct Layout {
   static constexpr int XCH = BARS + NTEAM * NST * 8;        // score exchange of the teams: [NTEAM][2][DS][32] float4 + flags
   static constexpr int XCH_TEAM = DS > 1 ? 2 * DS * 32 * 16 + 2 * DS * 4 : 0;
   static constexpr int MERGE_OFF = SEP ? XCH + NTEAM * XCH_TEAM : 0;
-  static constexpr int WTS = MERGE_OFF + ((MERGE + 15) & ~15);  // weights of the fused step's reduction
+  static constexpr int WTS = SEP ? 0 : (MERGE + 15) & ~15;  // weights of the fused step's reduction (inside the rings)
   static constexpr int WTS_BYTES = 8 * TQ_MAX_SPLITS * 4 + 16 + 8 * 4;  // [8 heads][splits] + ticket + 1 / denominators
-  static constexpr int SMEM = SEP ? WTS + WTS_BYTES : XCH + NTEAM * XCH_TEAM;
+  static constexpr int SMEM = SEP ? MERGE_OFF + MERGE : XCH + NTEAM * XCH_TEAM;
   static_assert(XCH % 16 == 0 && SMEM % 8 == 0, "alignment of the exchange arrays and the page addresses");
-  static_assert(SEP || WTS + WTS_BYTES <= PIPE, "the weights fit the rings");
+  static_assert(WTS + WTS_BYTES <= PIPE, "the weights fit the rings");
 };
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -1134,8 +1135,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
 
   // ---------------- fused step: Eq. 5 by the last block of this (sequence, KV head) to get here
   if (STEP && sa.out != nullptr) {
-    constexpr int kWts = Ly::WTS;  // behind the merge arrays
-        float* const wts = reinterpret_cast<float*>(smem + kWts) + warp * TQ_MAX_SPLITS;
+    constexpr int kWts = Ly::WTS;  // in the rings' memory: every warp is past the barrier below before they are written
+    float* const wts = reinterpret_cast<float*>(smem + kWts) + warp * TQ_MAX_SPLITS;
     int* const ticket = reinterpret_cast<int*>(smem + kWts + kWarps * TQ_MAX_SPLITS * 4);
     float* const inv_den = reinterpret_cast<float*>(smem + kWts + kWarps * TQ_MAX_SPLITS * 4 + 16);
     __threadfence();  // this block's partial is visible before its arrival is
