@@ -6,8 +6,8 @@
 // from HBM once per head tile.  The path is HBM-bound.  The cache is stored in 16-token blocks that are
 // already in the shared-memory layout this kernel wants (tq.h), so a stage is filled by ONE bulk
 // asynchronous copy (cp.async.bulk, the TMA unit) of a contiguous 2560-byte block (d = 128) issued by
-// one lane and completing on the stage's mbarrier.  Each warp owns a ring of 4 stages and its tokens
-// end to end, so the main loop has no block-wide barrier.  (Head dimensions 256 and 512 are split over
+// one lane and completing on the stage's mbarrier.  Each warp owns a ring of 4 stages (3 in the second
+// shared-memory layout, see Layout) and its tokens end to end, so the main loop has no block-wide barrier.  (Head dimensions 256 and 512 are split over
 // teams of 2 and 4 warps that share a ring and exchange their partial scores once per token block.)
 // Measured on the 128K Llama-shaped layer, the copies alone take 27.9 us with bulk copies against
 // 30.2 us with 16-byte cp.async.  The tensor cores only take the G-packed q.K^T and P.V contractions
@@ -896,9 +896,9 @@ __global__ void __launch_bounds__(kThreads, Cfg<D>::MINB)
   }
   fast_blocks:
   if constexpr (DS == 1) {
-   // Full blocks four at a time: ring slot, barrier and stage offsets are constants of each of the four
-   // copies of the block step, so the loop carries no slot arithmetic.  It starts on a block whose number is
-   // a multiple of four (plain decode: block 0; general form: the first such block behind the masked ones
+   // Full blocks one ring (NST blocks) at a time: ring slot, barrier and stage offsets are constants of each of
+   // the NST copies of the block step, so the loop carries no slot arithmetic.  It starts on a block whose number
+   // is a multiple of NST (plain decode: block 0; general form: the first such block behind the masked ones
    // at the old end of the attended range, reached by the one-block loop below).
    constexpr int NST = Ly::NST;
    if (phase == 0 && k % NST == 0 && k >= plain_lo && k + NST <= plain_hi) {
