@@ -50,6 +50,24 @@ def test_config1_tiny_then_append_one_token(gpu, oracle):
         assert_attention_close(out, oracle.attention(host, q1, sh.alpha), f"tiny/257 C={C}")
 
 
+def test_both_shared_memory_layouts_give_the_same_bits(gpu, oracle):
+    """At d = 128 the launch picks between two shared-memory layouts of the decode kernel by the cache's capacity
+    per split (rings of four stages whose memory the merge reuses, or three stages beside separate merge arrays).
+    Both hand the same token blocks to the same warps and merge in the same order, so the same sequence in a small
+    and in a large cache must give bit-equal partials; both are checked against the oracle as well."""
+    tq, torch = gpu
+    sh, S, C = I.LLAMA, 4096 + 37, 8
+    q = I.make_q(sh, 21)
+    partials = []
+    for S_cap in (4608, 8 * 1024):  # 576 and 1024 tokens of capacity per split: below and above the 768 of the rule
+        host, dev = _both(gpu, oracle, sh, S, 21, S_cap=S_cap)
+        out, (o, m, l), _ = fused_attention(tq, torch, dev, q, sh.alpha, num_splits=C)
+        assert_attention_close(out, oracle.attention(host, q, sh.alpha), f"S_cap={S_cap}")
+        partials.append((o.cpu().numpy(), m.cpu().numpy(), l.cpu().numpy()))
+    for a, b in zip(*partials):
+        assert np.array_equal(a, b)
+
+
 @pytest.mark.parametrize("S,seed", [(1024, 2), (4096, 3), (8192, 4)])
 def test_config2_llama_shape_short_contexts(gpu, oracle, S, seed):
     tq, torch = gpu
