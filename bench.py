@@ -365,8 +365,8 @@ def main():
     # launch-to-launch duration; with --classic the fused-attention kernel is timed in a graph of its own
     kernel_us = decode_classic_us if args.classic else us_per_layer
     achieved = alg_bytes / (kernel_us * 1e-6) / 1e9
-    roofline = {"bound": "hbm", "kernel": "decode_mma_kernel<128, 0>" if args.classic else
-                "decode_mma_kernel<128, 3> (append + attention + reduction in one launch)", "achieved": achieved, "peak": peak, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": "decode_mma_kernel<128, 0, 0, 1>" if args.classic else
+                "decode_mma_kernel<128, 3, 0, 1> (append + attention + reduction in one launch)", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src, "traffic": ncu_traffic_bytes() if S == CONTEXT else None,
                 "algorithmic_bytes_per_launch": alg_bytes, "us_per_launch": kernel_us,
                 "frac_of_nominal_8TBs": achieved / HBM_NOMINAL_GBS}
