@@ -258,13 +258,13 @@ int tq_sdpa_int4_step_window(const tq_kv_cache* cache /* host */, const void* k_
 size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, int32_t num_splits);
 /*
  * Split count that tq_sdpa_int4_step and tq_sdpa_int4_decode_overlapped pick for num_splits = 0 (host function).
- * Like tq_auto_splits, but when one wave of thread blocks fills the GPU it leaves one resident slot per
- * (sequence, KV head) unused: launches of these entry points overlap their predecessor, and with every slot
- * taken the blocks that finish a launch last (those that also reduce the partials) hold up the first blocks
- * of the next one.  Measured on the 128K Llama-shaped step: 36.5 us per layer with 37 splits, 32.3 us with 36.
- * The spare slots are a share (sequences x KV heads) / slots of the machine: they are left only where that
- * share is at most 1/32 (8 KV heads on 296 slots; with 16 KV heads the d = 256 shape measured 39.0 us with
- * the spare slots and 37.4 us without).  For a batch (more than a quarter of the slots per split) it picks about
+ * Like tq_auto_splits, but when one wave of thread blocks would fill the GPU it leaves an eighth of the resident
+ * slots (at least one per (sequence, KV head)) unused: launches of these entry points overlap their predecessor,
+ * and with every slot taken the blocks that finish a launch last (those that also reduce the partials) hold up
+ * the first blocks of the next one.  Measured on the 128K Llama-shaped step (8 KV heads, 296 slots), us per layer
+ * by number of splits: 37: 34.7, 36: 30.2, 32: 29.9, 28: 29.9, 24: 30.5; the 32K step: 36: 11.9, 32: 11.6, 28: 11.8.
+ * The slots are left only where (sequences x KV heads) is at most 1/32 of them (with 16 KV heads the d = 256
+ * shape measured 39.0 us with one spare slot per KV head and 37.4 us without).  For a batch (more than a quarter of the slots per split) it picks about
  * three and a half waves of thread blocks instead of tq_auto_splits' four: the overlap fills a launch's tail.
  * Up to 1024 tokens it picks one split: with num_splits = 1 the step's thread blocks write `out` themselves
  * (Eq. 5 with a single term), without partials, arrival counter or second pass.
