@@ -263,6 +263,8 @@ size_t tq_step_workspace_bytes(int32_t B, int32_t H_kv, int32_t H_q, int32_t d, 
  * and with every slot taken the blocks that finish a launch last (those that also reduce the partials) hold up
  * the first blocks of the next one.  Measured on the 128K Llama-shaped step (8 KV heads, 296 slots), us per layer
  * by number of splits: 37: 34.7, 36: 30.2, 32: 29.9, 28: 29.9, 24: 30.5; the 32K step: 36: 11.9, 32: 11.6, 28: 11.8.
+ * (A step that declares no stable part overlaps nothing: there every slot is worth taking, 35.8 us per layer with
+ * 37 splits against 37.5 with 32, and tq_auto_splits gives the better count.)
  * The slots are left only where (sequences x KV heads) is at most 1/32 of them (with 16 KV heads the d = 256
  * shape measured 39.0 us with one spare slot per KV head and 37.4 us without).  For a batch (more than a quarter of the slots per split) it picks about
  * three and a half waves of thread blocks instead of tq_auto_splits' four: the overlap fills a launch's tail.
