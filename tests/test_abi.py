@@ -67,6 +67,29 @@ def test_host_side_helpers(lib):
     assert tq.tq_auto_splits(1, 8, 64, 128, 100) == 1
 
 
+def test_split_policy_of_the_step(lib):
+    """tq_auto_splits_step on a machine that cannot be asked (no device: 148 SMs, 296 resident slots assumed):
+    within [1, TQ_MAX_SPLITS], never splits shorter than the stated minimum, one split up to 1K tokens, and an
+    eighth of the slots left free where (sequences x KV heads) is at most 1/32 of them."""
+    from paper_2604_16957_b200 import tq
+    slots = 296
+    for B, H_kv, H_q in ((1, 8, 64), (1, 4, 32), (1, 1, 8), (1, 2, 16), (1, 16, 32), (2, 8, 64), (16, 8, 64), (64, 8, 64)):
+        base = B * H_kv * ((H_q // H_kv + 7) // 8)
+        for n in (1, 100, 1024, 1025, 4096, 8192, 32768, 131072, 1 << 20):
+            c = tq.tq_auto_splits_step(B, H_kv, H_q, 128, n)
+            plain = tq.tq_auto_splits(B, H_kv, H_q, 128, n)
+            assert 1 <= c <= 256 and c <= max(1, plain)
+            if n <= 1024:
+                assert c == 1
+            else:
+                assert c <= max(1, n // 512)
+            if 32 * base <= slots and c > 1:
+                assert c * base <= slots - max(base, slots // 8)
+    assert tq.tq_auto_splits_step(1, 8, 64, 128, 131072) == 32 and tq.tq_auto_splits(1, 8, 64, 128, 131072) == 37
+    assert tq.tq_auto_splits_step(1, 16, 32, 256, 32768) == 18       # 16 KV heads: no spare slots
+    assert tq.tq_auto_splits_step(1, 0, 8, 128, 4096) == 1           # nonsense shapes give 1, not a crash
+
+
 def test_argument_validation_without_gpu(lib):
     from paper_2604_16957_b200 import tq
     lib.tq_result_string.restype = C.c_char_p
